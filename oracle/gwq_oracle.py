@@ -1,0 +1,259 @@
+"""CPU checker for the GWQ mixed-precision linear layer (arXiv 2411.00850).
+
+TEST INFRASTRUCTURE ONLY.  This file is the slow, plain definition that the
+CUDA library is compared against.  It shares no code with the CUDA path and
+must never be imported by it; only the test-suite, the smoke check and the
+CPU-baseline leg of the benchmark call it.
+
+Everything is NumPy in float64 (the inputs are fp16 / fp32 values, all of
+which are exact in float64).  The method is an encoding followed by a product,
+so the functions below take the paper's steps in the paper's order:
+
+  Section 3.2, Eq. "o"   select_outliers   mask of the largest |gradient|
+  Section 3.2, Eq. "s"   group_stats       per-group scale
+  Section 3.2, Eq. "z"   group_stats       per-group zero-point
+  Section 3.2, Eq. "q"   quantize_codes    round-to-nearest codes
+  Section 3.2, Eq. "w"   dequantize        s * (q - z), plus the kept outliers
+  Abstract / Section 1   linear            y = x (deq(Wq) + S)^T, outliers in FP16
+
+Readings taken where the paper is silent, garbled or ambiguous (each is a
+choice of this implementation, listed again in the design notes):
+
+  R1  Eq. "s" prints the denominator as 2^{b-1}; read as 2^b - 1 (the number of
+      steps between code 0 and code 2^b-1), otherwise most codes are unused.
+  R2  Eq. "z" gives a real number; the stored zero-point is
+      clip(rint(-lo / s), 0, 2^b - 1).
+  R3  The range used for a group always contains 0: lo = min(0, min w),
+      hi = max(0, max w); only then is an integer zero-point in range.
+  R4  "round" is round-half-to-even on the float64 quotient.
+  R5  Codes are clipped to [0, 2^b - 1].
+  R6  The scale is stored in fp16, rounded toward +inf from the float64
+      quotient, so that (hi - lo) / s never exceeds 2^b - 1.
+  R7  A group with hi == lo (all remaining entries zero, or every entry an
+      outlier) gets s = 1, z = 0.
+  R8  Eq. "o" (>= quantile) is read as an exact count: the
+      ceil(frac * numel) entries of largest |g| in the matrix, equal
+      magnitudes resolved in favour of the lower flat index n*K + k.  The
+      order on magnitudes is the order of the IEEE-754 bit patterns of |g|
+      (so -0 == +0 < finite < inf < NaN).
+  R9  Groups are runs of `group` consecutive input features (k) inside one
+      output row; outliers take no part in min / max and get code z, so their
+      dense reconstruction is exactly 0.
+  R10 The product accumulates in float64 here; the kept outliers enter with
+      their exact fp16 values.
+
+Parity status: every function below is pinned by tests that do not restate its
+formula (brute force, closed forms, invariants, library special cases); see
+tests/test_oracle_*.py.  The paper prints no worked numeric example, and never
+defines its "GWQ-O"/"GWQ-R" variants nor the storage format behind its average
+bit-widths: the bit layout of `pack_codes` is this project's own documented
+format (parity with the paper unpinned for the format alone).
+"""
+from __future__ import annotations
+
+import math
+
+import numpy as np
+
+__all__ = [
+    "outlier_count",
+    "select_outliers",
+    "outlier_mask",
+    "group_stats",
+    "quantize_codes",
+    "pack_codes",
+    "unpack_codes",
+    "dequantize",
+    "linear",
+    "quantize_layer",
+]
+
+
+# --------------------------------------------------------------------------
+# Eq. "o": outlier location
+# --------------------------------------------------------------------------
+def outlier_count(frac: float, numel: int) -> int:
+    """Number of kept outliers: ceil(frac * numel) in IEEE double, clamped."""
+    if not (0.0 <= frac <= 1.0):
+        raise ValueError("frac must lie in [0, 1]")
+    k = int(math.ceil(float(frac) * float(numel)))
+    return max(0, min(int(numel), k))
+
+
+def _abs_key(G: np.ndarray) -> np.ndarray:
+    """Bit pattern of |g| as an unsigned integer; its integer order is the
+    order used for ranking (reading R8)."""
+    g = np.ascontiguousarray(G, dtype=np.float32)
+    return g.view(np.uint32).reshape(-1) & np.uint32(0x7FFFFFFF)
+
+
+def select_outliers(W: np.ndarray, G: np.ndarray, frac: float):
+    """Eq. "o" with reading R8.
+
+    W: fp16 [N, K]; G: fp32 [N, K].
+    Returns (row_ptr int32 [N+1], col_idx int32 [nnz], val uint16 [nnz]): the
+    CSR matrix S holding W's bit patterns at the selected positions, columns
+    ascending inside every row.
+    """
+    if W.shape != G.shape or W.ndim != 2:
+        raise ValueError("W and G must be 2-D and of equal shape")
+    if W.dtype != np.float16 or G.dtype != np.float32:
+        raise ValueError("W must be fp16 and G fp32")
+    N, K = W.shape
+    numel = N * K
+    k_out = outlier_count(frac, numel)
+    key = _abs_key(G)
+    flat = np.arange(numel, dtype=np.int64)
+    # sort by magnitude descending, then flat index ascending
+    order = np.lexsort((flat, -key.astype(np.int64)))
+    chosen = np.sort(order[:k_out])
+    rows = chosen // K
+    cols = chosen % K
+    row_ptr = np.zeros(N + 1, dtype=np.int64)
+    np.add.at(row_ptr, rows + 1, 1)
+    row_ptr = np.cumsum(row_ptr)
+    val = np.ascontiguousarray(W).view(np.uint16).reshape(-1)[chosen]
+    return row_ptr.astype(np.int32), cols.astype(np.int32), val.astype(np.uint16)
+
+
+def outlier_mask(row_ptr: np.ndarray, col_idx: np.ndarray, N: int, K: int) -> np.ndarray:
+    """Dense boolean mask O [N, K] of the CSR pattern."""
+    mask = np.zeros((N, K), dtype=bool)
+    counts = np.diff(row_ptr.astype(np.int64))
+    rows = np.repeat(np.arange(N, dtype=np.int64), counts)
+    mask[rows, col_idx.astype(np.int64)] = True
+    return mask
+
+
+# --------------------------------------------------------------------------
+# Eqs. "s", "z": per-group scale and zero-point
+# --------------------------------------------------------------------------
+def _fp16_round_up(v: np.ndarray) -> np.ndarray:
+    """Smallest fp16 value >= v (v float64, finite, >= 0)."""
+    h = v.astype(np.float16)
+    low = h.astype(np.float64) < v
+    h_up = np.nextafter(h, np.float16(np.inf))
+    return np.where(low, h_up, h).astype(np.float16)
+
+
+def group_stats(W: np.ndarray, mask: np.ndarray, bits: int, group: int):
+    """Eqs. "s" and "z" with readings R1-R3, R6, R7, R9.
+
+    Returns (scales fp16 [N, K/group], zeros uint8 [N, K/group]).
+    """
+    N, K = W.shape
+    if K % group != 0:
+        raise ValueError("K must be a multiple of the group size")
+    if not np.all(np.isfinite(W)):
+        raise ValueError("non-finite weight")
+    qmax = float(2 ** bits - 1)
+    ng = K // group
+    w = W.astype(np.float64).reshape(N, ng, group)
+    m = mask.reshape(N, ng, group)
+    lo = np.where(m, np.inf, w).min(axis=2)
+    hi = np.where(m, -np.inf, w).max(axis=2)
+    lo = np.minimum(lo, 0.0)
+    hi = np.maximum(hi, 0.0)
+    flat_range = hi == lo
+    s64 = (hi - lo) / qmax
+    s16 = _fp16_round_up(np.where(flat_range, 1.0, s64))
+    s = s16.astype(np.float64)
+    z = np.clip(np.rint(-lo / s), 0.0, qmax)
+    z = np.where(flat_range, 0.0, z)
+    return s16, z.astype(np.uint8)
+
+
+# --------------------------------------------------------------------------
+# Eq. "q": codes
+# --------------------------------------------------------------------------
+def quantize_codes(W, mask, scales, zeros, bits: int, group: int) -> np.ndarray:
+    """Eq. "q" with readings R4, R5, R9.  Returns codes uint8 [N, K]."""
+    N, K = W.shape
+    qmax = float(2 ** bits - 1)
+    s = np.repeat(scales.astype(np.float64), group, axis=1)
+    z = np.repeat(zeros.astype(np.float64), group, axis=1)
+    q = np.clip(np.rint(W.astype(np.float64) / s) + z, 0.0, qmax)
+    q = np.where(mask, z, q)
+    return q.astype(np.uint8)
+
+
+# --------------------------------------------------------------------------
+# Storage format (this project's own; the paper specifies none)
+# --------------------------------------------------------------------------
+def pack_codes(codes: np.ndarray, bits: int) -> np.ndarray:
+    """Pack codes [N, K] into little-endian 32-bit words.
+
+    Every run of 32 consecutive columns of a row is one little-endian integer
+    of 32*bits bits, column 32r+i occupying bits [bits*i, bits*(i+1)); the
+    integer is stored as `bits` consecutive uint32 words, least significant
+    first.  (For 4 bits this is simply: word t holds columns 8t..8t+7, column
+    8t+i in bits [4i, 4i+4).  For 3 bits, codes 10 and 21 of a run straddle
+    two words.)  Returns uint32 [N, K*bits/32].
+    """
+    N, K = codes.shape
+    if K % 32 != 0:
+        raise ValueError("K must be a multiple of 32")
+    if codes.max(initial=0) > 2 ** bits - 1:
+        raise ValueError("code out of range")
+    out = np.zeros((N, K // 32, bits), dtype=np.uint32)
+    c = codes.reshape(N, K // 32, 32).astype(np.uint64)
+    for i in range(32):
+        pos = bits * i
+        word, off = divmod(pos, 32)
+        out[:, :, word] |= ((c[:, :, i] << np.uint64(off)) & np.uint64(0xFFFFFFFF)).astype(np.uint32)
+        if off + bits > 32:
+            out[:, :, word + 1] |= (c[:, :, i] >> np.uint64(32 - off)).astype(np.uint32)
+    return out.reshape(N, K * bits // 32)
+
+
+def unpack_codes(words: np.ndarray, bits: int, K: int) -> np.ndarray:
+    """Inverse of pack_codes.  Returns codes uint8 [N, K]."""
+    N = words.shape[0]
+    w = words.reshape(N, K // 32, bits).astype(np.uint64)
+    codes = np.zeros((N, K // 32, 32), dtype=np.uint8)
+    m = np.uint64(2 ** bits - 1)
+    for i in range(32):
+        pos = bits * i
+        word, off = divmod(pos, 32)
+        v = w[:, :, word] >> np.uint64(off)
+        if off + bits > 32:
+            v = v | (w[:, :, word + 1] << np.uint64(32 - off))
+        codes[:, :, i] = (v & m).astype(np.uint8)
+    return codes.reshape(N, K)
+
+
+# --------------------------------------------------------------------------
+# Eq. "w": reconstruction, and the layer product
+# --------------------------------------------------------------------------
+def dequantize(codes, scales, zeros, group: int, row_ptr, col_idx, val) -> np.ndarray:
+    """Eq. "w" plus the kept FP16 outliers: w_hat = s*(q - z) + S, float64 [N,K]."""
+    N, K = codes.shape
+    s = np.repeat(scales.astype(np.float64), group, axis=1)
+    z = np.repeat(zeros.astype(np.float64), group, axis=1)
+    w_hat = s * (codes.astype(np.float64) - z)
+    counts = np.diff(row_ptr.astype(np.int64))
+    rows = np.repeat(np.arange(N, dtype=np.int64), counts)
+    S = np.zeros((N, K), dtype=np.float64)
+    S[rows, col_idx.astype(np.int64)] = val.view(np.float16).astype(np.float64)
+    return w_hat + S
+
+
+def linear(x: np.ndarray, w_hat: np.ndarray):
+    """y = x w_hat^T in float64, and bound = |x| |w_hat|^T (the per-output sum
+    of |x_k * w_hat_k| that the floating-point tolerance is stated against)."""
+    x64 = np.asarray(x, dtype=np.float64)
+    y = x64 @ w_hat.T
+    bound = np.abs(x64) @ np.abs(w_hat).T
+    return y, bound
+
+
+def quantize_layer(W, G, frac: float, bits: int, group: int) -> dict:
+    """All encoding steps in order; returns every intermediate by name."""
+    N, K = W.shape
+    row_ptr, col_idx, val = select_outliers(W, G, frac)
+    mask = outlier_mask(row_ptr, col_idx, N, K)
+    scales, zeros = group_stats(W, mask, bits, group)
+    codes = quantize_codes(W, mask, scales, zeros, bits, group)
+    words = pack_codes(codes, bits)
+    return dict(N=N, K=K, bits=bits, group=group, row_ptr=row_ptr, col_idx=col_idx,
+                val=val, mask=mask, scales=scales, zeros=zeros, codes=codes, words=words)
