@@ -1,0 +1,130 @@
+/*
+ * gwq.h - C ABI of the GWQ mixed-precision linear layer for NVIDIA B200 (sm_100a).
+ *
+ * Method: "GWQ: Gradient-Aware Weight Quantization for Large Language Models"
+ * (arXiv 2411.00850).  A weight matrix W [N, K] (N output features, K input
+ * features) is split by the magnitude of a calibration gradient G of the same
+ * shape: the largest ~1 % of |g| mark "outlier" weights that stay in FP16
+ * (Section 3.2, Eq. "o"; Section 1); all other weights are quantized to b = 3 or
+ * 4 bits with one scale s and one zero-point z per group of consecutive input
+ * features (Section 3.2, Eqs. "s", "z", "q"), and the layer computes
+ *
+ *        y = x (s (q - z) + S)^T                      (Section 3.2, Eq. "w")
+ *
+ * where S is the sparse FP16 outlier matrix.
+ *
+ * Conventions for every call
+ *  - Pointers are DEVICE pointers unless an argument says "host".
+ *  - `stream` is a cudaStream_t passed as void* (NULL = default stream).
+ *  - Caller-owned buffers (W, G, x, y) are never freed by the library and only
+ *    y is written.  Objects returned through `out` are owned by the library and
+ *    released with gwq_free().
+ *  - Nothing aborts or throws: every failure is a gwq_status.  There is no CPU
+ *    fallback: without a CUDA device the calls return GWQ_ERR_CUDA.
+ *  - Matrices are row-major.  fp16 / bf16 data are passed as uint16_t bit
+ *    patterns.  Device pointers must be 16-byte aligned.
+ */
+#ifndef GWQ_H_
+#define GWQ_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  GWQ_OK = 0,
+  GWQ_ERR_INVALID_ARG = 1, /* null or misaligned pointer, non-positive size, frac outside [0,1] */
+  GWQ_ERR_UNSUPPORTED = 2, /* bits not in {3,4}, group not in {64,128}, K % group != 0, ...    */
+  GWQ_ERR_ALLOC = 3,       /* device or host allocation failed                                  */
+  GWQ_ERR_NONFINITE = 4,   /* W holds an inf or NaN                                             */
+  GWQ_ERR_TIMEOUT = 5,     /* a bounded device-side wait ran out (kernel returned early)        */
+  GWQ_ERR_CUDA = 6         /* a CUDA runtime call failed                                        */
+} gwq_status;
+
+typedef enum { GWQ_F16 = 0, GWQ_BF16 = 1, GWQ_F32 = 2 } gwq_dtype;
+
+/* Sparse FP16 outlier matrix S in CSR form (Section 3.2, Eq. "o": the mask O; the
+ * values are the original FP16 weights at the masked positions).                    */
+typedef struct gwq_outliers {
+  uint32_t tag;      /* library-private type tag, do not modify                          */
+  int32_t N, K;      /* shape of W                                                       */
+  int64_t nnz;       /* = ceil(frac * N * K)                                             */
+  int32_t* row_ptr;  /* device [N+1]                                                     */
+  int32_t* col_idx;  /* device [nnz], strictly ascending inside each row                 */
+  uint16_t* val;     /* device [nnz], fp16 bit patterns copied from W                    */
+} gwq_outliers;
+
+/* Packed layer.
+ * codes: every run of 32 consecutive columns of a row is one little-endian integer of
+ *   32*bits bits, column 32r+i in bits [bits*i, bits*i+bits), stored as `bits`
+ *   consecutive uint32 words (least significant first).  Row n starts at word
+ *   n * K*bits/32.  For 4 bits: word t of a row holds columns 8t..8t+7, column 8t+i in
+ *   bits [4i, 4i+4).
+ * scales: fp16 [N, K/group]; zeros: uint8 [N, K/group], each in [0, 2^bits - 1].
+ * An outlier position stores the code z of its group, so its dense term is exactly 0. */
+typedef struct gwq_packed {
+  uint32_t tag;
+  int32_t N, K, bits, group;
+  uint32_t* codes;
+  uint16_t* scales;
+  uint8_t* zeros;
+  gwq_outliers* S; /* owned by this object                                               */
+  void* priv;      /* kernel-private derived tables and staging; opaque                  */
+} gwq_packed;
+
+/* Outlier location (Section 3.2, Eq. "o"; Figure 2: "the top 1% with the largest |g|").
+ * Selects exactly ceil(frac * N*K) entries (the product evaluated in IEEE double) with
+ * the largest |G| over the whole matrix; entries of equal magnitude are taken in
+ * ascending flat index n*K + k.  Magnitudes are ordered by the bit pattern of |g|
+ * (so -0 == +0 < finite < inf < NaN); G may hold any bit pattern.
+ *   W_f16 [N,K] fp16, G_f32 [N,K] fp32: device, caller-owned, read only.
+ *   *out: new library-owned CSR object.  The call synchronises `stream` before it
+ *   returns.
+ * Errors: INVALID_ARG (null / misaligned pointer, N or K <= 0, N*K >= 2^31, frac outside
+ *   [0,1]), UNSUPPORTED (K % 32 != 0), ALLOC, CUDA.  On error *out is NULL.             */
+gwq_status gwq_select_outliers(const uint16_t* W_f16, const float* G_f32, int32_t N, int32_t K,
+                               double frac, gwq_outliers** out, void* stream);
+
+/* Group-wise asymmetric quantization of the non-outliers (Section 3.2, Eqs. "s", "z",
+ * "q") and bit-packing.  Per (row, group of `group` consecutive k), over non-outlier
+ * entries only: lo = min(0, min w), hi = max(0, max w); s = (hi - lo) / (2^bits - 1)
+ * rounded up to fp16 (the paper's printed denominator 2^{b-1} is read as 2^b - 1);
+ * z = clip(rint(-lo / s), 0, 2^bits - 1); q = clip(rint(w / s) + z, 0, 2^bits - 1),
+ * round-half-to-even; outliers get q = z.  A group with hi == lo gets s = 1, z = 0.
+ *   W_f16: device, caller-owned, read only.
+ *   S: from gwq_select_outliers with the same N, K; on success its ownership moves into
+ *      *out (do not free it separately); on failure it stays with the caller.
+ *   *out: new library-owned packed layer.  Synchronises `stream` before returning.
+ * Errors: INVALID_ARG, UNSUPPORTED (bits, group, K % group, K > 131072), NONFINITE (W has
+ *   inf/NaN), ALLOC, CUDA.  On error *out is NULL.                                       */
+gwq_status gwq_pack(const uint16_t* W_f16, gwq_outliers* S, int32_t N, int32_t K, int32_t bits,
+                    int32_t group, gwq_packed** out, void* stream);
+
+/* Forward product y = x (s (q - z) + S)^T (Section 3.2, Eq. "w", outliers in FP16).
+ *   x: device [M, K], fp16 or bf16 (x_dtype).  y: device [M, N], y_dtype one of
+ *   F16 / BF16 / F32.  Accumulation is FP32.  M >= 1; M <= 32 takes the bandwidth-bound
+ *   streaming path, larger M the tensor-core path.
+ *   Asynchronous on `stream`; argument errors are returned immediately.
+ * Errors: INVALID_ARG, UNSUPPORTED (x_dtype F32), CUDA (launch failure).               */
+gwq_status gwq_linear(const gwq_packed* P, const void* x, gwq_dtype x_dtype, int32_t M, void* y,
+                      gwq_dtype y_dtype, void* stream);
+
+/* Same product with HOST buffers: copies x_host [M,K] to a staging buffer kept inside P,
+ * runs gwq_linear, copies y back into y_host [M,N] and synchronises `stream`.
+ * For best copy speed the host buffers should be page-locked.  The staging buffers grow
+ * on demand (cudaMalloc) and are shared by all calls on P: not re-entrant per P.       */
+gwq_status gwq_linear_host(gwq_packed* P, const void* x_host, gwq_dtype x_dtype, int32_t M,
+                           void* y_host, gwq_dtype y_dtype, void* stream);
+
+/* Releases a gwq_outliers* or a gwq_packed* (and everything it owns).  NULL is a no-op. */
+void gwq_free(void* obj);
+
+/* Static, NUL-terminated name of a status code.                                        */
+const char* gwq_status_string(gwq_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GWQ_H_ */

@@ -1,0 +1,46 @@
+// Shared host/device helpers of the GWQ library (internal; not part of the ABI).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/gwq.h"
+
+#define GWQ_TAG_OUTLIERS 0x4F515747u /* "GWQO" */
+#define GWQ_TAG_PACKED 0x50515747u   /* "GWQP" */
+
+// Needs a local `gwq_status st` and a label `fail`.
+#define GWQ_CUDA_TRY(expr)                                                    \
+  do {                                                                        \
+    cudaError_t e__ = (expr);                                                 \
+    if (e__ != cudaSuccess) {                                                 \
+      (void)cudaGetLastError();                                               \
+      st = (e__ == cudaErrorMemoryAllocation) ? GWQ_ERR_ALLOC : GWQ_ERR_CUDA; \
+      goto fail;                                                              \
+    }                                                                         \
+  } while (0)
+
+// Kernel-private part of a packed layer.
+struct gwq_priv {
+  uint16_t* col16;       // outlier columns narrowed to 16 bit (NULL when K > 65536)
+  void* x_stage;         // staging for gwq_linear_host
+  void* y_stage;
+  size_t x_stage_bytes;
+  size_t y_stage_bytes;
+  int32_t* dev_status;   // device status word written by bounded waits
+  int sm_count;
+};
+
+static inline bool gwq_aligned16(const void* p) {
+  return (reinterpret_cast<uintptr_t>(p) & 15u) == 0;
+}
+
+// Kernel launchers implemented in the other translation units.
+gwq_status gwq_launch_simt(const gwq_packed* P, const void* x, gwq_dtype xd, int M, void* y,
+                           gwq_dtype yd, cudaStream_t stream);
+gwq_status gwq_launch_decode(const gwq_packed* P, const void* x, gwq_dtype xd, int M, void* y,
+                             gwq_dtype yd, cudaStream_t stream);
+gwq_status gwq_launch_prefill(const gwq_packed* P, const void* x, gwq_dtype xd, int M, void* y,
+                              gwq_dtype yd, cudaStream_t stream);
