@@ -1,0 +1,96 @@
+// Entry points that are not kernels of their own: dispatch of the forward product,
+// the host-buffer variant, object release and status names.
+#include "common.cuh"
+
+static size_t dtype_bytes(gwq_dtype d) { return d == GWQ_F32 ? 4 : 2; }
+
+extern "C" gwq_status gwq_linear(const gwq_packed* P, const void* x, gwq_dtype xd, int32_t M, void* y,
+                                 gwq_dtype yd, void* stream_) {
+  if (!P || P->tag != GWQ_TAG_PACKED || !P->S || !P->priv || !x || !y || M <= 0) return GWQ_ERR_INVALID_ARG;
+  if (xd != GWQ_F16 && xd != GWQ_BF16) return GWQ_ERR_UNSUPPORTED;
+  if (yd != GWQ_F16 && yd != GWQ_BF16 && yd != GWQ_F32) return GWQ_ERR_INVALID_ARG;
+  if (!gwq_aligned16(x) || !gwq_aligned16(y)) return GWQ_ERR_INVALID_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  return gwq_launch_simt(P, x, xd, M, y, yd, stream);
+}
+
+extern "C" gwq_status gwq_linear_host(gwq_packed* P, const void* x_host, gwq_dtype xd, int32_t M,
+                                      void* y_host, gwq_dtype yd, void* stream_) {
+  if (!P || P->tag != GWQ_TAG_PACKED || !P->priv || !x_host || !y_host || M <= 0) return GWQ_ERR_INVALID_ARG;
+  if (xd != GWQ_F16 && xd != GWQ_BF16) return GWQ_ERR_UNSUPPORTED;
+  if (yd != GWQ_F16 && yd != GWQ_BF16 && yd != GWQ_F32) return GWQ_ERR_INVALID_ARG;
+  gwq_priv* pv = static_cast<gwq_priv*>(P->priv);
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  const size_t xb = (size_t)M * P->K * dtype_bytes(xd), yb = (size_t)M * P->N * dtype_bytes(yd);
+  gwq_status st = GWQ_OK;
+  if (pv->x_stage_bytes < xb) {
+    GWQ_CUDA_TRY(cudaStreamSynchronize(stream));
+    if (pv->x_stage) cudaFree(pv->x_stage);
+    pv->x_stage = nullptr;
+    pv->x_stage_bytes = 0;
+    GWQ_CUDA_TRY(cudaMalloc(&pv->x_stage, xb));
+    pv->x_stage_bytes = xb;
+  }
+  if (pv->y_stage_bytes < yb) {
+    GWQ_CUDA_TRY(cudaStreamSynchronize(stream));
+    if (pv->y_stage) cudaFree(pv->y_stage);
+    pv->y_stage = nullptr;
+    pv->y_stage_bytes = 0;
+    GWQ_CUDA_TRY(cudaMalloc(&pv->y_stage, yb));
+    pv->y_stage_bytes = yb;
+  }
+  GWQ_CUDA_TRY(cudaMemcpyAsync(pv->x_stage, x_host, xb, cudaMemcpyHostToDevice, stream));
+  st = gwq_linear(P, pv->x_stage, xd, M, pv->y_stage, yd, stream);
+  if (st != GWQ_OK) return st;
+  GWQ_CUDA_TRY(cudaMemcpyAsync(y_host, pv->y_stage, yb, cudaMemcpyDeviceToHost, stream));
+  GWQ_CUDA_TRY(cudaStreamSynchronize(stream));
+  return GWQ_OK;
+fail:
+  return st;
+}
+
+static void free_outliers(gwq_outliers* S) {
+  if (!S) return;
+  if (S->row_ptr) cudaFree(S->row_ptr);
+  if (S->col_idx) cudaFree(S->col_idx);
+  if (S->val) cudaFree(S->val);
+  S->tag = 0;
+  delete S;
+}
+
+extern "C" void gwq_free(void* obj) {
+  if (!obj) return;
+  const uint32_t tag = *static_cast<const uint32_t*>(obj);
+  if (tag == GWQ_TAG_OUTLIERS) {
+    free_outliers(static_cast<gwq_outliers*>(obj));
+  } else if (tag == GWQ_TAG_PACKED) {
+    gwq_packed* P = static_cast<gwq_packed*>(obj);
+    if (P->codes) cudaFree(P->codes);
+    if (P->scales) cudaFree(P->scales);
+    if (P->zeros) cudaFree(P->zeros);
+    free_outliers(P->S);
+    gwq_priv* pv = static_cast<gwq_priv*>(P->priv);
+    if (pv) {
+      if (pv->col16) cudaFree(pv->col16);
+      if (pv->x_stage) cudaFree(pv->x_stage);
+      if (pv->y_stage) cudaFree(pv->y_stage);
+      if (pv->dev_status) cudaFree(pv->dev_status);
+      delete pv;
+    }
+    P->tag = 0;
+    delete P;
+  }
+}
+
+extern "C" const char* gwq_status_string(gwq_status s) {
+  switch (s) {
+    case GWQ_OK: return "GWQ_OK";
+    case GWQ_ERR_INVALID_ARG: return "GWQ_ERR_INVALID_ARG";
+    case GWQ_ERR_UNSUPPORTED: return "GWQ_ERR_UNSUPPORTED";
+    case GWQ_ERR_ALLOC: return "GWQ_ERR_ALLOC";
+    case GWQ_ERR_NONFINITE: return "GWQ_ERR_NONFINITE";
+    case GWQ_ERR_TIMEOUT: return "GWQ_ERR_TIMEOUT";
+    case GWQ_ERR_CUDA: return "GWQ_ERR_CUDA";
+  }
+  return "GWQ_ERR_UNKNOWN";
+}

@@ -1,0 +1,189 @@
+// Group-wise asymmetric quantization of the non-outliers and bit-packing
+// (Section 3.2, Eqs. "s", "z", "q"; outliers excluded from the group range).
+//
+// One CTA per output row.  The row's outlier columns are expanded into a bitmask in
+// shared memory, each warp then quantizes whole groups (min / max by shuffles, the
+// scale and zero-point in FP64 so that every rounding is fixed bit for bit), codes go
+// to shared memory as bytes and are finally packed into 32-bit words.
+#include <new>
+
+#include "common.cuh"
+
+namespace {
+
+constexpr int kThreads = 256;
+
+__device__ __forceinline__ bool half_bits_finite(unsigned int h) { return (h & 0x7C00u) != 0x7C00u; }
+
+template <int GROUP>
+__global__ void __launch_bounds__(kThreads)
+pack_row_kernel(const uint16_t* __restrict__ W, const int32_t* __restrict__ row_ptr,
+                const int32_t* __restrict__ col_idx, int K, int bits, uint32_t* __restrict__ codes,
+                uint16_t* __restrict__ scales, uint8_t* __restrict__ zeros, int32_t* __restrict__ status) {
+  extern __shared__ unsigned char smem[];
+  unsigned int* mask = reinterpret_cast<unsigned int*>(smem);  // K/32 words
+  unsigned char* q8 = smem + (K / 32) * 4;                      // K bytes
+  const int row = blockIdx.x;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (int i = threadIdx.x; i < K / 32; i += kThreads) mask[i] = 0;
+  __syncthreads();
+  const int jb = row_ptr[row], je = row_ptr[row + 1];
+  for (int j = jb + threadIdx.x; j < je; j += kThreads) {
+    const int c = col_idx[j];
+    if (c >= 0 && c < K) atomicOr(&mask[c >> 5], 1u << (c & 31));
+  }
+  __syncthreads();
+
+  constexpr int EPL = GROUP / 32;  // consecutive elements per lane
+  const int ngroups = K / GROUP;
+  const double qmax = (double)((1 << bits) - 1);
+  const uint16_t* wrow = W + (long long)row * K;
+  bool bad = false;
+  for (int g = warp; g < ngroups; g += kThreads / 32) {
+    const int c0 = g * GROUP + lane * EPL;
+    unsigned int hb[EPL];
+    if (EPL == 4) {
+      const uint2 v = *reinterpret_cast<const uint2*>(wrow + c0);
+      hb[0] = v.x & 0xFFFFu; hb[1] = v.x >> 16; hb[EPL - 2] = v.y & 0xFFFFu; hb[EPL - 1] = v.y >> 16;
+    } else {
+      const unsigned int v = *reinterpret_cast<const unsigned int*>(wrow + c0);
+      hb[0] = v & 0xFFFFu; hb[1] = v >> 16;
+    }
+    // this lane's EPL mask bits: c0 is a multiple of EPL, so they sit in one mask word
+    const unsigned int mbits = (mask[c0 >> 5] >> (c0 & 31)) & ((1u << EPL) - 1u);
+    float w[EPL];
+    float lo = 0.f, hi = 0.f;
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) {
+      bad |= !half_bits_finite(hb[e]);
+      w[e] = __half2float(__ushort_as_half((unsigned short)hb[e]));
+      if (!((mbits >> e) & 1u)) {
+        lo = fminf(lo, w[e]);
+        hi = fmaxf(hi, w[e]);
+      }
+    }
+    for (int o = 16; o > 0; o >>= 1) {
+      lo = fminf(lo, __shfl_xor_sync(0xFFFFFFFFu, lo, o));
+      hi = fmaxf(hi, __shfl_xor_sync(0xFFFFFFFFu, hi, o));
+    }
+    __half sh = __ushort_as_half((unsigned short)0x3C00u);  // 1.0
+    double z = 0.0;
+    if (hi > lo) {
+      const double s64 = ((double)hi - (double)lo) / qmax;
+      // smallest fp16 >= s64: two directed roundings compose to one
+      sh = __float2half_ru(__double2float_ru(s64));
+      const double s = (double)__half2float(sh);
+      z = fmin(fmax(rint(-(double)lo / s), 0.0), qmax);
+    }
+    const double s = (double)__half2float(sh);
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) {
+      double q = z;
+      if (!((mbits >> e) & 1u)) q = fmin(fmax(rint((double)w[e] / s) + z, 0.0), qmax);
+      q8[c0 + e] = (unsigned char)(int)q;
+    }
+    if (lane == 0) {
+      scales[(long long)row * ngroups + g] = __half_as_ushort(sh);
+      zeros[(long long)row * ngroups + g] = (uint8_t)(int)z;
+    }
+  }
+  if (bad) atomicExch(status, (int32_t)GWQ_ERR_NONFINITE);
+  __syncthreads();
+
+  // pack: word wi of the row belongs to run wi / bits, word j = wi % bits of that run
+  const int nwords = K / 32 * bits;
+  uint32_t* crow = codes + (long long)row * nwords;
+  for (int wi = threadIdx.x; wi < nwords; wi += kThreads) {
+    const int run = wi / bits, j = wi - run * bits;
+    const unsigned char* c = q8 + run * 32;
+    const int first = (32 * j) / bits;
+    unsigned int word = 0;
+    for (int i = first; i < 32 && i * bits < 32 * j + 32; ++i) {
+      const int p = i * bits - 32 * j;
+      const unsigned int v = c[i];
+      word |= (p >= 0) ? (v << p) : (v >> (-p));
+    }
+    crow[wi] = word;
+  }
+}
+
+__global__ void narrow_cols_kernel(const int32_t* __restrict__ col, uint16_t* __restrict__ col16, long long n) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) col16[i] = (uint16_t)col[i];
+}
+
+}  // namespace
+
+extern "C" gwq_status gwq_pack(const uint16_t* W, gwq_outliers* S, int32_t N, int32_t K, int32_t bits,
+                               int32_t group, gwq_packed** out, void* stream_) {
+  if (out) *out = nullptr;
+  if (!W || !S || !out || N <= 0 || K <= 0) return GWQ_ERR_INVALID_ARG;
+  if (S->tag != GWQ_TAG_OUTLIERS || S->N != N || S->K != K) return GWQ_ERR_INVALID_ARG;
+  if (!gwq_aligned16(W)) return GWQ_ERR_INVALID_ARG;
+  if (bits != 3 && bits != 4) return GWQ_ERR_UNSUPPORTED;
+  if (group != 64 && group != 128) return GWQ_ERR_UNSUPPORTED;
+  if (K % group != 0 || K > 131072) return GWQ_ERR_UNSUPPORTED;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+
+  gwq_status st = GWQ_OK;
+  int32_t host_status = 0;
+  const size_t ngroups = (size_t)N * (K / group);
+  const size_t nwords = (size_t)N * (K / 32) * bits;
+  const size_t smem = (size_t)(K / 32) * 4 + (size_t)K;
+  gwq_packed* P = new (std::nothrow) gwq_packed();
+  gwq_priv* pv = new (std::nothrow) gwq_priv();
+  if (!P || !pv) {
+    delete P;
+    delete pv;
+    return GWQ_ERR_ALLOC;
+  }
+  *pv = gwq_priv{};
+  P->tag = GWQ_TAG_PACKED;
+  P->N = N; P->K = K; P->bits = bits; P->group = group;
+  P->codes = nullptr; P->scales = nullptr; P->zeros = nullptr; P->S = nullptr; P->priv = pv;
+  int dev = 0;
+  GWQ_CUDA_TRY(cudaGetDevice(&dev));
+  GWQ_CUDA_TRY(cudaDeviceGetAttribute(&pv->sm_count, cudaDevAttrMultiProcessorCount, dev));
+  GWQ_CUDA_TRY(cudaMalloc(&P->codes, nwords * sizeof(uint32_t)));
+  GWQ_CUDA_TRY(cudaMalloc(&P->scales, ngroups * sizeof(uint16_t) + 16));
+  GWQ_CUDA_TRY(cudaMalloc(&P->zeros, ngroups + 16));
+  GWQ_CUDA_TRY(cudaMalloc(&pv->dev_status, 64));
+  GWQ_CUDA_TRY(cudaMemsetAsync(pv->dev_status, 0, 64, stream));
+  if (group == 128) {
+    GWQ_CUDA_TRY(cudaFuncSetAttribute(pack_row_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    pack_row_kernel<128><<<N, kThreads, smem, stream>>>(W, S->row_ptr, S->col_idx, K, bits, P->codes,
+                                                        P->scales, P->zeros, pv->dev_status);
+  } else {
+    GWQ_CUDA_TRY(cudaFuncSetAttribute(pack_row_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    pack_row_kernel<64><<<N, kThreads, smem, stream>>>(W, S->row_ptr, S->col_idx, K, bits, P->codes,
+                                                       P->scales, P->zeros, pv->dev_status);
+  }
+  GWQ_CUDA_TRY(cudaGetLastError());
+  if (K <= 65536) {
+    const long long nnz = S->nnz;
+    GWQ_CUDA_TRY(cudaMalloc(&pv->col16, (size_t)(nnz > 0 ? nnz : 1) * sizeof(uint16_t) + 16));
+    if (nnz > 0) {
+      narrow_cols_kernel<<<(unsigned)((nnz + 255) / 256), 256, 0, stream>>>(S->col_idx, pv->col16, nnz);
+      GWQ_CUDA_TRY(cudaGetLastError());
+    }
+  }
+  GWQ_CUDA_TRY(cudaMemcpyAsync(&host_status, pv->dev_status, sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
+  GWQ_CUDA_TRY(cudaStreamSynchronize(stream));
+  if (host_status != 0) {
+    st = (gwq_status)host_status;
+    goto fail;
+  }
+  GWQ_CUDA_TRY(cudaMemsetAsync(pv->dev_status, 0, 64, stream));
+  P->S = S;
+  *out = P;
+  return GWQ_OK;
+fail:
+  if (P->codes) cudaFree(P->codes);
+  if (P->scales) cudaFree(P->scales);
+  if (P->zeros) cudaFree(P->zeros);
+  if (pv->col16) cudaFree(pv->col16);
+  if (pv->dev_status) cudaFree(pv->dev_status);
+  delete pv;
+  delete P;
+  return st;
+}
