@@ -1,0 +1,258 @@
+"""Thin ctypes binding of the C-ABI library (include/gwq.h).
+
+Argument marshalling only: every step of the method runs in the CUDA kernels of
+libgwq.so.  PyTorch tensors are used as plain device buffers (data_ptr) and for
+the current stream.  There is no CPU fallback: a missing library or a missing
+CUDA device raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libgwq.so")
+
+GWQ_OK = 0
+GWQ_F16, GWQ_BF16, GWQ_F32 = 0, 1, 2
+STATUS_NAMES = {
+    0: "GWQ_OK", 1: "GWQ_ERR_INVALID_ARG", 2: "GWQ_ERR_UNSUPPORTED", 3: "GWQ_ERR_ALLOC",
+    4: "GWQ_ERR_NONFINITE", 5: "GWQ_ERR_TIMEOUT", 6: "GWQ_ERR_CUDA",
+}
+EXPORTS = ("gwq_select_outliers", "gwq_pack", "gwq_linear", "gwq_linear_host", "gwq_free",
+           "gwq_status_string")
+
+
+class GwqError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {STATUS_NAMES.get(status, status)}")
+
+
+class gwq_outliers(C.Structure):
+    _fields_ = [("tag", C.c_uint32), ("N", C.c_int32), ("K", C.c_int32), ("nnz", C.c_int64),
+                ("row_ptr", C.c_void_p), ("col_idx", C.c_void_p), ("val", C.c_void_p)]
+
+
+class gwq_packed(C.Structure):
+    _fields_ = [("tag", C.c_uint32), ("N", C.c_int32), ("K", C.c_int32), ("bits", C.c_int32),
+                ("group", C.c_int32), ("codes", C.c_void_p), ("scales", C.c_void_p),
+                ("zeros", C.c_void_p), ("S", C.POINTER(gwq_outliers)), ("priv", C.c_void_p)]
+
+
+_lib = None
+
+
+def load_library(path: str = LIB_PATH) -> C.CDLL:
+    """Load libgwq.so and declare the prototypes of include/gwq.h."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(path):
+        raise RuntimeError(f"{path} is missing: build it with `python -m paper_2411_00850_b200.build` "
+                           "(there is no fallback path)")
+    lib = C.CDLL(path)
+    lib.gwq_select_outliers.restype = C.c_int
+    lib.gwq_select_outliers.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_double,
+                                        C.POINTER(C.POINTER(gwq_outliers)), C.c_void_p]
+    lib.gwq_pack.restype = C.c_int
+    lib.gwq_pack.argtypes = [C.c_void_p, C.POINTER(gwq_outliers), C.c_int32, C.c_int32, C.c_int32, C.c_int32,
+                             C.POINTER(C.POINTER(gwq_packed)), C.c_void_p]
+    lib.gwq_linear.restype = C.c_int
+    lib.gwq_linear.argtypes = [C.POINTER(gwq_packed), C.c_void_p, C.c_int, C.c_int32, C.c_void_p, C.c_int,
+                               C.c_void_p]
+    lib.gwq_linear_host.restype = C.c_int
+    lib.gwq_linear_host.argtypes = lib.gwq_linear.argtypes
+    lib.gwq_free.restype = None
+    lib.gwq_free.argtypes = [C.c_void_p]
+    lib.gwq_status_string.restype = C.c_char_p
+    lib.gwq_status_string.argtypes = [C.c_int]
+    _lib = lib
+    return lib
+
+
+def _stream_ptr() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _dtype_code(t: torch.dtype) -> int:
+    if t == torch.float16:
+        return GWQ_F16
+    if t == torch.bfloat16:
+        return GWQ_BF16
+    if t == torch.float32:
+        return GWQ_F32
+    raise TypeError(f"unsupported dtype {t}")
+
+
+def _check(st: int, where: str):
+    if st != GWQ_OK:
+        raise GwqError(st, where)
+
+
+def _view(ptr: int, n: int, dtype: torch.dtype, device) -> torch.Tensor:
+    """Copy n elements at device address ptr into a new tensor (D2D copy)."""
+    out = torch.empty(n, dtype=dtype, device=device)
+    if n:
+        nbytes = n * out.element_size()
+        rc = torch.cuda.cudart().cudaMemcpy(out.data_ptr(), ptr, nbytes, 3)  # 3 = device to device
+        if int(rc) != 0:
+            raise RuntimeError(f"cudaMemcpy failed: {rc}")
+    return out
+
+
+class Outliers:
+    """Owner of a gwq_outliers* (CSR of the FP16 outlier matrix S)."""
+
+    def __init__(self, handle, device):
+        self._h = handle
+        self.device = device
+
+    @property
+    def N(self): return self._h.contents.N
+    @property
+    def K(self): return self._h.contents.K
+    @property
+    def nnz(self): return self._h.contents.nnz
+
+    def arrays(self):
+        """(row_ptr int32 [N+1], col_idx int32 [nnz], val int16-bit patterns [nnz]) as tensors."""
+        c = self._h.contents
+        return (_view(c.row_ptr, c.N + 1, torch.int32, self.device),
+                _view(c.col_idx, c.nnz, torch.int32, self.device),
+                _view(c.val, c.nnz, torch.int16, self.device))
+
+    def free(self):
+        if self._h is not None:
+            load_library().gwq_free(C.cast(self._h, C.c_void_p))
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.free()
+        except Exception:
+            pass
+
+
+class Packed:
+    """Owner of a gwq_packed* (codes, scales, zero-points and the outliers)."""
+
+    def __init__(self, handle, device):
+        self._h = handle
+        self.device = device
+
+    @property
+    def N(self): return self._h.contents.N
+    @property
+    def K(self): return self._h.contents.K
+    @property
+    def bits(self): return self._h.contents.bits
+    @property
+    def group(self): return self._h.contents.group
+    @property
+    def nnz(self): return self._h.contents.S.contents.nnz
+
+    def arrays(self):
+        """dict of tensors copied out of the packed object (for inspection and parity)."""
+        c = self._h.contents
+        s = c.S.contents
+        nw = c.N * (c.K // 32) * c.bits
+        ng = c.N * (c.K // c.group)
+        return dict(
+            words=_view(c.codes, nw, torch.int32, self.device).view(c.N, -1),
+            scales=_view(c.scales, ng, torch.int16, self.device).view(c.N, -1),
+            zeros=_view(c.zeros, ng, torch.uint8, self.device).view(c.N, -1),
+            row_ptr=_view(s.row_ptr, s.N + 1, torch.int32, self.device),
+            col_idx=_view(s.col_idx, s.nnz, torch.int32, self.device),
+            val=_view(s.val, s.nnz, torch.int16, self.device),
+        )
+
+    def packed_bytes(self) -> int:
+        """Bytes of codes + scales + zero-points + CSR as stored by the ABI-visible format."""
+        c = self._h.contents
+        nnz = c.S.contents.nnz
+        return (c.N * (c.K // 32) * c.bits * 4 + c.N * (c.K // c.group) * 3 + (c.N + 1) * 4 + nnz * 6)
+
+    def free(self):
+        if self._h is not None:
+            load_library().gwq_free(C.cast(self._h, C.c_void_p))
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.free()
+        except Exception:
+            pass
+
+
+def _require_cuda(t: torch.Tensor, name: str):
+    if not t.is_cuda:
+        raise ValueError(f"{name} must be a CUDA tensor (no CPU path exists)")
+    if not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous")
+
+
+def gwq_select_outliers(W: torch.Tensor, G: torch.Tensor, frac: float) -> Outliers:
+    """W fp16 [N,K], G fp32 [N,K] on the GPU -> CSR of the ceil(frac*N*K) largest-|G| weights."""
+    lib = load_library()
+    _require_cuda(W, "W"); _require_cuda(G, "G")
+    if W.dtype != torch.float16 or G.dtype != torch.float32 or W.shape != G.shape or W.dim() != 2:
+        raise ValueError("W must be fp16 [N,K] and G fp32 [N,K]")
+    N, K = W.shape
+    out = C.POINTER(gwq_outliers)()
+    with torch.cuda.device(W.device):
+        st = lib.gwq_select_outliers(W.data_ptr(), G.data_ptr(), N, K, float(frac), C.byref(out), _stream_ptr())
+    _check(st, "gwq_select_outliers")
+    return Outliers(out, W.device)
+
+
+def gwq_pack(W: torch.Tensor, S: Outliers, bits: int, group: int) -> Packed:
+    """Quantize the non-outliers of W and pack; S is consumed (owned by the result)."""
+    lib = load_library()
+    _require_cuda(W, "W")
+    if W.dtype != torch.float16 or W.dim() != 2:
+        raise ValueError("W must be fp16 [N,K]")
+    N, K = W.shape
+    out = C.POINTER(gwq_packed)()
+    with torch.cuda.device(W.device):
+        st = lib.gwq_pack(W.data_ptr(), S._h, N, K, int(bits), int(group), C.byref(out), _stream_ptr())
+    _check(st, "gwq_pack")
+    S._h = None  # ownership moved
+    return Packed(out, W.device)
+
+
+def gwq_linear(P: Packed, x: torch.Tensor, out_dtype: torch.dtype | None = None,
+               out: torch.Tensor | None = None) -> torch.Tensor:
+    """y = x (deq(Wq) + S)^T for x [M,K] fp16/bf16 on the GPU; asynchronous on the current stream."""
+    lib = load_library()
+    _require_cuda(x, "x")
+    if x.dim() != 2 or x.shape[1] != P.K:
+        raise ValueError("x must be [M, K]")
+    M = x.shape[0]
+    if out is None:
+        out = torch.empty((M, P.N), dtype=out_dtype or x.dtype, device=x.device)
+    else:
+        _require_cuda(out, "out")
+    st = lib.gwq_linear(P._h, x.data_ptr(), _dtype_code(x.dtype), M, out.data_ptr(), _dtype_code(out.dtype),
+                        _stream_ptr())
+    _check(st, "gwq_linear")
+    return out
+
+
+def gwq_linear_host(P: Packed, x_host: torch.Tensor, y_host: torch.Tensor) -> torch.Tensor:
+    """Same product with HOST tensors (ideally pinned); copies in, computes, copies out, synchronises."""
+    lib = load_library()
+    if x_host.is_cuda or y_host.is_cuda:
+        raise ValueError("gwq_linear_host takes host tensors")
+    M = x_host.shape[0]
+    with torch.cuda.device(P.device):
+        st = lib.gwq_linear_host(P._h, x_host.data_ptr(), _dtype_code(x_host.dtype), M, y_host.data_ptr(),
+                                 _dtype_code(y_host.dtype), _stream_ptr())
+    _check(st, "gwq_linear_host")
+    return y_host
+
+
+def gwq_free(obj) -> None:
+    obj.free()

@@ -1,0 +1,93 @@
+"""GPU parity of y = x (deq(Wq) + S)^T against the CPU checker:
+|y_gpu - y_ref| <= 1e-3 * sum_k |x_k w_hat_k| + 1e-5 per output."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import gwq_oracle as orc
+from paper_2411_00850_b200 import binding as gwq
+from paper_2411_00850_b200 import synth
+from tests.gpu_util import (assert_linear_close, assert_packed_equal, oracle_w_hat, quantize_on_gpu, x_tensor)
+
+pytestmark = pytest.mark.gpu
+
+_cache = {}
+
+
+def _layer(N, K, frac, bits, group, seed):
+    key = (N, K, frac, bits, group, seed)
+    if key not in _cache:
+        W, G = synth.make_weight_and_grad(N, K, seed)
+        L = orc.quantize_layer(W, G, frac, bits, group)
+        P = quantize_on_gpu(W, G, frac, bits, group)
+        assert_packed_equal(P, L)
+        _cache[key] = (P, L, oracle_w_hat(L))
+    return _cache[key]
+
+
+DECODE_LAYERS = [
+    (1024, 1024, 0.01, 4, 128, 20),
+    (1024, 1024, 0.01, 3, 128, 21),
+    (1000, 2112, 0.02, 4, 64, 22),
+    (1000, 2112, 0.005, 3, 64, 23),
+    (528, 4096, 0.01, 4, 128, 24),
+]
+
+
+@pytest.mark.parametrize("layer", DECODE_LAYERS)
+@pytest.mark.parametrize("M", [1, 2, 4, 7, 8, 16, 17, 32])
+@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+def test_decode_sizes(layer, M, dtype):
+    P, L, w_hat = _layer(*layer)
+    bits16, xv = synth.make_activations(M, P.K, seed=M, dtype=dtype)
+    y_ref, bound = orc.linear(xv, w_hat)
+    y = gwq.gwq_linear(P, x_tensor(bits16, dtype), out_dtype=torch.float32)
+    assert_linear_close(y, y_ref, bound)
+    y16 = gwq.gwq_linear(P, x_tensor(bits16, dtype))
+    assert_linear_close(y16, y_ref, bound, extra_rel=2.0 ** -9 if dtype == "bf16" else 0.0)
+
+
+@pytest.mark.parametrize("layer", DECODE_LAYERS[:4])
+def test_unit_activations_read_back_weight_columns(layer):
+    P, L, w_hat = _layer(*layer)
+    cols = [0, 1, 31, 32, 63, 64, 127, 128, P.K - 1]
+    cols += [int(c) for c in L["col_idx"][:7]]          # some outlier columns
+    bits16, xv = synth.unit_activations(cols, P.K, "f16")
+    y_ref, bound = orc.linear(xv, w_hat)
+    y = gwq.gwq_linear(P, x_tensor(bits16, "f16"), out_dtype=torch.float32)
+    assert_linear_close(y, y_ref, bound)
+
+
+@pytest.mark.parametrize("M", [33, 63, 64, 100, 128, 300])
+@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+def test_larger_batches(M, dtype):
+    P, L, w_hat = _layer(*DECODE_LAYERS[0])
+    bits16, xv = synth.make_activations(M, P.K, seed=M, dtype=dtype, heavy_channels=8)
+    y_ref, bound = orc.linear(xv, w_hat)
+    y = gwq.gwq_linear(P, x_tensor(bits16, dtype), out_dtype=torch.float32)
+    assert_linear_close(y, y_ref, bound)
+
+
+def test_all_outliers_is_the_dense_product():
+    N, K = 128, 512
+    W, G = synth.make_weight_and_grad(N, K, 30)
+    P = quantize_on_gpu(W, G, 1.0, 4, 128)
+    bits16, xv = synth.make_activations(3, K, seed=30)
+    y = gwq.gwq_linear(P, x_tensor(bits16, "f16"), out_dtype=torch.float32)
+    y_ref = xv @ W.astype(np.float64).T
+    bound = np.abs(xv) @ np.abs(W.astype(np.float64)).T
+    assert_linear_close(y, y_ref, bound)
+    P.free()
+
+
+def test_host_buffer_entry_point_and_argument_errors():
+    P, L, w_hat = _layer(*DECODE_LAYERS[0])
+    bits16, xv = synth.make_activations(4, P.K, seed=5)
+    y_ref, bound = orc.linear(xv, w_hat)
+    xh = torch.from_numpy(bits16.view(np.int16).copy()).view(torch.float16).pin_memory()
+    yh = torch.empty((4, P.N), dtype=torch.float32).pin_memory()
+    gwq.gwq_linear_host(P, xh, yh)
+    assert_linear_close(yh, y_ref, bound)
+    with pytest.raises(gwq.GwqError) as e:
+        gwq.gwq_linear(P, torch.zeros((2, P.K), dtype=torch.float32, device="cuda:0"))
+    assert e.value.status == 2
