@@ -92,12 +92,33 @@ def _check(st: int, where: str):
         raise GwqError(st, where)
 
 
+_rt = None
+
+
+def _cudart() -> C.CDLL:
+    """The CUDA runtime that torch has already loaded (used only to copy results out)."""
+    global _rt
+    if _rt is None:
+        last = None
+        for name in ("libcudart.so.12", "libcudart.so.13", "libcudart.so"):
+            try:
+                _rt = C.CDLL(name)
+                break
+            except OSError as e:
+                last = e
+        if _rt is None:
+            raise RuntimeError(f"CUDA runtime library not found: {last}")
+        _rt.cudaMemcpy.restype = C.c_int
+    return _rt
+
+
 def _view(ptr: int, n: int, dtype: torch.dtype, device) -> torch.Tensor:
     """Copy n elements at device address ptr into a new tensor (D2D copy)."""
     out = torch.empty(n, dtype=dtype, device=device)
     if n:
         nbytes = n * out.element_size()
-        rc = torch.cuda.cudart().cudaMemcpy(out.data_ptr(), ptr, nbytes, 3)  # 3 = device to device
+        torch.cuda.current_stream().synchronize()
+        rc = _cudart().cudaMemcpy(C.c_void_p(out.data_ptr()), C.c_void_p(ptr), C.c_size_t(nbytes), 3)  # 3 = D2D
         if int(rc) != 0:
             raise RuntimeError(f"cudaMemcpy failed: {rc}")
     return out

@@ -28,8 +28,8 @@ def _layer(N, K, frac, bits, group, seed):
 DECODE_LAYERS = [
     (1024, 1024, 0.01, 4, 128, 20),
     (1024, 1024, 0.01, 3, 128, 21),
-    (1000, 2112, 0.02, 4, 64, 22),
-    (1000, 2112, 0.005, 3, 64, 23),
+    (1000, 2176, 0.02, 4, 64, 22),
+    (1000, 2176, 0.005, 3, 64, 23),
     (528, 4096, 0.01, 4, 128, 24),
 ]
 
