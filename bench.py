@@ -1,0 +1,479 @@
+#!/usr/bin/env python
+"""Benchmark of the GWQ mixed-precision linear layer on B200.
+
+One "step" is one pass of gwq_linear over the Llama-7B-shaped decode layer set
+(7 projections, each packed to 4 and to 3 bits, group 128, 1 % outliers) at
+M = 1, 4 and 16 tokens: 42 launches, replayed as one CUDA graph.  The headline
+value is the HBM rate over the algorithmic bytes of that step.  Beside it the
+line reports per-layer decode times, the tensor-core prefill cases, the encode
+kernels, a dense fp16 GEMM (torch.matmul, a library call) on the unquantized
+weights, the end-to-end rate through the host-buffer entry point, and the CPU
+checker timed on the host cores.
+
+  python bench.py --gpus 1 --steps 20 --warmup 3
+  python bench.py --impl reference ...      (times the CPU checker instead)
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+from paper_2411_00850_b200 import synth
+
+METRIC = "GWQ W4/W3 linear: decode µs & HBM GB/s (% roofline); prefill TFLOP/s"
+WORKLOAD = "llama7b_decode_layer_set_w4_w3_g128_1pct_M1_4_16"
+DECODE_MS = (1, 4, 16)
+BIT_WIDTHS = (4, 3)
+GROUP = 128
+FRAC = 0.01
+CONFIG_INDEX = 1
+PREFILL_SHAPES = ((11008, 4096), (4096, 11008))
+PREFILL_MS = (512, 2048, 8192)
+
+
+def measured_peaks():
+    """(hbm GB/s, bf16 TFLOP/s burst, sustained, source) from the pool's measured file, else the fallback."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        d = json.load(open(path))
+        return float(d["hbm_gbs"]), float(d["bf16_tflops"]), float(d["bf16_tflops_sustained"]), "measured"
+    except Exception:
+        return 6650.0, 1590.0, 1400.0, "fallback"
+
+
+def algorithmic_bytes(N: int, K: int, bits: int, group: int, nnz: int, M: int, col_bytes: int = 2) -> int:
+    """Bytes one decode launch has to move: codes, scales, zero-points, the CSR (row
+    pointers, columns as the kernel reads them, fp16 values), x and y."""
+    codes = N * K * bits // 8
+    meta = N * (K // group) * 3
+    csr = (N + 1) * 4 + nnz * (col_bytes + 2)
+    return codes + meta + csr + M * K * 2 + M * N * 2
+
+
+def linear_flops(N: int, K: int, nnz: int, M: int) -> int:
+    return 2 * M * (N * K + nnz)
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while a region runs."""
+
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.QUERY}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons, power = [], [], set(), []
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for ln in self.lines:
+            f = [t.strip() for t in ln.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); smax.append(float(f[1])); power.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(smax)), "power_w_max": float(max(power)),
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ----------------------------------------------------------------------------- the CUDA arm
+def build_layer_set(torch, gwq, dev, replicas: int, keep_dense: bool):
+    """Generate the 7 seeded layers, encode each to 4 and 3 bits on the GPU.
+    Returns (layers, encode_stats); layers[i] = dict(name, N, K, packed={bits: [Packed]*replicas}, W=dense)."""
+    layers, enc = [], {"select_ms": 0.0, "pack_ms": 0.0, "select_bytes": 0, "pack_bytes": 0}
+    for li, (name, N, K) in enumerate(synth.LLAMA7B_LAYER_SET):
+        W, G = synth.make_weight_and_grad(N, K, synth.layer_seed(CONFIG_INDEX, li))
+        Wd, Gd = torch.from_numpy(W).to(dev), torch.from_numpy(G).to(dev)
+        entry = dict(name=name, N=N, K=K, packed={}, W=Wd if keep_dense else None)
+        for bits in BIT_WIDTHS:
+            reps = []
+            for r in range(replicas):
+                e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+                e0.record()
+                S = gwq.gwq_select_outliers(Wd, Gd, FRAC)
+                e1.record()
+                P = gwq.gwq_pack(Wd, S, bits, GROUP)
+                e2.record()
+                torch.cuda.synchronize()
+                if r == 0:
+                    enc["select_ms"] += e0.elapsed_time(e1)
+                    enc["pack_ms"] += e1.elapsed_time(e2)
+                    enc["select_bytes"] += N * K * 4
+                    enc["pack_bytes"] += N * K * 2 + N * K * bits // 8
+                reps.append(P)
+            entry["packed"][bits] = reps
+        layers.append(entry)
+        del Gd
+    return layers, enc
+
+
+def decode_cases(layers):
+    """(layer index, bits, M) for every launch of one step, in launch order."""
+    return [(li, bits, M) for M in DECODE_MS for bits in BIT_WIDTHS for li in range(len(layers))]
+
+
+def time_region(torch, fn, iters: int) -> float:
+    """Milliseconds per call of fn(i), CUDA events on the current stream, synchronised on both sides."""
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(iters):
+        fn(i)
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / iters
+
+
+def capture(torch, fn):
+    """Capture fn() into a CUDA graph (after one eager run) and return a replay callable."""
+    fn()
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        fn()
+    return g.replay
+
+
+def run_cuda_arm(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2411_00850_b200 import binding as gwq
+    from paper_2411_00850_b200 import build as gbuild
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    if rank == 0:
+        gbuild.build()
+    if world > 1:
+        dist.barrier()
+    gwq.load_library()
+    hbm_peak, tf_burst, tf_sust, peak_src = measured_peaks()
+
+    replicas = 2   # two copies of every packed layer: ~420 MB touched between reuses (L2 is 126 MB)
+    layers, enc = build_layer_set(torch, gwq, dev, replicas, keep_dense=True)
+    cases = decode_cases(layers)
+    xs = {}
+    for li, L in enumerate(layers):
+        for M in DECODE_MS:
+            bits16, _ = synth.make_activations(M, L["K"], seed=synth.layer_seed(CONFIG_INDEX, li), dtype="f16")
+            xs[(li, M)] = torch.from_numpy(bits16.view(np.int16).copy()).to(dev).view(torch.float16)
+    ys = {(li, bits, M): torch.empty((M, layers[li]["N"]), dtype=torch.float16, device=dev)
+          for (li, bits, M) in cases}
+
+    def step_fn(rep):
+        def run():
+            for (li, bits, M) in cases:
+                gwq.gwq_linear(layers[li]["packed"][bits][rep], xs[(li, M)], out=ys[(li, bits, M)])
+        return run
+
+    graphs = [capture(torch, step_fn(r)) for r in range(replicas)]
+    step_bytes = sum(algorithmic_bytes(layers[li]["N"], layers[li]["K"], bits, GROUP,
+                                       layers[li]["packed"][bits][0].nnz, M) for (li, bits, M) in cases)
+
+    # ---- headline: W warm-up steps, then exactly K timed steps, barrier + synchronize on both sides
+    for i in range(args.warmup):
+        graphs[i % replicas]()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    ms_step = time_region(torch, lambda i: graphs[i % replicas](), args.steps)
+    if world > 1:
+        t = torch.tensor([ms_step], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_step = float(t.item())
+        dist.barrier()
+    clocks = sampler.stop() if rank == 0 else {}
+    value = world * step_bytes / (ms_step * 1e-3) / 1e9
+
+    out = {
+        "metric": METRIC, "value": round(value, 1), "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": round(ms_step, 4), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f16 x int4/int3 -> f32 accumulate", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "layers": [f"{n}:{N}x{K}" for n, N, K in synth.LLAMA7B_LAYER_SET],
+                   "bits": list(BIT_WIDTHS), "group": GROUP, "outlier_frac": FRAC, "M": list(DECODE_MS),
+                   "launches_per_step": len(cases), "step_bytes": step_bytes,
+                   "l2": f"{replicas} rotating copies of the packed set ({replicas * step_bytes // 3 / 1e6:.0f} MB) "
+                         "exceed the 126 MB L2 between reuses; one CUDA graph per copy"},
+        "gpu_launches": len(cases) * args.steps,
+        "clocks": clocks,
+    }
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return None
+
+    # ---- everything below: rank 0 only, N = 1 detail
+    detail_iters = max(5, min(args.steps, 20))
+    out["roofline"] = {
+        "bound": "hbm", "kernel": "gwq decode linear (all 42 launches of the step)",
+        "achieved": round(step_bytes / (ms_step * 1e-3) / 1e9, 1), "peak": hbm_peak, "unit": "GB/s",
+        "frac": round(step_bytes / (ms_step * 1e-3) / 1e9 / hbm_peak, 4), "peak_source": peak_src,
+        "frac_of_nominal_8TBs": round(step_bytes / (ms_step * 1e-3) / 1e9 / 8000.0, 4),
+        "avg_launch_us": round(ms_step * 1e3 / len(cases), 3), "traffic": None,
+    }
+    if world == 1 and not args.headline_only:
+        out["decode_cases"] = bench_decode_detail(torch, gwq, layers, xs, ys, detail_iters, hbm_peak)
+        out["cublas_fp16"] = bench_dense_library(torch, layers, xs, detail_iters, step_bytes, ms_step)
+        out["e2e"] = bench_e2e(torch, gwq, layers, cases, detail_iters, step_bytes)
+        out["encode"] = {"select_ms": round(enc["select_ms"], 3), "pack_ms": round(enc["pack_ms"], 3),
+                         "select_gbs_per_pass_of_G": round(enc["select_bytes"] / (enc["select_ms"] * 1e-3) / 1e9, 1),
+                         "pack_gbs": round(enc["pack_bytes"] / (enc["pack_ms"] * 1e-3) / 1e9, 1),
+                         "note": "14 encodes of the layer set (7 layers x 2 bit widths), first replica"}
+        for L in layers:
+            L["W"] = None
+        out["prefill"] = bench_prefill(torch, gwq, dev, args, tf_burst, tf_sust)
+        out["cpu_baseline"] = cpu_baseline(sample_seconds=args.cpu_seconds)
+    else:
+        out["e2e"] = bench_e2e(torch, gwq, layers, cases, detail_iters, step_bytes, world)
+    if world > 1:
+        dist.destroy_process_group()
+    return out
+
+
+def bench_decode_detail(torch, gwq, layers, xs, ys, iters, hbm_peak):
+    """Per (shape, bits, M): microseconds per launch with a cold L2 (the launches of one graph
+    cycle through the layers of equal shape in both copies and a 256 MB scrub precedes every timing)."""
+    rows = []
+    scrub = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=xs[(0, 1)].device)
+    shapes = {}
+    for li, L in enumerate(layers):
+        shapes.setdefault((L["N"], L["K"]), []).append(li)
+    for (N, K), lis in shapes.items():
+        for bits in BIT_WIDTHS:
+            for M in DECODE_MS:
+                members = [(li, r) for r in range(len(layers[lis[0]]["packed"][bits])) for li in lis]
+
+                def run():
+                    for (li, r) in members:
+                        gwq.gwq_linear(layers[li]["packed"][bits][r], xs[(li, M)], out=ys[(li, bits, M)])
+                replay = capture(torch, run)
+                best = None
+                for _ in range(iters):
+                    scrub.fill_(1)
+                    ms = time_region(torch, lambda i: replay(), 1)
+                    best = ms if best is None else min(best, ms)
+                us = best * 1e3 / len(members)
+                nnz = layers[lis[0]]["packed"][bits][0].nnz
+                b = algorithmic_bytes(N, K, bits, GROUP, nnz, M)
+                rows.append({"N": N, "K": K, "bits": bits, "M": M, "us": round(us, 3), "bytes": b,
+                             "gbs": round(b / us / 1e3, 1), "frac_measured_peak": round(b / us / 1e3 / hbm_peak, 4),
+                             "frac_8TBs": round(b / us / 1e3 / 8000.0, 4), "launches_in_graph": len(members)})
+    del scrub
+    return rows
+
+
+def bench_dense_library(torch, layers, xs, iters, step_bytes, ms_step):
+    """torch.matmul (cuBLAS) fp16 on the unquantized weights: same layers, same M, one graph, two
+    passes per replay so that each weight matrix (404 MB in total) is cold when it is read again."""
+    ws = [L["W"] for L in layers]
+
+    def run():
+        for M in DECODE_MS:
+            for _ in BIT_WIDTHS:          # the GWQ step visits every layer twice per M (W4 and W3)
+                for li, W in enumerate(ws):
+                    torch.matmul(xs[(li, M)], W.t())
+    replay = capture(torch, run)
+    for _ in range(3):
+        replay()
+    ms = time_region(torch, lambda i: replay(), iters)
+    dense_bytes = sum(W.numel() * 2 for W in ws) * len(DECODE_MS) * len(BIT_WIDTHS)
+    return {"ms_per_step": round(ms, 4), "dense_bytes_per_step": dense_bytes,
+            "gbs_on_dense_bytes": round(dense_bytes / (ms * 1e-3) / 1e9, 1),
+            "gwq_speedup_over_library": round(ms / ms_step, 3),
+            "note": "library call (torch.matmul fp16), same 42 (layer, M) products, CUDA graph"}
+
+
+def bench_e2e(torch, gwq, layers, cases, iters, step_bytes, world=1):
+    """The same step through gwq_linear_host: pinned host x in, pinned host y out, copies and the
+    synchronisation inside the timed region."""
+    xh, yh = {}, {}
+    for li, L in enumerate(layers):
+        for M in DECODE_MS:
+            bits16, _ = synth.make_activations(M, L["K"], seed=synth.layer_seed(CONFIG_INDEX, li), dtype="f16")
+            xh[(li, M)] = torch.from_numpy(bits16.view(np.int16).copy()).view(torch.float16).pin_memory()
+    for (li, bits, M) in cases:
+        yh[(li, bits, M)] = torch.empty((M, layers[li]["N"]), dtype=torch.float16).pin_memory()
+    h2d = sum(xh[(li, M)].numel() * 2 for (li, bits, M) in cases)
+    d2h = sum(yh[c].numel() * 2 for c in cases)
+
+    def step(i):
+        r = i % 2
+        for (li, bits, M) in cases:
+            gwq.gwq_linear_host(layers[li]["packed"][bits][r], xh[(li, M)], yh[(li, bits, M)])
+    for i in range(2):
+        step(i)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for i in range(iters):
+        step(i)
+    torch.cuda.synchronize()
+    sec = (time.perf_counter() - t0) / iters
+    return {"value": round(world * step_bytes / sec / 1e9, 1), "unit": "GB/s", "ms_per_step": round(sec * 1e3, 4),
+            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+            "note": "42 synchronous host-buffer calls per step; bound by per-call copy and sync latency"}
+
+
+def bench_prefill(torch, gwq, dev, args, tf_burst, tf_sust):
+    """4-bit, group 128, 1 % outliers, bf16 activations with 8 heavy channels; TFLOP/s on 2 M (N K + nnz)."""
+    rows = []
+    for si, (N, K) in enumerate(PREFILL_SHAPES):
+        W, G = synth.make_weight_and_grad(N, K, synth.layer_seed(2, si))
+        Wd, Gd = torch.from_numpy(W).to(dev), torch.from_numpy(G).to(dev)
+        P = gwq.gwq_pack(Wd, gwq.gwq_select_outliers(Wd, Gd, FRAC), 4, GROUP)
+        del Gd
+        Wb = Wd.to(torch.bfloat16)
+        for M in PREFILL_MS:
+            bits16, _ = synth.make_activations(M, K, seed=synth.layer_seed(2, si), dtype="bf16", heavy_channels=8)
+            x = torch.from_numpy(bits16.view(np.int16).copy()).to(dev).view(torch.bfloat16)
+            y = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
+            for _ in range(2):
+                gwq.gwq_linear(P, x, out=y)
+            ms = time_region(torch, lambda i: gwq.gwq_linear(P, x, out=y), args.prefill_iters)
+            for _ in range(2):
+                torch.matmul(x, Wb.t())
+            ms_lib = time_region(torch, lambda i: torch.matmul(x, Wb.t()), args.prefill_iters)
+            fl = linear_flops(N, K, P.nnz, M)
+            tf = fl / (ms * 1e-3) / 1e12
+            rows.append({"N": N, "K": K, "M": M, "us": round(ms * 1e3, 2), "tflops": round(tf, 2),
+                         "frac_measured_burst": round(tf / tf_burst, 4), "frac_measured_sustained": round(tf / tf_sust, 4),
+                         "frac_nominal_2250": round(tf / 2250.0, 4), "library_bf16_us": round(ms_lib * 1e3, 2),
+                         "library_bf16_tflops": round(2 * M * N * K / (ms_lib * 1e-3) / 1e12, 2)})
+            del x, y
+        P.free()
+        del Wd, Wb
+    return rows
+
+
+# ----------------------------------------------------------------------------- the CPU checker, timed
+def cpu_baseline(sample_seconds: float = 20.0) -> dict:
+    """Times the CPU checker's forward product (reconstruction + float64 product) as it stands, on a
+    bounded sample of the same workload: the first 4096x4096 layer of the set, 4 and 3 bits,
+    M = 1, 4, 16, repeated until about `sample_seconds` have passed."""
+    from oracle import gwq_oracle as orc
+    try:
+        from threadpoolctl import threadpool_info
+        blas_threads = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        blas_threads = 1
+    name, N, K = synth.LLAMA7B_LAYER_SET[0]
+    W, G = synth.make_weight_and_grad(N, K, synth.layer_seed(CONFIG_INDEX, 0))
+    t_enc = time.perf_counter()
+    enc = {bits: orc.quantize_layer(W, G, FRAC, bits, GROUP) for bits in BIT_WIDTHS}
+    t_enc = time.perf_counter() - t_enc
+    xs = {M: synth.make_activations(M, K, seed=synth.layer_seed(CONFIG_INDEX, 0), dtype="f16")[1] for M in DECODE_MS}
+    done_bytes, passes = 0, 0
+    t0 = time.perf_counter()
+    while True:
+        for bits in BIT_WIDTHS:
+            L = enc[bits]
+            for M in DECODE_MS:
+                w_hat = orc.dequantize(L["codes"], L["scales"], L["zeros"], GROUP, L["row_ptr"], L["col_idx"], L["val"])
+                orc.linear(xs[M], w_hat)
+                done_bytes += algorithmic_bytes(N, K, bits, GROUP, int(L["row_ptr"][-1]), M)
+        passes += 1
+        if time.perf_counter() - t0 >= sample_seconds or passes >= 50:
+            break
+    sec = time.perf_counter() - t0
+    return {"value": round(done_bytes / sec / 1e9, 4), "unit": "GB/s", "cores": int(blas_threads),
+            "host_cores_available": len(os.sched_getaffinity(0)), "kind": "oracle",
+            "sample": f"{passes} passes over q_proj 4096x4096 (W4 and W3, g128, 1% outliers) x M in (1,4,16): "
+                      f"reconstruction + float64 product per call, {sec:.1f} s; encode on the CPU took {t_enc:.1f} s (untimed)",
+            "seconds": round(sec, 2)}
+
+
+def run_reference_arm(args):
+    """--impl reference: the CPU checker on the host cores, same metric and unit."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return None
+    per_step = max(2.0, min(20.0, 120.0 / max(1, args.steps + args.warmup)))
+    vals = []
+    for i in range(args.warmup + args.steps):
+        r = cpu_baseline(sample_seconds=per_step)
+        if i >= args.warmup:
+            vals.append(r)
+    value = float(np.mean([v["value"] for v in vals]))
+    ms = float(np.mean([v["seconds"] for v in vals])) * 1e3
+    return {"impl": "reference", "metric": METRIC, "value": round(value, 4), "unit": "GB/s",
+            "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": round(ms, 2), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64", "data": "synthetic", "config": {"workload": WORKLOAD, "sampled": vals[-1]["sample"]},
+            "cpu_baseline": {"value": round(value, 4), "unit": "GB/s", "cores": vals[-1]["cores"], "kind": "oracle",
+                             "sample": vals[-1]["sample"]},
+            "e2e": {"value": round(value, 4), "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=("ours", "reference"))
+    ap.add_argument("--prefill-iters", type=int, default=5)
+    ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    ap.add_argument("--headline-only", action="store_true", help="skip the per-case detail sections")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    out = run_reference_arm(args) if args.impl == "reference" else run_cuda_arm(args)
+    if out is not None:
+        print(json.dumps(out, ensure_ascii=False))
+
+
+if __name__ == "__main__":
+    main()
