@@ -87,6 +87,29 @@ typedef struct gwq_packed {
 gwq_status gwq_select_outliers(const uint16_t* W_f16, const float* G_f32, int32_t N, int32_t K,
                                double frac, gwq_outliers** out, void* stream);
 
+/* Outlier selection for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this is a deployment variant of gwq_select_outliers with identical
+ * results.)
+ *
+ * Who needs it: processes that have handed the whole device to their own memory pool or
+ * run under a fixed memory budget, so that a cudaMalloc inside a library call would
+ * fail, fragment the pool, or stall every stream of the process while the driver
+ * synchronises; and callers on a latency-critical path that may not take that stall.
+ * This call performs no cudaMalloc / cudaFree and calls no allocating routine.
+ *
+ *   row_ptr [N+1], col_idx [capacity], val [capacity]: device buffers supplied by the
+ *   caller; capacity must be >= ceil(frac * N*K), which is written to *nnz_host (host).
+ *   The work area is a fixed ~386 KiB array inside the library image, present on every
+ *   GPU that loads the library; it bounds the row count: N <= 32768, otherwise
+ *   GWQ_ERR_UNSUPPORTED.  All calls on one GPU share that array, so two calls that
+ *   overlap on the GPU (different streams or threads) corrupt each other; serialise
+ *   them.  The first call on each device looks up the array's device address; make that
+ *   first call outside any stream capture.  Synchronises `stream` before returning.
+ * Errors: as gwq_select_outliers, plus INVALID_ARG when capacity is too small.           */
+gwq_status gwq_select_outliers_static(const uint16_t* W_f16, const float* G_f32, int32_t N, int32_t K,
+                                      double frac, int32_t* row_ptr, int32_t* col_idx, uint16_t* val,
+                                      int64_t capacity, int64_t* nnz_host, void* stream);
+
 /* Group-wise asymmetric quantization of the non-outliers (Section 3.2, Eqs. "s", "z",
  * "q") and bit-packing.  Per (row, group of `group` consecutive k), over non-outlier
  * entries only: lo = min(0, min w), hi = max(0, max w); s = (hi - lo) / (2^bits - 1)

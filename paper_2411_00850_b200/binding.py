@@ -21,7 +21,7 @@ STATUS_NAMES = {
     0: "GWQ_OK", 1: "GWQ_ERR_INVALID_ARG", 2: "GWQ_ERR_UNSUPPORTED", 3: "GWQ_ERR_ALLOC",
     4: "GWQ_ERR_NONFINITE", 5: "GWQ_ERR_TIMEOUT", 6: "GWQ_ERR_CUDA",
 }
-EXPORTS = ("gwq_select_outliers", "gwq_pack", "gwq_linear", "gwq_linear_host", "gwq_free",
+EXPORTS = ("gwq_select_outliers", "gwq_select_outliers_static", "gwq_pack", "gwq_linear", "gwq_linear_host", "gwq_free",
            "gwq_status_string")
 
 
@@ -57,6 +57,10 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     lib.gwq_select_outliers.restype = C.c_int
     lib.gwq_select_outliers.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_double,
                                         C.POINTER(C.POINTER(gwq_outliers)), C.c_void_p]
+    lib.gwq_select_outliers_static.restype = C.c_int
+    lib.gwq_select_outliers_static.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_double,
+                                               C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64,
+                                               C.POINTER(C.c_int64), C.c_void_p]
     lib.gwq_pack.restype = C.c_int
     lib.gwq_pack.argtypes = [C.c_void_p, C.POINTER(gwq_outliers), C.c_int32, C.c_int32, C.c_int32, C.c_int32,
                              C.POINTER(C.POINTER(gwq_packed)), C.c_void_p]
@@ -227,6 +231,29 @@ def gwq_select_outliers(W: torch.Tensor, G: torch.Tensor, frac: float) -> Outlie
         st = lib.gwq_select_outliers(W.data_ptr(), G.data_ptr(), N, K, float(frac), C.byref(out), _stream_ptr())
     _check(st, "gwq_select_outliers")
     return Outliers(out, W.device)
+
+
+def gwq_select_outliers_static(W: torch.Tensor, G: torch.Tensor, frac: float, row_ptr: torch.Tensor,
+                               col_idx: torch.Tensor, val: torch.Tensor) -> int:
+    """Selection into caller-owned device tensors (row_ptr int32 [N+1], col_idx int32 [cap],
+    val int16 [cap]) without any device allocation inside the library; returns nnz.
+    For processes whose device memory is fully owned by their own pool, or that may not
+    take the stall of a cudaMalloc.  Calls must not overlap on one GPU; N <= 32768."""
+    lib = load_library()
+    for t, name in ((W, "W"), (G, "G"), (row_ptr, "row_ptr"), (col_idx, "col_idx"), (val, "val")):
+        _require_cuda(t, name)
+    N, K = W.shape
+    if row_ptr.dtype != torch.int32 or col_idx.dtype != torch.int32 or val.element_size() != 2:
+        raise ValueError("row_ptr / col_idx must be int32 and val 16-bit")
+    if row_ptr.numel() < N + 1:
+        raise ValueError("row_ptr too short")
+    cap = min(col_idx.numel(), val.numel())
+    nnz = C.c_int64(0)
+    with torch.cuda.device(W.device):
+        st = lib.gwq_select_outliers_static(W.data_ptr(), G.data_ptr(), N, K, float(frac), row_ptr.data_ptr(),
+                                            col_idx.data_ptr(), val.data_ptr(), cap, C.byref(nnz), _stream_ptr())
+    _check(st, "gwq_select_outliers_static")
+    return int(nnz.value)
 
 
 def gwq_pack(W: torch.Tensor, S: Outliers, bits: int, group: int) -> Packed:
