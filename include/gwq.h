@@ -57,11 +57,14 @@ typedef struct gwq_outliers {
 } gwq_outliers;
 
 /* Packed layer.
- * codes: every run of 32 consecutive columns of a row is one little-endian integer of
- *   32*bits bits, column 32r+i in bits [bits*i, bits*i+bits), stored as `bits`
- *   consecutive uint32 words (least significant first).  Row n starts at word
- *   n * K*bits/32.  For 4 bits: word t of a row holds columns 8t..8t+7, column 8t+i in
- *   bits [4i, 4i+4).
+ * codes: uint32 [N, K*bits/32], `bits` words per run of 32 consecutive columns, in
+ *   pair-interleaved order: the low 16 bits of a word hold even columns, the high 16 bits
+ *   the odd columns that follow them.
+ *     4 bits: word t of a row holds columns 8t..8t+7; column 8t + 2j + e (j = 0..3,
+ *             e = 0,1) is in bits [16e + 4j, 16e + 4j + 4).
+ *     3 bits: word w (0..2) of run r holds columns 32r + 10w + 2p + e (p = 0..4, e = 0,1)
+ *             in bits [16e + 3p, 16e + 3p + 3); bit b of the codes of columns 32r+30 and
+ *             32r+31 is in bit 15 and bit 31 of word b.
  * scales: fp16 [N, K/group]; zeros: uint8 [N, K/group], each in [0, 2^bits - 1].
  * An outlier position stores the code z of its group, so its dense term is exactly 0. */
 typedef struct gwq_packed {

@@ -180,15 +180,41 @@ def quantize_codes(W, mask, scales, zeros, bits: int, group: int) -> np.ndarray:
 # --------------------------------------------------------------------------
 # Storage format (this project's own; the paper specifies none)
 # --------------------------------------------------------------------------
-def pack_codes(codes: np.ndarray, bits: int) -> np.ndarray:
-    """Pack codes [N, K] into little-endian 32-bit words.
+def _bit_positions(bits: int):
+    """For column i of a 32-column run: list of (word, bit offset, code bit) triples,
+    one per code bit, following the written format definition (see pack_codes)."""
+    pos = []
+    for i in range(32):
+        if bits == 4:
+            t, r = divmod(i, 8)          # word t holds columns 8t..8t+7
+            j, e = divmod(r, 2)          # column 8t + 2j + e
+            pos.append([(t, 16 * e + 4 * j + b, b) for b in range(4)])
+        elif bits == 3:
+            if i < 30:
+                w, r = divmod(i, 10)     # word w holds columns 10w..10w+9
+                p_, e = divmod(r, 2)     # column 10w + 2p + e
+                pos.append([(w, 16 * e + 3 * p_ + b, b) for b in range(3)])
+            else:
+                e = i - 30               # columns 30 / 31: bit b lives in word b, bit 15 / 31
+                pos.append([(b, 16 * e + 15, b) for b in range(3)])
+        else:
+            raise ValueError("bits must be 3 or 4")
+    return pos
 
-    Every run of 32 consecutive columns of a row is one little-endian integer
-    of 32*bits bits, column 32r+i occupying bits [bits*i, bits*(i+1)); the
-    integer is stored as `bits` consecutive uint32 words, least significant
-    first.  (For 4 bits this is simply: word t holds columns 8t..8t+7, column
-    8t+i in bits [4i, 4i+4).  For 3 bits, codes 10 and 21 of a run straddle
-    two words.)  Returns uint32 [N, K*bits/32].
+
+def pack_codes(codes: np.ndarray, bits: int) -> np.ndarray:
+    """Pack codes [N, K] into 32-bit words, `bits` words per run of 32 columns.
+
+    Pair-interleaved order: in every word the low 16 bits hold even columns and
+    the high 16 bits hold the odd columns that follow them, so that one mask
+    yields a (column 2j, column 2j+1) pair in the two halves of a register.
+      4 bits: word t of a row holds columns 8t..8t+7; column 8t + 2j + e
+              (j = 0..3, e = 0,1) sits in bits [16e + 4j, 16e + 4j + 4).
+      3 bits: word w (0..2) of run r holds columns 32r + 10w + 2p + e
+              (p = 0..4, e = 0,1) in bits [16e + 3p, 16e + 3p + 3); bit b of the
+              codes of columns 32r+30 and 32r+31 sits in bit 15 and bit 31 of
+              word b.
+    Returns uint32 [N, K*bits/32].
     """
     N, K = codes.shape
     if K % 32 != 0:
@@ -196,30 +222,22 @@ def pack_codes(codes: np.ndarray, bits: int) -> np.ndarray:
     if codes.max(initial=0) > 2 ** bits - 1:
         raise ValueError("code out of range")
     out = np.zeros((N, K // 32, bits), dtype=np.uint32)
-    c = codes.reshape(N, K // 32, 32).astype(np.uint64)
-    for i in range(32):
-        pos = bits * i
-        word, off = divmod(pos, 32)
-        out[:, :, word] |= ((c[:, :, i] << np.uint64(off)) & np.uint64(0xFFFFFFFF)).astype(np.uint32)
-        if off + bits > 32:
-            out[:, :, word + 1] |= (c[:, :, i] >> np.uint64(32 - off)).astype(np.uint32)
+    c = codes.reshape(N, K // 32, 32).astype(np.uint32)
+    for i, triples in enumerate(_bit_positions(bits)):
+        for (word, off, b) in triples:
+            out[:, :, word] |= ((c[:, :, i] >> np.uint32(b)) & np.uint32(1)) << np.uint32(off)
     return out.reshape(N, K * bits // 32)
 
 
 def unpack_codes(words: np.ndarray, bits: int, K: int) -> np.ndarray:
     """Inverse of pack_codes.  Returns codes uint8 [N, K]."""
     N = words.shape[0]
-    w = words.reshape(N, K // 32, bits).astype(np.uint64)
-    codes = np.zeros((N, K // 32, 32), dtype=np.uint8)
-    m = np.uint64(2 ** bits - 1)
-    for i in range(32):
-        pos = bits * i
-        word, off = divmod(pos, 32)
-        v = w[:, :, word] >> np.uint64(off)
-        if off + bits > 32:
-            v = v | (w[:, :, word + 1] << np.uint64(32 - off))
-        codes[:, :, i] = (v & m).astype(np.uint8)
-    return codes.reshape(N, K)
+    w = words.reshape(N, K // 32, bits).astype(np.uint32)
+    codes = np.zeros((N, K // 32, 32), dtype=np.uint32)
+    for i, triples in enumerate(_bit_positions(bits)):
+        for (word, off, b) in triples:
+            codes[:, :, i] |= ((w[:, :, word] >> np.uint32(off)) & np.uint32(1)) << np.uint32(b)
+    return codes.reshape(N, K).astype(np.uint8)
 
 
 # --------------------------------------------------------------------------

@@ -1,7 +1,7 @@
 // General CUDA-core path of y = x (s (q - z) + S)^T (Section 3.2, Eq. "w").
 //
 // One warp owns one output row at a time: each lane takes runs of 32 columns (the
-// unit of the packed format), unpacks the codes with 64-bit shifts, accumulates
+// unit of the packed format), unpacks the codes one by one, accumulates
 // sum_k x_k (q_k - z) per run in FP32 and scales it by s once per run; the row's CSR
 // outliers are appended, then the lanes are reduced with shuffles.  It handles every
 // M by looping over tiles of 4 tokens and serves the shapes the specialised paths do
@@ -41,7 +41,6 @@ linear_simt_kernel(const uint32_t* __restrict__ codes, const uint16_t* __restric
   const int wid = blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5);
   const int nruns = K / 32;
   const int ngroups = K / group;
-  const unsigned long long cmask = (1ull << bits) - 1ull;
   for (int row = wid; row < N; row += warps_total) {
     const uint32_t* crow = codes + (long long)row * nruns * bits;
     const int jb = row_ptr[row], je = row_ptr[row + 1];
@@ -59,10 +58,19 @@ linear_simt_kernel(const uint32_t* __restrict__ codes, const uint16_t* __restric
 #pragma unroll
         for (int t = 0; t < MT; ++t) part[t] = 0.f;
         for (int i = 0; i < 32; ++i) {
-          const int pos = i * bits;
-          const int wi = pos >> 5, off = pos & 31;
-          const unsigned long long two = (unsigned long long)w[wi] | ((unsigned long long)w[(wi + 1) & 3] << 32);
-          const float qz = (float)(int)((two >> off) & cmask) - z;
+          // pair-interleaved packed order (see include/gwq.h)
+          unsigned int code;
+          const int e = i & 1;
+          if (bits == 4) {
+            code = (w[i >> 3] >> (16 * e + 4 * ((i & 7) >> 1))) & 15u;
+          } else if (i < 30) {
+            const int wi = i / 10, r10 = i - 10 * wi;
+            code = (w[wi] >> (16 * e + 3 * (r10 >> 1))) & 7u;
+          } else {
+            const int sh = 15 + 16 * e;
+            code = ((w[0] >> sh) & 1u) | (((w[1] >> sh) & 1u) << 1) | (((w[2] >> sh) & 1u) << 2);
+          }
+          const float qz = (float)(int)code - z;
 #pragma unroll
           for (int t = 0; t < MT; ++t) {
             if (m0 + t < M) part[t] = fmaf(ld_act<BF16>(x + (long long)(m0 + t) * K + r * 32 + i), qz, part[t]);

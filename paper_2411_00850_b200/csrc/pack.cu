@@ -90,18 +90,28 @@ pack_row_kernel(const uint16_t* __restrict__ W, const int32_t* __restrict__ row_
   if (bad) atomicExch(status, (int32_t)GWQ_ERR_NONFINITE);
   __syncthreads();
 
-  // pack: word wi of the row belongs to run wi / bits, word j = wi % bits of that run
+  // pack (pair-interleaved order: even columns in the low half-word, odd in the high):
+  //  4 bits: word j of a run holds its columns 8j..8j+7, column 8j+2p+e in bits [16e+4p, +4)
+  //  3 bits: word j holds columns 10j..10j+9, column 10j+2p+e in bits [16e+3p, +3); bit j of the
+  //          codes of columns 30 / 31 goes to bit 15 / 31 of word j
   const int nwords = K / 32 * bits;
   uint32_t* crow = codes + (long long)row * nwords;
   for (int wi = threadIdx.x; wi < nwords; wi += kThreads) {
     const int run = wi / bits, j = wi - run * bits;
-    const unsigned char* c = q8 + run * 32;
-    const int first = (32 * j) / bits;
+    const unsigned char* r = q8 + run * 32;
     unsigned int word = 0;
-    for (int i = first; i < 32 && i * bits < 32 * j + 32; ++i) {
-      const int p = i * bits - 32 * j;
-      const unsigned int v = c[i];
-      word |= (p >= 0) ? (v << p) : (v >> (-p));
+    if (bits == 4) {
+      const unsigned char* c = r + 8 * j;
+#pragma unroll
+      for (int p = 0; p < 4; ++p)
+        word |= ((unsigned int)c[2 * p] << (4 * p)) | ((unsigned int)c[2 * p + 1] << (16 + 4 * p));
+    } else {
+      const unsigned char* c = r + 10 * j;
+#pragma unroll
+      for (int p = 0; p < 5; ++p)
+        word |= ((unsigned int)c[2 * p] << (3 * p)) | ((unsigned int)c[2 * p + 1] << (16 + 3 * p));
+      word |= (((unsigned int)r[30] >> j) & 1u) << 15;
+      word |= (((unsigned int)r[31] >> j) & 1u) << 31;
     }
     crow[wi] = word;
   }

@@ -175,17 +175,37 @@ def test_pack_golden_bytes():
         assert np.array_equal(orc.unpack_codes(words, c["bits"], 32), codes)
 
 
+def _pack_run_scalar(codes32, bits):
+    """The written format definition, one column at a time, in plain Python integers."""
+    words = [0] * bits
+    for i, c in enumerate(codes32):
+        c = int(c)
+        if bits == 4:
+            t, j, e = i // 8, (i % 8) // 2, i % 2
+            words[t] |= c << (16 * e + 4 * j)
+        else:
+            if i < 30:
+                w, p_, e = i // 10, (i % 10) // 2, i % 2
+                words[w] |= c << (16 * e + 3 * p_)
+            else:
+                for b in range(3):
+                    words[b] |= ((c >> b) & 1) << (15 if i == 30 else 31)
+    return words
+
+
 @pytest.mark.parametrize("bits", [3, 4])
-def test_pack_matches_bigint_definition_and_roundtrips(bits):
+def test_pack_matches_scalar_definition_and_roundtrips(bits):
     rng = np.random.default_rng(bits)
     codes = rng.integers(0, 2 ** bits, size=(5, 160), dtype=np.uint8)
     words = orc.pack_codes(codes, bits)
     assert words.shape == (5, 160 * bits // 32) and words.dtype == np.uint32
     for n in range(5):
         for r in range(160 // 32):
-            big = sum(int(c) << (bits * i) for i, c in enumerate(codes[n, 32 * r:32 * r + 32]))
-            want = [(big >> (32 * j)) & 0xFFFFFFFF for j in range(bits)]
+            want = _pack_run_scalar(codes[n, 32 * r:32 * r + 32], bits)
             assert [int(w) for w in words[n, bits * r:bits * r + bits]] == want
     assert np.array_equal(orc.unpack_codes(words, bits, 160), codes)
+    # every bit of every word is used exactly once: all-ones codes fill the words
+    full = orc.pack_codes(np.full((1, 32), 2 ** bits - 1, dtype=np.uint8), bits)
+    assert [int(w) for w in full[0]] == [0xFFFFFFFF] * bits
     with pytest.raises(ValueError):
         orc.pack_codes(np.full((1, 32), 2 ** bits, dtype=np.uint8), bits)
