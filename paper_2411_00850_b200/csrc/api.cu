@@ -11,6 +11,7 @@ extern "C" gwq_status gwq_linear(const gwq_packed* P, const void* x, gwq_dtype x
   if (yd != GWQ_F16 && yd != GWQ_BF16 && yd != GWQ_F32) return GWQ_ERR_INVALID_ARG;
   if (!gwq_aligned16(x) || !gwq_aligned16(y)) return GWQ_ERR_INVALID_ARG;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  if (M <= 32) return gwq_launch_decode(P, x, xd, M, y, yd, stream);
   return gwq_launch_simt(P, x, xd, M, y, yd, stream);
 }
 
@@ -71,7 +72,7 @@ extern "C" void gwq_free(void* obj) {
     free_outliers(P->S);
     gwq_priv* pv = static_cast<gwq_priv*>(P->priv);
     if (pv) {
-      if (pv->col16) cudaFree(pv->col16);
+      if (pv->cv) cudaFree(pv->cv);
       if (pv->x_stage) cudaFree(pv->x_stage);
       if (pv->y_stage) cudaFree(pv->y_stage);
       if (pv->dev_status) cudaFree(pv->dev_status);

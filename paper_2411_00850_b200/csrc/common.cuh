@@ -24,7 +24,7 @@
 
 // Kernel-private part of a packed layer.
 struct gwq_priv {
-  uint16_t* col16;       // outlier columns narrowed to 16 bit (NULL when K > 65536)
+  uint32_t* cv;          // per outlier: fp16 value << 16 | column (NULL when K > 65536)
   void* x_stage;         // staging for gwq_linear_host
   void* y_stage;
   size_t x_stage_bytes;

@@ -117,9 +117,11 @@ pack_row_kernel(const uint16_t* __restrict__ W, const int32_t* __restrict__ row_
   }
 }
 
-__global__ void narrow_cols_kernel(const int32_t* __restrict__ col, uint16_t* __restrict__ col16, long long n) {
+// Decode-side copy of the CSR payload: one 32-bit word per outlier, value << 16 | column.
+__global__ void fuse_col_val_kernel(const int32_t* __restrict__ col, const uint16_t* __restrict__ val,
+                                    uint32_t* __restrict__ cv, long long n) {
   const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < n) col16[i] = (uint16_t)col[i];
+  if (i < n) cv[i] = ((uint32_t)val[i] << 16) | ((uint32_t)col[i] & 0xFFFFu);
 }
 
 }  // namespace
@@ -171,9 +173,9 @@ extern "C" gwq_status gwq_pack(const uint16_t* W, gwq_outliers* S, int32_t N, in
   GWQ_CUDA_TRY(cudaGetLastError());
   if (K <= 65536) {
     const long long nnz = S->nnz;
-    GWQ_CUDA_TRY(cudaMalloc(&pv->col16, (size_t)(nnz > 0 ? nnz : 1) * sizeof(uint16_t) + 16));
+    GWQ_CUDA_TRY(cudaMalloc(&pv->cv, (size_t)(nnz > 0 ? nnz : 1) * sizeof(uint32_t) + 16));
     if (nnz > 0) {
-      narrow_cols_kernel<<<(unsigned)((nnz + 255) / 256), 256, 0, stream>>>(S->col_idx, pv->col16, nnz);
+      fuse_col_val_kernel<<<(unsigned)((nnz + 255) / 256), 256, 0, stream>>>(S->col_idx, S->val, pv->cv, nnz);
       GWQ_CUDA_TRY(cudaGetLastError());
     }
   }
@@ -191,7 +193,7 @@ fail:
   if (P->codes) cudaFree(P->codes);
   if (P->scales) cudaFree(P->scales);
   if (P->zeros) cudaFree(P->zeros);
-  if (pv->col16) cudaFree(pv->col16);
+  if (pv->cv) cudaFree(pv->cv);
   if (pv->dev_status) cudaFree(pv->dev_status);
   delete pv;
   delete P;
