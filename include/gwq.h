@@ -144,6 +144,12 @@ gwq_status gwq_linear(const gwq_packed* P, const void* x, gwq_dtype x_dtype, int
 gwq_status gwq_linear_host(gwq_packed* P, const void* x_host, gwq_dtype x_dtype, int32_t M,
                            void* y_host, gwq_dtype y_dtype, void* stream);
 
+/* Device-side status of the gwq_linear calls made on P so far: synchronises `stream`, returns
+ * GWQ_OK or the error a kernel recorded (GWQ_ERR_TIMEOUT when a bounded wait inside the
+ * tensor-core path ran out and the kernel returned early; y is then undefined, and later
+ * tensor-core calls on P do no work until the status has been read) and clears it.            */
+gwq_status gwq_device_status(const gwq_packed* P, void* stream);
+
 /* Releases a gwq_outliers* or a gwq_packed* (and everything it owns).  NULL is a no-op. */
 void gwq_free(void* obj);
 

@@ -21,7 +21,7 @@ STATUS_NAMES = {
     0: "GWQ_OK", 1: "GWQ_ERR_INVALID_ARG", 2: "GWQ_ERR_UNSUPPORTED", 3: "GWQ_ERR_ALLOC",
     4: "GWQ_ERR_NONFINITE", 5: "GWQ_ERR_TIMEOUT", 6: "GWQ_ERR_CUDA",
 }
-EXPORTS = ("gwq_select_outliers", "gwq_select_outliers_static", "gwq_pack", "gwq_linear", "gwq_linear_host", "gwq_free",
+EXPORTS = ("gwq_select_outliers", "gwq_select_outliers_static", "gwq_pack", "gwq_linear", "gwq_linear_host", "gwq_device_status", "gwq_free",
            "gwq_status_string")
 
 
@@ -69,6 +69,8 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
                                C.c_void_p]
     lib.gwq_linear_host.restype = C.c_int
     lib.gwq_linear_host.argtypes = lib.gwq_linear.argtypes
+    lib.gwq_device_status.restype = C.c_int
+    lib.gwq_device_status.argtypes = [C.POINTER(gwq_packed), C.c_void_p]
     lib.gwq_free.restype = None
     lib.gwq_free.argtypes = [C.c_void_p]
     lib.gwq_status_string.restype = C.c_char_p
@@ -300,6 +302,12 @@ def gwq_linear_host(P: Packed, x_host: torch.Tensor, y_host: torch.Tensor) -> to
                                  _dtype_code(y_host.dtype), _stream_ptr())
     _check(st, "gwq_linear_host")
     return y_host
+
+
+def gwq_device_status(P: Packed) -> int:
+    """Status recorded by the kernels of earlier gwq_linear calls on P (0 = ok); synchronises."""
+    with torch.cuda.device(P.device):
+        return int(load_library().gwq_device_status(P._h, _stream_ptr()))
 
 
 def gwq_free(obj) -> None:

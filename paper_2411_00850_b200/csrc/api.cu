@@ -12,7 +12,7 @@ extern "C" gwq_status gwq_linear(const gwq_packed* P, const void* x, gwq_dtype x
   if (!gwq_aligned16(x) || !gwq_aligned16(y)) return GWQ_ERR_INVALID_ARG;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
   if (M <= 32) return gwq_launch_decode(P, x, xd, M, y, yd, stream);
-  return gwq_launch_simt(P, x, xd, M, y, yd, stream);
+  return gwq_launch_prefill(P, x, xd, M, y, yd, stream);
 }
 
 extern "C" gwq_status gwq_linear_host(gwq_packed* P, const void* x_host, gwq_dtype xd, int32_t M,
@@ -48,6 +48,20 @@ extern "C" gwq_status gwq_linear_host(gwq_packed* P, const void* x_host, gwq_dty
   return GWQ_OK;
 fail:
   return st;
+}
+
+extern "C" gwq_status gwq_device_status(const gwq_packed* P, void* stream_) {
+  if (!P || P->tag != GWQ_TAG_PACKED || !P->priv) return GWQ_ERR_INVALID_ARG;
+  const gwq_priv* pv = static_cast<const gwq_priv*>(P->priv);
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  int32_t h = 0;
+  if (cudaMemcpyAsync(&h, pv->dev_status, sizeof(h), cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+      cudaStreamSynchronize(stream) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return GWQ_ERR_CUDA;
+  }
+  if (h != 0) (void)cudaMemsetAsync(pv->dev_status, 0, sizeof(int32_t), stream);
+  return (gwq_status)h;
 }
 
 static void free_outliers(gwq_outliers* S) {

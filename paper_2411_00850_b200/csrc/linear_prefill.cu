@@ -1,0 +1,415 @@
+// Prefill path (M > 32) of y = x (s (q - z) + S)^T (Section 3.2, Eq. "w"): a dense contraction
+// on the 5th-generation tensor cores.
+//
+// One CTA computes a tile of 128 output features x TOK tokens.  The weight rows are the M side
+// of the MMA (A operand), the tokens its N side (B operand); both are K-major in shared memory
+// in the 128-byte-swizzled layout, the FP32 accumulator lives in tensor memory.
+//   warp 0, one thread : TMA loads of the activation tile (TOK x 64) per k-block
+//   warp 1, one thread : tcgen05.mma (4 x K=16 per k-block), tcgen05.commit frees the stage
+//   warps 2..5         : one thread per weight row: packed codes from global memory -> exact
+//                        q - z by a magic-number subtract -> times the group scale -> 128 bytes
+//                        of the swizzled A tile; the row's CSR outliers are written over their
+//                        (exactly zero) dense entries, so the tensor cores also do the SpMM;
+//                        afterwards the same warps drain the accumulator (tcgen05.ld) and store y
+// Stages are handed over with mbarriers; every wait is bounded and, when it runs out, the CTA
+// records GWQ_ERR_TIMEOUT, leaves its loops, frees its tensor memory and returns.
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace {
+
+constexpr int kTileN = 128;      // weight rows per CTA (UMMA M)
+constexpr int kBlockK = 64;      // k-block: 128 bytes of 16-bit operands
+constexpr int kDequantWarps = 4;
+constexpr int kThreads = 32 * (2 + kDequantWarps);
+constexpr int kMaxStages = 8;
+constexpr long long kSpinCycles = 1000LL * 1000LL * 1000LL;   // about half a second of SM clock
+
+__device__ __forceinline__ unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(unsigned bar, unsigned count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(unsigned bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(unsigned bar, unsigned bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// Bounded wait for the phase with the given parity: gives up (false) after kSpinCycles, or as
+// soon as another role of the CTA has given up.
+__device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity, volatile int* abort_flag) {
+  const long long t0 = clock64();
+  for (unsigned it = 0;; ++it) {
+    unsigned done;
+    asm volatile(
+        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.b32 %0, 1, 0, p;\n}\n"
+        : "=r"(done)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    if (done) return true;
+    if ((it & 63u) == 63u && (*abort_flag || clock64() - t0 > kSpinCycles)) return false;
+  }
+}
+
+__device__ __forceinline__ void tma_load_2d(unsigned dst, const CUtensorMap* map, int c0, int c1, unsigned bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar)
+      : "memory");
+}
+
+// Shared-memory matrix descriptor, K-major, 128-byte swizzle: rows of 128 bytes, 8-row atoms
+// 1024 bytes apart (tile base 1024-byte aligned).
+__device__ __forceinline__ uint64_t umma_desc(unsigned smem_addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr >> 4) & 0x3FFFu);   // start address, 16-byte units
+  d |= (uint64_t)1 << 16;                        // leading byte offset (not used by swizzled K-major)
+  d |= (uint64_t)(1024 >> 4) << 32;              // stride byte offset: next 8-row atom
+  d |= (uint64_t)1 << 46;                        // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;                        // layout type: 128-byte swizzle
+  return d;
+}
+
+__device__ __forceinline__ void umma_f16(unsigned tmem_d, uint64_t da, uint64_t db, unsigned idesc, unsigned accumulate) {
+  asm volatile(
+      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+      " tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
+      ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(unsigned bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld32(unsigned taddr, unsigned (&v)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,"
+      "%29,%30,%31}, [%32];\n"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+        "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+        "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr)
+      : "memory");
+}
+
+struct PrefillArgs {
+  const uint32_t* codes;
+  const uint16_t* scales;
+  const uint8_t* zeros;
+  const int32_t* row_ptr;
+  const uint32_t* cv;   // per outlier: fp16 value << 16 | column
+  void* y;
+  gwq_dtype yd;
+  int32_t* status;
+  int N, K, M, group;
+};
+
+template <bool BF16>
+__device__ __forceinline__ unsigned mul_scale(unsigned d, unsigned s_hi2, unsigned s_lo2) {
+  if (BF16) {
+    // s = s_hi + s_lo exactly (both bf16): d s_hi + (d s_lo) keeps the bits of s that bf16 alone would drop
+    const __nv_bfloat162 dd = *reinterpret_cast<const __nv_bfloat162*>(&d);
+    const __nv_bfloat162 r = __hfma2(dd, *reinterpret_cast<const __nv_bfloat162*>(&s_hi2),
+                                     __hmul2(dd, *reinterpret_cast<const __nv_bfloat162*>(&s_lo2)));
+    return *reinterpret_cast<const unsigned*>(&r);
+  } else {
+    const __half2 r = __hmul2(*reinterpret_cast<const __half2*>(&d), *reinterpret_cast<const __half2*>(&s_hi2));
+    return *reinterpret_cast<const unsigned*>(&r);
+  }
+}
+template <bool BF16>
+__device__ __forceinline__ unsigned sub_magic(unsigned qm, unsigned zm) {
+  if (BF16) {
+    const __nv_bfloat162 r =
+        __hsub2(*reinterpret_cast<const __nv_bfloat162*>(&qm), *reinterpret_cast<const __nv_bfloat162*>(&zm));
+    return *reinterpret_cast<const unsigned*>(&r);
+  } else {
+    const __half2 r = __hsub2(*reinterpret_cast<const __half2*>(&qm), *reinterpret_cast<const __half2*>(&zm));
+    return *reinterpret_cast<const unsigned*>(&r);
+  }
+}
+
+template <int BITS, int TOK, bool BF16>
+__global__ void __launch_bounds__(kThreads, 1)
+prefill_kernel(const __grid_constant__ CUtensorMap tmx, const PrefillArgs p, const int stages) {
+  constexpr int kABytes = kTileN * kBlockK * 2;   // 16 KB
+  constexpr int kBBytes = TOK * kBlockK * 2;
+  extern __shared__ unsigned char smem_dyn[];
+  unsigned char* tiles =
+      reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
+  __shared__ __align__(8) unsigned long long bars[3 * kMaxStages + 1];
+  __shared__ unsigned tmem_base_s;
+  __shared__ int abort_s;
+  volatile int* abort_flag = &abort_s;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int n0 = blockIdx.x * kTileN, m0 = blockIdx.y * TOK;
+  const int nkb = p.K / kBlockK;
+  const unsigned bar0 = smem_u32(bars);
+  auto full_b = [&](int s) { return bar0 + 8u * s; };
+  auto full_a = [&](int s) { return bar0 + 8u * (kMaxStages + s); };
+  auto empty = [&](int s) { return bar0 + 8u * (2 * kMaxStages + s); };
+  const unsigned accum_bar = bar0 + 8u * (3 * kMaxStages);
+  auto a_tile = [&](int s) { return tiles + (size_t)s * (kABytes + kBBytes); };
+  auto b_tile = [&](int s) { return tiles + (size_t)s * (kABytes + kBBytes) + kABytes; };
+
+  if (tid == 0) {
+    abort_s = 0;
+    for (int s = 0; s < stages; ++s) {
+      mbar_init(full_b(s), 1);
+      mbar_init(full_a(s), kDequantWarps);
+      mbar_init(empty(s), 1);
+    }
+    mbar_init(accum_bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {   // tensor memory for the accumulator: TOK columns of 128 lanes
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)),
+                 "r"(TOK)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const unsigned tmem_acc = tmem_base_s;
+  bool ok = *reinterpret_cast<volatile int32_t*>(p.status) == 0;   // an earlier CTA gave up: do no work
+  int issued = 0;   // k-blocks whose activation copy was started (producer thread only)
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ activation tiles by TMA
+    if (lane == 0) {
+      for (int kb = 0; kb < nkb && ok; ++kb) {
+        const int s = kb % stages, round = kb / stages;
+        if (round > 0) ok = mbar_wait(empty(s), (round - 1) & 1, abort_flag);
+        if (!ok) break;
+        mbar_expect_tx(full_b(s), kBBytes);
+        tma_load_2d(smem_u32(b_tile(s)), &tmx, kb * kBlockK, m0, full_b(s));
+        issued = kb + 1;
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issue
+    if (lane == 0) {
+      // instruction descriptor: FP32 accumulate, A and B both fp16 or both bf16, K-major, N = TOK, M = 128
+      const unsigned idesc = (1u << 4) | ((BF16 ? 1u : 0u) << 7) | ((BF16 ? 1u : 0u) << 10) |
+                             ((unsigned)(TOK >> 3) << 17) | ((unsigned)(kTileN >> 4) << 24);
+      for (int kb = 0; kb < nkb && ok; ++kb) {
+        const int s = kb % stages, round = kb / stages;
+        ok = mbar_wait(full_a(s), round & 1, abort_flag) && mbar_wait(full_b(s), round & 1, abort_flag);
+        if (!ok) break;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint64_t da = umma_desc(smem_u32(a_tile(s))), db = umma_desc(smem_u32(b_tile(s)));
+#pragma unroll
+        for (int k = 0; k < kBlockK / 16; ++k)   // 32 bytes further along K inside the swizzle atom
+          umma_f16(tmem_acc, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (kb | k) != 0);
+        umma_commit(empty(s));
+      }
+      if (ok) umma_commit(accum_bar);
+    }
+  } else {
+    // ------------------------------------------------------------------ dequantization, then epilogue
+    const int quad = warp & 3;                 // tensor-memory lane quarter this warp may access
+    const int r = quad * 32 + lane;            // row inside the tile
+    const int row = n0 + r;
+    const bool live = row < p.N;
+    const int rowc = live ? row : p.N - 1;
+    const int ngroups = p.K / p.group;
+    constexpr int WPB = kBlockK * BITS / 32;   // packed words per row per k-block (8 or 6)
+    const uint32_t* crow = p.codes + (size_t)rowc * (p.K / 32) * BITS;
+    const uint16_t* srow = p.scales + (size_t)rowc * ngroups;
+    const uint8_t* zrow = p.zeros + (size_t)rowc * ngroups;
+    int j = 0, je = 0;
+    if (live) {
+      j = p.row_ptr[row];
+      je = p.row_ptr[row + 1];
+    }
+    unsigned nxt = j < je ? __ldg(p.cv + j) : 0xFFFFFFFFu;   // next outlier of the row
+    constexpr unsigned MAGIC = BF16 ? 0x43004300u : 0x64006400u;   // 128.0 / 1024.0: ulp = 1
+    unsigned wq[WPB];
+#pragma unroll
+    for (int i = 0; i < WPB; ++i) wq[i] = __ldg(crow + i);
+    for (int kb = 0; kb < nkb && ok; ++kb) {
+      const int s = kb % stages, round = kb / stages;
+      const int g = (kb * kBlockK) / p.group;
+      const float sc = live ? __half2float(__ushort_as_half(__ldg(srow + g))) : 0.f;
+      const unsigned z = __ldg(zrow + g);
+      unsigned s_hi2, s_lo2 = 0;
+      if (BF16) {
+        const __nv_bfloat16 hi = __float2bfloat16_rn(sc);
+        const __nv_bfloat16 lo = __float2bfloat16_rn(sc - __bfloat162float(hi));
+        s_hi2 = (unsigned)__bfloat16_as_ushort(hi) * 0x00010001u;
+        s_lo2 = (unsigned)__bfloat16_as_ushort(lo) * 0x00010001u;
+      } else {
+        s_hi2 = (unsigned)__half_as_ushort(__float2half_rn(sc)) * 0x00010001u;
+      }
+      const unsigned zm = MAGIC | (z * 0x00010001u);
+      unsigned cur[WPB];
+#pragma unroll
+      for (int i = 0; i < WPB; ++i) cur[i] = wq[i];
+      if (kb + 1 < nkb) {
+#pragma unroll
+        for (int i = 0; i < WPB; ++i) wq[i] = __ldg(crow + (size_t)(kb + 1) * WPB + i);
+      }
+      // 64 codes -> 32 pairs (columns 2h, 2h+1) -> 8 chunks of 16 bytes
+      unsigned out[32];
+      if (BITS == 4) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+#pragma unroll
+          for (int q4 = 0; q4 < 4; ++q4)
+            out[4 * i + q4] = mul_scale<BF16>(
+                sub_magic<BF16>(((cur[i % WPB] >> (4 * q4)) & 0x000F000Fu) | MAGIC, zm), s_hi2, s_lo2);
+      } else {
+#pragma unroll
+        for (int run = 0; run < 2; ++run) {
+          const unsigned* w3 = cur + (run * 3) % WPB;
+#pragma unroll
+          for (int i = 0; i < 3; ++i)
+#pragma unroll
+            for (int pp = 0; pp < 5; ++pp)
+              out[16 * run + 5 * i + pp] =
+                  mul_scale<BF16>(sub_magic<BF16>(((w3[i] >> (3 * pp)) & 0x00070007u) | MAGIC, zm), s_hi2, s_lo2);
+          const unsigned last =
+              ((w3[0] >> 15) & 0x00010001u) | ((w3[1] >> 14) & 0x00020002u) | ((w3[2] >> 13) & 0x00040004u);
+          out[16 * run + 15] = mul_scale<BF16>(sub_magic<BF16>(last | MAGIC, zm), s_hi2, s_lo2);
+        }
+      }
+      if (round > 0) ok = mbar_wait(empty(s), (round - 1) & 1, abort_flag);
+      if (!ok) break;
+      unsigned char* arow = a_tile(s) + r * 128;
+#pragma unroll
+      for (int c = 0; c < 8; ++c)
+        *reinterpret_cast<uint4*>(arow + ((c ^ (r & 7)) << 4)) =
+            make_uint4(out[4 * c], out[4 * c + 1], out[4 * c + 2], out[4 * c + 3]);
+      // the row's outliers inside this k-block replace their dense entries (which are exactly 0)
+      const unsigned k_end = (unsigned)(kb + 1) * kBlockK;
+      while (j < je && (nxt & 0xFFFFu) < k_end) {
+        const unsigned col = (nxt & 0xFFFFu) - (unsigned)kb * kBlockK;
+        unsigned short v16 = (unsigned short)(nxt >> 16);
+        if (BF16) v16 = __bfloat16_as_ushort(__float2bfloat16_rn(__half2float(__ushort_as_half(v16))));
+        *reinterpret_cast<unsigned short*>(arow + ((((col >> 3) ^ (r & 7)) << 4) | ((col & 7) << 1))) = v16;
+        ++j;
+        nxt = j < je ? __ldg(p.cv + j) : 0xFFFFFFFFu;
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to the MMA
+      __syncwarp();
+      if (lane == 0) mbar_arrive(full_a(s));
+    }
+    // ---- epilogue: accumulator lane = output feature, column = token
+    if (ok) ok = mbar_wait(accum_bar, 0, abort_flag);
+    if (ok) {
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+#pragma unroll 1
+      for (int c0 = 0; c0 < TOK; c0 += 32) {
+        if (m0 + c0 >= p.M) break;             // warp-uniform
+        unsigned v[32];
+        tmem_ld32(tmem_acc + ((unsigned)(quad * 32) << 16) + (unsigned)c0, v);
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        if (live) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            const int m = m0 + c0 + i;
+            if (m < p.M) {
+              const float f = __uint_as_float(v[i]);
+              const size_t idx = (size_t)m * p.N + row;
+              if (p.yd == GWQ_F32) reinterpret_cast<float*>(p.y)[idx] = f;
+              else if (p.yd == GWQ_F16) reinterpret_cast<__half*>(p.y)[idx] = __float2half_rn(f);
+              else reinterpret_cast<__nv_bfloat16*>(p.y)[idx] = __float2bfloat16_rn(f);
+            }
+          }
+        }
+      }
+    }
+  }
+  if (!ok) {
+    *abort_flag = 1;
+    atomicExch(p.status, (int32_t)GWQ_ERR_TIMEOUT);
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 0 && lane == 0 && abort_s) {
+    // bulk copies that were issued must land before the shared memory is given back: wait (bounded)
+    // for the last phase armed on every stage
+    int zero = 0;
+    for (int s = 0; s < stages; ++s) {
+      if (issued > s) {
+        const int last_kb = ((issued - 1 - s) / stages) * stages + s;   // last k-block issued on stage s
+        (void)mbar_wait(full_b(s), (last_kb / stages) & 1, &zero);
+      }
+    }
+  }
+  __syncthreads();
+  if (warp == 1) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(TOK) : "memory");
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  }
+  return fn;
+}
+
+template <int BITS, int TOK, bool BF16>
+gwq_status launch(const gwq_packed* P, const void* x, int M, void* y, gwq_dtype yd, cudaStream_t stream) {
+  const gwq_priv* pv = static_cast<const gwq_priv*>(P->priv);
+  EncodeTiledFn enc = encode_fn();
+  if (!enc) return GWQ_ERR_CUDA;
+  CUtensorMap tmx;
+  const cuuint64_t dims[2] = {(cuuint64_t)P->K, (cuuint64_t)M};
+  const cuuint64_t strides[1] = {(cuuint64_t)P->K * 2};
+  const cuuint32_t box[2] = {(cuuint32_t)kBlockK, (cuuint32_t)TOK};
+  const cuuint32_t estr[2] = {1, 1};
+  if (enc(&tmx, BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(x),
+          dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return GWQ_ERR_CUDA;
+  const int stage_bytes = kTileN * kBlockK * 2 + TOK * kBlockK * 2;
+  int stages = (220 * 1024 - 1024) / stage_bytes;
+  if (stages > kMaxStages) stages = kMaxStages;
+  const size_t smem = (size_t)stages * stage_bytes + 1024;
+  if (cudaFuncSetAttribute(prefill_kernel<BITS, TOK, BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           (int)smem) != cudaSuccess)
+    return GWQ_ERR_CUDA;
+  PrefillArgs a;
+  a.codes = P->codes; a.scales = P->scales; a.zeros = P->zeros; a.row_ptr = P->S->row_ptr; a.cv = pv->cv;
+  a.y = y; a.yd = yd; a.status = pv->dev_status; a.N = P->N; a.K = P->K; a.M = M; a.group = P->group;
+  dim3 grid((unsigned)((P->N + kTileN - 1) / kTileN), (unsigned)((M + TOK - 1) / TOK));
+  prefill_kernel<BITS, TOK, BF16><<<grid, kThreads, smem, stream>>>(tmx, a, stages);
+  return cudaGetLastError() == cudaSuccess ? GWQ_OK : GWQ_ERR_CUDA;
+}
+
+template <int BITS, bool BF16>
+gwq_status launch_tok(const gwq_packed* P, const void* x, int M, void* y, gwq_dtype yd, cudaStream_t stream) {
+  if (M <= 64) return launch<BITS, 64, BF16>(P, x, M, y, yd, stream);
+  if (M <= 128) return launch<BITS, 128, BF16>(P, x, M, y, yd, stream);
+  return launch<BITS, 256, BF16>(P, x, M, y, yd, stream);
+}
+
+}  // namespace
+
+// Prefill launcher: K <= 65536 (16-bit outlier columns).  Other shapes go to the general kernel.
+gwq_status gwq_launch_prefill(const gwq_packed* P, const void* x, gwq_dtype xd, int M, void* y, gwq_dtype yd,
+                              cudaStream_t stream) {
+  const gwq_priv* pv = static_cast<const gwq_priv*>(P->priv);
+  if (!pv->cv || P->K % kBlockK != 0) return gwq_launch_simt(P, x, xd, M, y, yd, stream);
+  if (P->bits == 4)
+    return xd == GWQ_BF16 ? launch_tok<4, true>(P, x, M, y, yd, stream) : launch_tok<4, false>(P, x, M, y, yd, stream);
+  return xd == GWQ_BF16 ? launch_tok<3, true>(P, x, M, y, yd, stream) : launch_tok<3, false>(P, x, M, y, yd, stream);
+}

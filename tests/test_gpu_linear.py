@@ -68,6 +68,40 @@ def test_larger_batches(M, dtype):
     assert_linear_close(y, y_ref, bound)
 
 
+PREFILL_LAYERS = [
+    (1024, 1024, 0.01, 4, 128, 20),
+    (1024, 1024, 0.01, 3, 128, 21),
+    (1000, 2176, 0.02, 4, 64, 22),      # N not a multiple of the 128-row tile, group 64
+    (1000, 2176, 0.005, 3, 64, 23),
+    (256, 4096, 0.3, 4, 128, 25),       # outlier-heavy rows
+]
+
+
+@pytest.mark.parametrize("layer", PREFILL_LAYERS)
+@pytest.mark.parametrize("M,dtype", [(33, "f16"), (64, "bf16"), (65, "f16"), (200, "bf16"), (256, "f16"),
+                                     (257, "bf16"), (700, "f16")])
+def test_tensor_core_path(layer, M, dtype):
+    P, L, w_hat = _layer(*layer)
+    bits16, xv = synth.make_activations(M, P.K, seed=100 + M, dtype=dtype, heavy_channels=8)
+    y_ref, bound = orc.linear(xv, w_hat)
+    y = gwq.gwq_linear(P, x_tensor(bits16, dtype), out_dtype=torch.float32)
+    assert gwq.gwq_device_status(P) == 0
+    assert_linear_close(y, y_ref, bound)
+    y16 = gwq.gwq_linear(P, x_tensor(bits16, dtype))
+    assert_linear_close(y16, y_ref, bound, extra_rel=2.0 ** -9 if dtype == "bf16" else 0.0)
+
+
+def test_tensor_core_path_reads_back_columns_exactly_in_fp16():
+    # one-hot fp16 activations: y[m] is column c of the reconstructed weight, outliers included
+    P, L, w_hat = _layer(*PREFILL_LAYERS[0])
+    cols = list(range(0, 1024, 17)) + [int(c) for c in L["col_idx"][:20]]
+    bits16, xv = synth.unit_activations(cols, P.K, "f16")
+    assert len(cols) > 64
+    y_ref, bound = orc.linear(xv, w_hat)
+    y = gwq.gwq_linear(P, x_tensor(bits16, "f16"), out_dtype=torch.float32)
+    assert_linear_close(y, y_ref, bound)
+
+
 def test_all_outliers_is_the_dense_product():
     N, K = 128, 512
     W, G = synth.make_weight_and_grad(N, K, 30)
