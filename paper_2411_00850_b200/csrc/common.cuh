@@ -29,6 +29,8 @@ struct gwq_priv {
   void* y_stage;
   size_t x_stage_bytes;
   size_t y_stage_bytes;
+  void* x16;             // fp16 copy of bf16 activations for the tensor-core path (+ per-token scales)
+  size_t x16_bytes;
   int32_t* dev_status;   // device status word written by bounded waits
   int sm_count;
 };

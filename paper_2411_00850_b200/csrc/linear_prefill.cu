@@ -11,6 +11,11 @@
 //                        of the swizzled A tile; the row's CSR outliers are written over their
 //                        (exactly zero) dense entries, so the tensor cores also do the SpMM;
 //                        afterwards the same warps drain the accumulator (tcgen05.ld) and store y
+// The tensor cores always run in fp16: bf16 activations are first rewritten, one pass, as
+// fp16 x 2^-e with one power of two per token (exact for every element within 2^-14 of the
+// token's largest, i.e. for everything that matters), because weights rounded to bf16 (8 bits)
+// cannot meet the 1e-3 tolerance when a few activation channels dominate a sum; the epilogue
+// multiplies the token's column by 2^e again.  fp16 also keeps the FP16 outliers exact.
 // Stages are handed over with mbarriers; every wait is bounded and, when it runs out, the CTA
 // records GWQ_ERR_TIMEOUT, leaves its loops, frees its tensor memory and returns.
 #include <cuda.h>
@@ -105,8 +110,51 @@ struct PrefillArgs {
   void* y;
   gwq_dtype yd;
   int32_t* status;
+  const float* tok_scale;   // per token 2^e, or null (activations were fp16 already)
   int N, K, M, group;
 };
+
+// bf16 [M,K] -> fp16 [M,K] scaled per token row by a power of two that puts the row's largest
+// magnitude just below 2^15; tok_scale[m] receives the inverse factor.  One CTA per token.
+__global__ void __launch_bounds__(256) bf16_rows_to_scaled_f16(const uint16_t* __restrict__ x, uint16_t* __restrict__ x16,
+                                                               float* __restrict__ tok_scale, int K) {
+  __shared__ float red[8];
+  const uint16_t* row = x + (size_t)blockIdx.x * K;
+  uint16_t* out = x16 + (size_t)blockIdx.x * K;
+  unsigned amax = 0;   // largest |x| as a bf16 bit pattern (monotone in magnitude)
+  for (int i = threadIdx.x; i < K / 8; i += 256) {
+    const uint4 v = __ldg(reinterpret_cast<const uint4*>(row) + i);
+    const unsigned w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      amax = max(amax, w[j] & 0x7FFFu);
+      amax = max(amax, (w[j] >> 16) & 0x7FFFu);
+    }
+  }
+  for (int o = 16; o > 0; o >>= 1) amax = max(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, o));
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = __uint_as_float(amax);
+  __syncthreads();
+  for (int w = 0; w < 8; ++w) amax = max(amax, __float_as_uint(red[w]));
+  // exponent of the largest magnitude (non-finite inputs keep e = 0 and simply propagate)
+  const int ex = (int)(amax >> 7) & 0xFF;
+  int e = (ex == 0 || ex == 0xFF) ? 0 : ex - 127 - 14;
+  e = max(-100, min(100, e));
+  const float down = __uint_as_float((unsigned)(127 - e) << 23);   // 2^-e
+  if (threadIdx.x == 0) tok_scale[blockIdx.x] = __uint_as_float((unsigned)(127 + e) << 23);
+  for (int i = threadIdx.x; i < K / 8; i += 256) {
+    const uint4 v = __ldg(reinterpret_cast<const uint4*>(row) + i);
+    const unsigned w[4] = {v.x, v.y, v.z, v.w};
+    unsigned o4[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float lo = __uint_as_float(w[j] << 16) * down, hi = __uint_as_float(w[j] & 0xFFFF0000u) * down;
+      const __half2 h = __floats2half2_rn(lo, hi);
+      o4[j] = *reinterpret_cast<const unsigned*>(&h);
+    }
+    reinterpret_cast<uint4*>(out)[i] = make_uint4(o4[0], o4[1], o4[2], o4[3]);
+  }
+}
+
 
 template <bool BF16>
 __device__ __forceinline__ unsigned mul_scale(unsigned d, unsigned s_hi2, unsigned s_lo2) {
@@ -315,7 +363,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmx, const PrefillArgs p, con
           for (int i = 0; i < 32; ++i) {
             const int m = m0 + c0 + i;
             if (m < p.M) {
-              const float f = __uint_as_float(v[i]);
+              float f = __uint_as_float(v[i]);
+              if (p.tok_scale) f *= __ldg(p.tok_scale + m);
               const size_t idx = (size_t)m * p.N + row;
               if (p.yd == GWQ_F32) reinterpret_cast<float*>(p.y)[idx] = f;
               else if (p.yd == GWQ_F16) reinterpret_cast<__half*>(p.y)[idx] = __float2half_rn(f);
@@ -366,8 +415,10 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-template <int BITS, int TOK, bool BF16>
-gwq_status launch(const gwq_packed* P, const void* x, int M, void* y, gwq_dtype yd, cudaStream_t stream) {
+template <int BITS, int TOK>
+gwq_status launch(const gwq_packed* P, const void* x, const float* tok_scale, int M, void* y, gwq_dtype yd,
+                  cudaStream_t stream) {
+  constexpr bool BF16 = false;   // operands are always fp16 here (see the file header)
   const gwq_priv* pv = static_cast<const gwq_priv*>(P->priv);
   EncodeTiledFn enc = encode_fn();
   if (!enc) return GWQ_ERR_CUDA;
@@ -389,27 +440,50 @@ gwq_status launch(const gwq_packed* P, const void* x, int M, void* y, gwq_dtype 
     return GWQ_ERR_CUDA;
   PrefillArgs a;
   a.codes = P->codes; a.scales = P->scales; a.zeros = P->zeros; a.row_ptr = P->S->row_ptr; a.cv = pv->cv;
-  a.y = y; a.yd = yd; a.status = pv->dev_status; a.N = P->N; a.K = P->K; a.M = M; a.group = P->group;
+  a.y = y; a.yd = yd; a.status = pv->dev_status; a.tok_scale = tok_scale; a.N = P->N; a.K = P->K; a.M = M; a.group = P->group;
   dim3 grid((unsigned)((P->N + kTileN - 1) / kTileN), (unsigned)((M + TOK - 1) / TOK));
   prefill_kernel<BITS, TOK, BF16><<<grid, kThreads, smem, stream>>>(tmx, a, stages);
   return cudaGetLastError() == cudaSuccess ? GWQ_OK : GWQ_ERR_CUDA;
 }
 
-template <int BITS, bool BF16>
-gwq_status launch_tok(const gwq_packed* P, const void* x, int M, void* y, gwq_dtype yd, cudaStream_t stream) {
-  if (M <= 64) return launch<BITS, 64, BF16>(P, x, M, y, yd, stream);
-  if (M <= 128) return launch<BITS, 128, BF16>(P, x, M, y, yd, stream);
-  return launch<BITS, 256, BF16>(P, x, M, y, yd, stream);
+template <int BITS>
+gwq_status launch_tok(const gwq_packed* P, const void* x, const float* tok_scale, int M, void* y, gwq_dtype yd,
+                      cudaStream_t stream) {
+  if (M <= 64) return launch<BITS, 64>(P, x, tok_scale, M, y, yd, stream);
+  if (M <= 128) return launch<BITS, 128>(P, x, tok_scale, M, y, yd, stream);
+  return launch<BITS, 256>(P, x, tok_scale, M, y, yd, stream);
 }
 
 }  // namespace
 
 // Prefill launcher: K <= 65536 (16-bit outlier columns).  Other shapes go to the general kernel.
+// bf16 activations need a scratch copy of x in fp16 (M K 2 bytes + M 4 bytes), kept in the packed
+// object and grown on demand (a growing call synchronises the stream and allocates).
 gwq_status gwq_launch_prefill(const gwq_packed* P, const void* x, gwq_dtype xd, int M, void* y, gwq_dtype yd,
                               cudaStream_t stream) {
-  const gwq_priv* pv = static_cast<const gwq_priv*>(P->priv);
+  gwq_priv* pv = static_cast<gwq_priv*>(P->priv);
   if (!pv->cv || P->K % kBlockK != 0) return gwq_launch_simt(P, x, xd, M, y, yd, stream);
-  if (P->bits == 4)
-    return xd == GWQ_BF16 ? launch_tok<4, true>(P, x, M, y, yd, stream) : launch_tok<4, false>(P, x, M, y, yd, stream);
-  return xd == GWQ_BF16 ? launch_tok<3, true>(P, x, M, y, yd, stream) : launch_tok<3, false>(P, x, M, y, yd, stream);
+  const float* tok_scale = nullptr;
+  if (xd == GWQ_BF16) {
+    const size_t need = (size_t)M * P->K * 2 + (size_t)M * 4 + 256;
+    if (pv->x16_bytes < need) {
+      if (cudaStreamSynchronize(stream) != cudaSuccess) return GWQ_ERR_CUDA;
+      if (pv->x16) cudaFree(pv->x16);
+      pv->x16 = nullptr;
+      pv->x16_bytes = 0;
+      if (cudaMalloc(&pv->x16, need) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return GWQ_ERR_ALLOC;
+      }
+      pv->x16_bytes = need;
+    }
+    float* ts = reinterpret_cast<float*>(static_cast<char*>(pv->x16) + (((size_t)M * P->K * 2 + 255) & ~(size_t)255));
+    bf16_rows_to_scaled_f16<<<M, 256, 0, stream>>>(static_cast<const uint16_t*>(x), static_cast<uint16_t*>(pv->x16), ts,
+                                                   P->K);
+    if (cudaGetLastError() != cudaSuccess) return GWQ_ERR_CUDA;
+    x = pv->x16;
+    tok_scale = ts;
+  }
+  if (P->bits == 4) return launch_tok<4>(P, x, tok_scale, M, y, yd, stream);
+  return launch_tok<3>(P, x, tok_scale, M, y, yd, stream);
 }
