@@ -6,7 +6,8 @@
 // in the 128-byte-swizzled layout, the FP32 accumulator lives in tensor memory.
 //   warp 0, one thread : TMA loads of the activation tile (TOK x 64) per k-block
 //   warp 1, one thread : tcgen05.mma (4 x K=16 per k-block), tcgen05.commit frees the stage
-//   warps 2..5         : one thread per weight row: packed codes from global memory -> exact
+//   warps 2..          : G groups of 4 warps, group g taking the k-blocks g, g+G, ...; in a group
+//                        one thread per weight row: packed codes from global memory -> exact
 //                        q - z by a magic-number subtract -> times the group scale -> 128 bytes
 //                        of the swizzled A tile; the row's CSR outliers are written over their
 //                        (exactly zero) dense entries, so the tensor cores also do the SpMM;
@@ -26,8 +27,9 @@ namespace {
 
 constexpr int kTileN = 128;      // weight rows per CTA (UMMA M)
 constexpr int kBlockK = 64;      // k-block: 128 bytes of 16-bit operands
-constexpr int kDequantWarps = 4;
-constexpr int kThreads = 32 * (2 + kDequantWarps);
+constexpr int kDequantWarps = 4;   // warps of one dequantisation group (one thread per tile row)
+__host__ __device__ constexpr int dq_groups(int tok) { return tok >= 128 ? 4 : 2; }
+__host__ __device__ constexpr int cta_threads(int tok) { return 32 * (2 + kDequantWarps * dq_groups(tok)); }
 constexpr int kMaxStages = 8;
 constexpr long long kSpinCycles = 1000LL * 1000LL * 1000LL;   // about half a second of SM clock
 
@@ -182,7 +184,7 @@ __device__ __forceinline__ unsigned sub_magic(unsigned qm, unsigned zm) {
 }
 
 template <int BITS, int TOK, bool BF16>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(cta_threads(TOK), 1)
 prefill_kernel(const __grid_constant__ CUtensorMap tmx, const PrefillArgs p, const int stages) {
   constexpr int kABytes = kTileN * kBlockK * 2;   // 16 KB
   constexpr int kBBytes = TOK * kBlockK * 2;
@@ -261,6 +263,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmx, const PrefillArgs p, con
     }
   } else {
     // ------------------------------------------------------------------ dequantization, then epilogue
+    constexpr int G = dq_groups(TOK);
+    const int gq = (warp - 2) >> 2;            // dequantisation group: k-blocks gq, gq + G, ...
     const int quad = warp & 3;                 // tensor-memory lane quarter this warp may access
     const int r = quad * 32 + lane;            // row inside the tile
     const int row = n0 + r;
@@ -279,13 +283,18 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmx, const PrefillArgs p, con
     unsigned nxt = j < je ? __ldg(p.cv + j) : 0xFFFFFFFFu;   // next outlier of the row
     constexpr unsigned MAGIC = BF16 ? 0x43004300u : 0x64006400u;   // 128.0 / 1024.0: ulp = 1
     unsigned wq[WPB];
+    unsigned short s_nx = 0;
+    unsigned char z_nx = 0;
+    if (gq < nkb) {
 #pragma unroll
-    for (int i = 0; i < WPB; ++i) wq[i] = __ldg(crow + i);
-    for (int kb = 0; kb < nkb && ok; ++kb) {
+      for (int i = 0; i < WPB; ++i) wq[i] = __ldg(crow + (size_t)gq * WPB + i);
+      s_nx = __ldg(srow + (gq * kBlockK) / p.group);
+      z_nx = __ldg(zrow + (gq * kBlockK) / p.group);
+    }
+    for (int kb = gq; kb < nkb && ok; kb += G) {
       const int s = kb % stages, round = kb / stages;
-      const int g = (kb * kBlockK) / p.group;
-      const float sc = live ? __half2float(__ushort_as_half(__ldg(srow + g))) : 0.f;
-      const unsigned z = __ldg(zrow + g);
+      const float sc = live ? __half2float(__ushort_as_half(s_nx)) : 0.f;
+      const unsigned z = z_nx;
       unsigned s_hi2, s_lo2 = 0;
       if (BF16) {
         const __nv_bfloat16 hi = __float2bfloat16_rn(sc);
@@ -299,9 +308,11 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmx, const PrefillArgs p, con
       unsigned cur[WPB];
 #pragma unroll
       for (int i = 0; i < WPB; ++i) cur[i] = wq[i];
-      if (kb + 1 < nkb) {
+      if (kb + G < nkb) {   // codes, scale and zero-point of this group's next k-block
 #pragma unroll
-        for (int i = 0; i < WPB; ++i) wq[i] = __ldg(crow + (size_t)(kb + 1) * WPB + i);
+        for (int i = 0; i < WPB; ++i) wq[i] = __ldg(crow + (size_t)(kb + G) * WPB + i);
+        s_nx = __ldg(srow + ((kb + G) * kBlockK) / p.group);
+        z_nx = __ldg(zrow + ((kb + G) * kBlockK) / p.group);
       }
       // 64 codes -> 32 pairs (columns 2h, 2h+1) -> 8 chunks of 16 bytes
       unsigned out[32];
@@ -336,11 +347,13 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmx, const PrefillArgs p, con
             make_uint4(out[4 * c], out[4 * c + 1], out[4 * c + 2], out[4 * c + 3]);
       // the row's outliers inside this k-block replace their dense entries (which are exactly 0)
       const unsigned k_end = (unsigned)(kb + 1) * kBlockK;
-      while (j < je && (nxt & 0xFFFFu) < k_end) {
-        const unsigned col = (nxt & 0xFFFFu) - (unsigned)kb * kBlockK;
-        unsigned short v16 = (unsigned short)(nxt >> 16);
-        if (BF16) v16 = __bfloat16_as_ushort(__float2bfloat16_rn(__half2float(__ushort_as_half(v16))));
-        *reinterpret_cast<unsigned short*>(arow + ((((col >> 3) ^ (r & 7)) << 4) | ((col & 7) << 1))) = v16;
+      while (j < je && (nxt & 0xFFFFu) < k_end) {   // entries of other groups' k-blocks are skipped
+        if ((nxt & 0xFFFFu) >= k_end - kBlockK) {
+          const unsigned col = (nxt & 0xFFFFu) - (unsigned)kb * kBlockK;
+          unsigned short v16 = (unsigned short)(nxt >> 16);
+          if (BF16) v16 = __bfloat16_as_ushort(__float2bfloat16_rn(__half2float(__ushort_as_half(v16))));
+          *reinterpret_cast<unsigned short*>(arow + ((((col >> 3) ^ (r & 7)) << 4) | ((col & 7) << 1))) = v16;
+        }
         ++j;
         nxt = j < je ? __ldg(p.cv + j) : 0xFFFFFFFFu;
       }
@@ -353,7 +366,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmx, const PrefillArgs p, con
     if (ok) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll 1
-      for (int c0 = 0; c0 < TOK; c0 += 32) {
+      for (int c0 = gq * (TOK / G); c0 < (gq + 1) * (TOK / G); c0 += 32) {   // each group drains its share
         if (m0 + c0 >= p.M) break;             // warp-uniform
         unsigned v[32];
         tmem_ld32(tmem_acc + ((unsigned)(quad * 32) << 16) + (unsigned)c0, v);
@@ -442,7 +455,7 @@ gwq_status launch(const gwq_packed* P, const void* x, const float* tok_scale, in
   a.codes = P->codes; a.scales = P->scales; a.zeros = P->zeros; a.row_ptr = P->S->row_ptr; a.cv = pv->cv;
   a.y = y; a.yd = yd; a.status = pv->dev_status; a.tok_scale = tok_scale; a.N = P->N; a.K = P->K; a.M = M; a.group = P->group;
   dim3 grid((unsigned)((P->N + kTileN - 1) / kTileN), (unsigned)((M + TOK - 1) / TOK));
-  prefill_kernel<BITS, TOK, BF16><<<grid, kThreads, smem, stream>>>(tmx, a, stages);
+  prefill_kernel<BITS, TOK, BF16><<<grid, cta_threads(TOK), smem, stream>>>(tmx, a, stages);
   return cudaGetLastError() == cudaSuccess ? GWQ_OK : GWQ_ERR_CUDA;
 }
 
