@@ -90,6 +90,7 @@ extern "C" void gwq_free(void* obj) {
       if (pv->x_stage) cudaFree(pv->x_stage);
       if (pv->y_stage) cudaFree(pv->y_stage);
       if (pv->x16) cudaFree(pv->x16);
+      if (pv->sz_t) cudaFree(pv->sz_t);
       if (pv->dev_status) cudaFree(pv->dev_status);
       delete pv;
     }

@@ -29,6 +29,7 @@ struct gwq_priv {
   void* y_stage;
   size_t x_stage_bytes;
   size_t y_stage_bytes;
+  uint32_t* sz_t;        // [K/group][N]: scale fp16 bits | zero-point << 16 (tensor-core path)
   void* x16;             // fp16 copy of bf16 activations for the tensor-core path (+ per-token scales)
   size_t x16_bytes;
   int32_t* dev_status;   // device status word written by bounded waits

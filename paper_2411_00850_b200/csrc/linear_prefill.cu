@@ -108,6 +108,7 @@ struct PrefillArgs {
   const uint16_t* scales;
   const uint8_t* zeros;
   const int32_t* row_ptr;
+  const uint32_t* sz_t; // [K/group][N]: scale fp16 bits | zero-point << 16
   const uint32_t* cv;   // per outlier: fp16 value << 16 | column
   void* y;
   gwq_dtype yd;
@@ -157,6 +158,21 @@ __global__ void __launch_bounds__(256) bf16_rows_to_scaled_f16(const uint16_t* _
   }
 }
 
+
+// Packed words of one row for one k-block (8 words for 4 bits, 6 for 3 bits) with the widest loads
+// the alignment allows: a thread reads its own row, so every load instruction of a warp touches 32
+// different lines, and the number of load instructions is what the load pipe pays for.
+template <int WPB>
+__device__ __forceinline__ void load_words(const uint32_t* __restrict__ p, unsigned (&w)[WPB]) {
+  if (WPB == 8) {
+    const uint4 a = __ldg(reinterpret_cast<const uint4*>(p)), b = __ldg(reinterpret_cast<const uint4*>(p) + 1);
+    w[0] = a.x; w[1] = a.y; w[2] = a.z; w[3] = a.w; w[4 % WPB] = b.x; w[5 % WPB] = b.y; w[6 % WPB] = b.z; w[7 % WPB] = b.w;
+  } else {   // 24 bytes, 8-byte aligned
+    const uint2 a = __ldg(reinterpret_cast<const uint2*>(p)), b = __ldg(reinterpret_cast<const uint2*>(p) + 1),
+                c = __ldg(reinterpret_cast<const uint2*>(p) + 2);
+    w[0] = a.x; w[1] = a.y; w[2] = b.x; w[3] = b.y; w[4] = c.x; w[5] = c.y;
+  }
+}
 
 template <bool BF16>
 __device__ __forceinline__ unsigned mul_scale(unsigned d, unsigned s_hi2, unsigned s_lo2) {
@@ -270,31 +286,30 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmx, const PrefillArgs p, con
     const int row = n0 + r;
     const bool live = row < p.N;
     const int rowc = live ? row : p.N - 1;
-    const int ngroups = p.K / p.group;
     constexpr int WPB = kBlockK * BITS / 32;   // packed words per row per k-block (8 or 6)
     const uint32_t* crow = p.codes + (size_t)rowc * (p.K / 32) * BITS;
-    const uint16_t* srow = p.scales + (size_t)rowc * ngroups;
-    const uint8_t* zrow = p.zeros + (size_t)rowc * ngroups;
+    const uint32_t* szcol = p.sz_t + rowc;   // [group][row] table: neighbouring rows are neighbouring words
     int j = 0, je = 0;
     if (live) {
       j = p.row_ptr[row];
       je = p.row_ptr[row + 1];
     }
-    unsigned nxt = j < je ? __ldg(p.cv + j) : 0xFFFFFFFFu;   // next outlier of the row
+    // the row's next outliers, kept kOutWin entries ahead so that walking the list never waits on memory
+    constexpr int kOutWin = 8;
+    unsigned win[kOutWin];
+#pragma unroll
+    for (int i = 0; i < kOutWin; ++i) win[i] = j + i < je ? __ldg(p.cv + j + i) : 0xFFFFFFFFu;
     constexpr unsigned MAGIC = BF16 ? 0x43004300u : 0x64006400u;   // 128.0 / 1024.0: ulp = 1
     unsigned wq[WPB];
-    unsigned short s_nx = 0;
-    unsigned char z_nx = 0;
+    unsigned sz_nx = 0;   // scale (fp16 bits) | zero-point << 16 of the group of the next k-block
     if (gq < nkb) {
-#pragma unroll
-      for (int i = 0; i < WPB; ++i) wq[i] = __ldg(crow + (size_t)gq * WPB + i);
-      s_nx = __ldg(srow + (gq * kBlockK) / p.group);
-      z_nx = __ldg(zrow + (gq * kBlockK) / p.group);
+      load_words<WPB>(crow + (size_t)gq * WPB, wq);
+      sz_nx = __ldg(szcol + (size_t)((gq * kBlockK) / p.group) * p.N);
     }
     for (int kb = gq; kb < nkb && ok; kb += G) {
       const int s = kb % stages, round = kb / stages;
-      const float sc = live ? __half2float(__ushort_as_half(s_nx)) : 0.f;
-      const unsigned z = z_nx;
+      const float sc = live ? __half2float(__ushort_as_half((unsigned short)(sz_nx & 0xFFFFu))) : 0.f;
+      const unsigned z = sz_nx >> 16;
       unsigned s_hi2, s_lo2 = 0;
       if (BF16) {
         const __nv_bfloat16 hi = __float2bfloat16_rn(sc);
@@ -309,10 +324,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmx, const PrefillArgs p, con
 #pragma unroll
       for (int i = 0; i < WPB; ++i) cur[i] = wq[i];
       if (kb + G < nkb) {   // codes, scale and zero-point of this group's next k-block
-#pragma unroll
-        for (int i = 0; i < WPB; ++i) wq[i] = __ldg(crow + (size_t)(kb + G) * WPB + i);
-        s_nx = __ldg(srow + ((kb + G) * kBlockK) / p.group);
-        z_nx = __ldg(zrow + ((kb + G) * kBlockK) / p.group);
+        load_words<WPB>(crow + (size_t)(kb + G) * WPB, wq);
+        sz_nx = __ldg(szcol + (size_t)(((kb + G) * kBlockK) / p.group) * p.N);
       }
       // 64 codes -> 32 pairs (columns 2h, 2h+1) -> 8 chunks of 16 bytes
       unsigned out[32];
@@ -347,15 +360,18 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmx, const PrefillArgs p, con
             make_uint4(out[4 * c], out[4 * c + 1], out[4 * c + 2], out[4 * c + 3]);
       // the row's outliers inside this k-block replace their dense entries (which are exactly 0)
       const unsigned k_end = (unsigned)(kb + 1) * kBlockK;
-      while (j < je && (nxt & 0xFFFFu) < k_end) {   // entries of other groups' k-blocks are skipped
-        if ((nxt & 0xFFFFu) >= k_end - kBlockK) {
-          const unsigned col = (nxt & 0xFFFFu) - (unsigned)kb * kBlockK;
-          unsigned short v16 = (unsigned short)(nxt >> 16);
+      while (j < je && (win[0] & 0xFFFFu) < k_end) {   // entries of other groups' k-blocks are skipped
+        const unsigned e = win[0];
+        if ((e & 0xFFFFu) >= k_end - kBlockK) {
+          const unsigned col = (e & 0xFFFFu) - (unsigned)kb * kBlockK;
+          unsigned short v16 = (unsigned short)(e >> 16);
           if (BF16) v16 = __bfloat16_as_ushort(__float2bfloat16_rn(__half2float(__ushort_as_half(v16))));
           *reinterpret_cast<unsigned short*>(arow + ((((col >> 3) ^ (r & 7)) << 4) | ((col & 7) << 1))) = v16;
         }
         ++j;
-        nxt = j < je ? __ldg(p.cv + j) : 0xFFFFFFFFu;
+#pragma unroll
+        for (int i = 0; i + 1 < kOutWin; ++i) win[i] = win[i + 1];
+        win[kOutWin - 1] = j + kOutWin - 1 < je ? __ldg(p.cv + j + kOutWin - 1) : 0xFFFFFFFFu;
       }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to the MMA
       __syncwarp();
@@ -452,7 +468,7 @@ gwq_status launch(const gwq_packed* P, const void* x, const float* tok_scale, in
                            (int)smem) != cudaSuccess)
     return GWQ_ERR_CUDA;
   PrefillArgs a;
-  a.codes = P->codes; a.scales = P->scales; a.zeros = P->zeros; a.row_ptr = P->S->row_ptr; a.cv = pv->cv;
+  a.codes = P->codes; a.scales = P->scales; a.zeros = P->zeros; a.row_ptr = P->S->row_ptr; a.cv = pv->cv; a.sz_t = pv->sz_t;
   a.y = y; a.yd = yd; a.status = pv->dev_status; a.tok_scale = tok_scale; a.N = P->N; a.K = P->K; a.M = M; a.group = P->group;
   dim3 grid((unsigned)((P->N + kTileN - 1) / kTileN), (unsigned)((M + TOK - 1) / TOK));
   prefill_kernel<BITS, TOK, BF16><<<grid, cta_threads(TOK), smem, stream>>>(tmx, a, stages);
@@ -475,7 +491,7 @@ gwq_status launch_tok(const gwq_packed* P, const void* x, const float* tok_scale
 gwq_status gwq_launch_prefill(const gwq_packed* P, const void* x, gwq_dtype xd, int M, void* y, gwq_dtype yd,
                               cudaStream_t stream) {
   gwq_priv* pv = static_cast<gwq_priv*>(P->priv);
-  if (!pv->cv || P->K % kBlockK != 0) return gwq_launch_simt(P, x, xd, M, y, yd, stream);
+  if (!pv->cv || !pv->sz_t || P->K % kBlockK != 0) return gwq_launch_simt(P, x, xd, M, y, yd, stream);
   const float* tok_scale = nullptr;
   if (xd == GWQ_BF16) {
     const size_t need = (size_t)M * P->K * 2 + (size_t)M * 4 + 256;

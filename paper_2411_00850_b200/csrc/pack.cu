@@ -124,6 +124,17 @@ __global__ void fuse_col_val_kernel(const int32_t* __restrict__ col, const uint1
   if (i < n) cv[i] = ((uint32_t)val[i] << 16) | ((uint32_t)col[i] & 0xFFFFu);
 }
 
+// Tensor-core-side copy of the group tables, transposed to [group][row] so that the 128 rows of a
+// tile read 128 neighbouring words.
+__global__ void transpose_scale_zero_kernel(const uint16_t* __restrict__ scales, const uint8_t* __restrict__ zeros,
+                                            uint32_t* __restrict__ sz_t, int N, int ngroups) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;   // output index g * N + n
+  if (i < (long long)N * ngroups) {
+    const int g = (int)(i / N), n = (int)(i - (long long)g * N);
+    sz_t[i] = (uint32_t)scales[(size_t)n * ngroups + g] | ((uint32_t)zeros[(size_t)n * ngroups + g] << 16);
+  }
+}
+
 }  // namespace
 
 extern "C" gwq_status gwq_pack(const uint16_t* W, gwq_outliers* S, int32_t N, int32_t K, int32_t bits,
@@ -179,6 +190,10 @@ extern "C" gwq_status gwq_pack(const uint16_t* W, gwq_outliers* S, int32_t N, in
       GWQ_CUDA_TRY(cudaGetLastError());
     }
   }
+  GWQ_CUDA_TRY(cudaMalloc(&pv->sz_t, ngroups * sizeof(uint32_t) + 16));
+  transpose_scale_zero_kernel<<<(unsigned)((ngroups + 255) / 256), 256, 0, stream>>>(P->scales, P->zeros, pv->sz_t, N,
+                                                                                     K / group);
+  GWQ_CUDA_TRY(cudaGetLastError());
   GWQ_CUDA_TRY(cudaMemcpyAsync(&host_status, pv->dev_status, sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
   GWQ_CUDA_TRY(cudaStreamSynchronize(stream));
   if (host_status != 0) {
@@ -194,6 +209,7 @@ fail:
   if (P->scales) cudaFree(P->scales);
   if (P->zeros) cudaFree(P->zeros);
   if (pv->cv) cudaFree(pv->cv);
+  if (pv->sz_t) cudaFree(pv->sz_t);
   if (pv->dev_status) cudaFree(pv->dev_status);
   delete pv;
   delete P;
