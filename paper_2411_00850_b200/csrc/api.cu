@@ -2,6 +2,10 @@
 // the host-buffer variant, object release and status names.
 #include "common.cuh"
 
+#ifndef GWQ_DECODE_MAX_M
+#define GWQ_DECODE_MAX_M 32   // up to here the streaming mma.sync kernel; above, the tcgen05 kernel
+#endif
+
 static size_t dtype_bytes(gwq_dtype d) { return d == GWQ_F32 ? 4 : 2; }
 
 extern "C" gwq_status gwq_linear(const gwq_packed* P, const void* x, gwq_dtype xd, int32_t M, void* y,
@@ -11,7 +15,7 @@ extern "C" gwq_status gwq_linear(const gwq_packed* P, const void* x, gwq_dtype x
   if (yd != GWQ_F16 && yd != GWQ_BF16 && yd != GWQ_F32) return GWQ_ERR_INVALID_ARG;
   if (!gwq_aligned16(x) || !gwq_aligned16(y)) return GWQ_ERR_INVALID_ARG;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-  if (M <= 32) return gwq_launch_decode(P, x, xd, M, y, yd, stream);
+  if (M <= GWQ_DECODE_MAX_M) return gwq_launch_decode(P, x, xd, M, y, yd, stream);
   return gwq_launch_prefill(P, x, xd, M, y, yd, stream);
 }
 
@@ -90,6 +94,7 @@ extern "C" void gwq_free(void* obj) {
       if (pv->x_stage) cudaFree(pv->x_stage);
       if (pv->y_stage) cudaFree(pv->y_stage);
       if (pv->x16) cudaFree(pv->x16);
+      if (pv->xt) cudaFree(pv->xt);
       if (pv->sz_t) cudaFree(pv->sz_t);
       if (pv->dev_status) cudaFree(pv->dev_status);
       delete pv;

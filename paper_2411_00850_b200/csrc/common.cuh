@@ -32,6 +32,8 @@ struct gwq_priv {
   uint32_t* sz_t;        // [K/group][N]: scale fp16 bits | zero-point << 16 (tensor-core path)
   void* x16;             // fp16 copy of bf16 activations for the tensor-core path (+ per-token scales)
   size_t x16_bytes;
+  void* xt;              // token-major copy [K][tokens] of the activations (decode path, outlier gathers)
+  size_t xt_bytes;
   int32_t* dev_status;   // device status word written by bounded waits
   int sm_count;
 };

@@ -14,12 +14,14 @@
 //    subtract per pair), no second MMA.
 // The pair-interleaved packed order makes both operands natural: pair h of a lane's run
 // holds columns (2h, 2h+1), the same pair as 32-bit word h of its activation segment.
-// Activations are staged once per CTA in shared memory (XOR-swizzled 16-byte chunks)
-// when they fit, else read through L1.  After the K loop the warps' partial sums meet in
-// shared memory, the CSR outliers of a row are added by the warp that owns it, and y is
-// stored.  The kernel is launched with programmatic stream serialization: its weight
+// Activations are staged in shared memory chunk by chunk (8 groups, double buffered, padded
+// against bank conflicts); the CSR outliers of a row are added, chunk by chunk and from the
+// same staged activations, by the warp that owns the row.  After the K loop the warps'
+// partial sums meet in shared memory and y is stored.  The kernel is launched with programmatic stream serialization: its weight
 // prefetch may overlap the previous kernel, everything that touches x or y comes after
 // griddepcontrol.wait.
+#include <type_traits>
+
 #include "common.cuh"
 
 namespace {
@@ -186,6 +188,25 @@ __device__ __forceinline__ void load_run(const uint32_t* __restrict__ base, unsi
   }
 }
 
+// Same load, executed only where `pred` holds (predicated instructions, no branch).
+template <int BITS>
+__device__ __forceinline__ void load_run_if(const uint32_t* __restrict__ base, unsigned off, unsigned (&w)[BITS],
+                                            bool pred) {
+  const uint32_t* p = base + off;
+  if (BITS == 4) {
+    asm volatile(
+        "{\n .reg .pred q;\n setp.ne.b32 q, %5, 0;\n @q ld.global.cs.v4.u32 {%0,%1,%2,%3}, [%4];\n}\n"
+        : "+r"(w[0]), "+r"(w[1]), "+r"(w[2]), "+r"(w[BITS - 1])
+        : "l"(p), "r"((int)pred));
+  } else {
+    asm volatile(
+        "{\n .reg .pred q;\n setp.ne.b32 q, %4, 0;\n @q ld.global.cs.u32 %0, [%3];\n @q ld.global.cs.u32 %1, [%3+4];\n"
+        " @q ld.global.cs.u32 %2, [%3+8];\n}\n"
+        : "+r"(w[0]), "+r"(w[1]), "+r"(w[2])
+        : "l"(p), "r"((int)pred));
+  }
+}
+
 __device__ __forceinline__ void store_y(void* y, gwq_dtype yd, long long idx, float v) {
   if (yd == GWQ_F32) reinterpret_cast<float*>(y)[idx] = v;
   else if (yd == GWQ_F16) reinterpret_cast<__half*>(y)[idx] = __float2half_rn(v);
@@ -205,6 +226,7 @@ struct DecodeArgs {
   const int32_t* row_ptr;
   const uint32_t* cv;  // per outlier: fp16 value << 16 | column
   const uint16_t* x;
+  const uint16_t* xt;  // [K][TP] copy of x (ring mode with more than one token), else null
   void* y;
   gwq_dtype yd;
   int N, K, M;
@@ -213,19 +235,31 @@ struct DecodeArgs {
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
-// Sum TP per-lane values over the 32 lanes with TP - 1 + log2(32 / TP) shuffles: every
-// stage halves the values a lane keeps.  Afterwards lane L holds the total of value
-// L / (32 / TP) in v[0].
-template <int TP>
-__device__ __forceinline__ void reduce_across_lanes(float (&v)[TP], int lane) {
-  int n = TP;
+// ---------------------------------------------------------------------------------------------
+// Activations are staged chunk by chunk: one chunk is 8 groups (1024 columns), one group per warp,
+// double buffered, so shared memory stays small for every M and K and the B fragments never come
+// from global memory.  16-byte piece c of token row m sits at piece c + (c >> 3) + 2 (m & 1) of its
+// row (one pad piece per 128 bytes, odd rows shifted by two): the 64-byte segments of the four lanes
+// of a quad and of two neighbouring token rows then fall into all eight 16-byte bank groups.
+constexpr int kOutSlots = 3;                          // outlier entries per lane kept in registers
+constexpr int kChunkGroups = kWarps;                 // groups per chunk
+constexpr int kChunkPieces = kChunkGroups * 16;      // 16-byte pieces per token row per chunk
+constexpr int kRowPitch = kChunkPieces + kChunkPieces / 8 + 4;   // pieces, with padding
+__device__ __forceinline__ int xs_piece(int c, int m) { return m * kRowPitch + c + (c >> 3) + ((m & 1) << 1); }
+
+// Sum, over the lanes that hold the same token group, VT per-lane values: TS token groups are
+// interleaved over the lanes (group = lane % TS).  Afterwards lane L holds, in v[0], the total of
+// token (L % TS) * VT + value index, the value index being L / (32 / VT) for VT < 8 ... see below.
+template <int VT, int TS>
+__device__ __forceinline__ void reduce_tokens(float (&v)[VT], int lane) {
+  int n = VT;
 #pragma unroll
-  for (int o = 16; o >= 1; o >>= 1) {
+  for (int o = 16; o >= TS; o >>= 1) {
     if (n > 1) {
       const int half = n >> 1;
       const bool up = (lane & o) != 0;
 #pragma unroll
-      for (int i = 0; i < (TP > 1 ? TP / 2 : 1); ++i) {
+      for (int i = 0; i < (VT > 1 ? VT / 2 : 1); ++i) {
         if (i < half) {
           const float send = up ? v[i] : v[i + half];
           const float keep = up ? v[i + half] : v[i];
@@ -239,38 +273,32 @@ __device__ __forceinline__ void reduce_across_lanes(float (&v)[TP], int lane) {
   }
 }
 
-
-constexpr int kOutSlots = 3;  // outlier entries per lane held in registers (96 per row); the rest is looped
-
-// Staged activations: 16-byte chunk c of token row m lives at chunk c + (c >> 3) + 2 (m & 1) of
-// its row (one pad chunk per 128 bytes, odd rows shifted by two chunks), so that the 64-byte
-// segments of the four lanes of a quad and of two neighbouring token rows fall into all eight
-// 16-byte bank groups.  Row pitch in chunks:
-__host__ __device__ inline int xs_pitch_chunks(int K) { return (K >> 3) + (K >> 6) + 4; }
-__device__ __forceinline__ int xs_chunk(int c, int m, int pitch) { return m * pitch + c + (c >> 3) + ((m & 1) << 1); }
-
 template <int BITS, int NB, bool BF16>
 struct StepAcc;
 template <int NB> struct StepAcc<4, NB, false> { using type = AccRaw4<NB>; };
 template <int NB> struct StepAcc<3, NB, false> { using type = AccRaw3<NB>; };
 template <int BITS, int NB> struct StepAcc<BITS, NB, true> { using type = AccSub<NB>; };
 
-// TP = tokens rounded up to 1, 4, 8, 16 or 32.  XS: activations staged in shared memory.  Group size 128.
-template <int BITS, int TP, bool BF16, bool XS>
+// TP = tokens rounded up to 1, 4, 8, 16 or 32.  Group size 128.
+// NBUF = 0: the activations of all chunks are staged up front by the whole CTA (small M K).
+// NBUF = 2: every warp keeps a private double buffer with the activations of its own group only
+//           (M x 128 columns), copied one step ahead with cp.async; no CTA barrier in the K loop.
+constexpr int kTilePitch = 16 + 2 + 2;   // pieces per token row of a warp tile (same padding rule)
+template <int BITS, int TP, bool BF16, int NBUF>
 __global__ void __launch_bounds__(kThreads, TP <= 8 ? 3 : (TP == 16 ? 2 : 1)) decode_kernel(const DecodeArgs p) {
-  constexpr int NB = TP <= 8 ? 1 : TP / 8;  // 8-token blocks
-  constexpr int WPR = BITS;                  // words per run of 32 columns
+  constexpr int NB = TP <= 8 ? 1 : TP / 8;   // 8-token blocks of the MMA
+  constexpr int WPR = BITS;                   // words per run of 32 columns
+  constexpr bool ONES = !BF16 && TP != 1;     // raw path: sum_k x_k by MMA unless there is one token
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int ngroups = p.K >> 7;
-  constexpr bool ONES = !BF16 && !(TP == 1 && XS);  // raw path: sum_k x_k by MMA unless one staged token
   // shared: zero page 64 B | scales [16][ngroups] f16 | zeros [16][ngroups] u8 | red [kWarps][NB][16][8] f32 |
-  //         outl [16][TP] f32 | x (XS)
+  //         outl [16][TP] f32 | x chunk buffers 2 x [M][kRowPitch] pieces
   uint16_t* sm_s = reinterpret_cast<uint16_t*>(smem_raw + 64);
   uint8_t* sm_z = reinterpret_cast<uint8_t*>(sm_s + kRows * ngroups);
   float* sm_red = reinterpret_cast<float*>(sm_z + kRows * ngroups);
   float* sm_out = sm_red + kWarps * NB * 128;
   uint4* sm_x = reinterpret_cast<uint4*>(sm_out + kRows * TP);
-  const int pitch = xs_pitch_chunks(p.K);
+  const int buf_pieces = p.M * kRowPitch;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int gid = lane >> 2, t = lane & 3;
@@ -280,7 +308,8 @@ __global__ void __launch_bounds__(kThreads, TP <= 8 ? 3 : (TP == 16 ? 2 : 1)) de
   constexpr unsigned kStepWords = kWarps * 4 * WPR;  // codes of 8 groups
   unsigned oa = (unsigned)ra * row_words + (unsigned)(warp * 4 + t) * WPR;  // group `warp`, this lane's run
   unsigned ob = (unsigned)rb * row_words + (unsigned)(warp * 4 + t) * WPR;
-  const int nsteps = (ngroups - warp + kWarps - 1) / kWarps;  // groups warp, warp+8, ...
+  const int nsteps = (ngroups - warp + kWarps - 1) / kWarps;  // this warp's groups: warp, warp + 8, ...
+  const int nchunks = (ngroups + kChunkGroups - 1) / kChunkGroups;
 
   pdl_launch_dependents();
 
@@ -294,7 +323,7 @@ __global__ void __launch_bounds__(kThreads, TP <= 8 ? 3 : (TP == 16 ? 2 : 1)) de
     const char* gs = reinterpret_cast<const char*>(p.scales + (size_t)r0 * ngroups);
     const char* gz = reinterpret_cast<const char*>(p.zeros + (size_t)r0 * ngroups);
     if (rows_here == kRows) {
-      for (int c = tid; c < 3 * ngroups; c += kThreads) {   // 32 ng + 16 ng bytes = 3 ng chunks
+      for (int c = tid; c < 3 * ngroups; c += kThreads) {   // 32 ng + 16 ng bytes = 3 ng pieces
         const bool is_s = c < 2 * ngroups;
         const char* src = is_s ? gs + c * 16 : gz + (c - 2 * ngroups) * 16;
         const unsigned dst = (unsigned)__cvta_generic_to_shared(reinterpret_cast<char*>(sm_s) + c * 16);
@@ -320,50 +349,113 @@ __global__ void __launch_bounds__(kThreads, TP <= 8 ? 3 : (TP == 16 ? 2 : 1)) de
 
   // ---- from here on x is read
   pdl_wait();
-  if (XS) {
-    const int chunks_per_row = p.K >> 3;
-    for (int m = 0; m < p.M; ++m) {
-      for (int c = tid; c < chunks_per_row; c += kThreads) {
-        const unsigned dst = (unsigned)__cvta_generic_to_shared(sm_x + xs_chunk(c, m, pitch));
-        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(p.x + (size_t)m * p.K + c * 8));
+  // NBUF == 0: copy of chunk c of the activations into its buffer, by the whole CTA
+  auto stage_chunk = [&](int c) {
+    const int col0 = c * kChunkGroups * 128;
+    const int pieces = min(kChunkPieces, (p.K - col0) >> 3);
+    uint4* buf = sm_x + c * buf_pieces;
+    for (int i = tid; i < p.M * kChunkPieces; i += kThreads) {
+      const int m = i / kChunkPieces, pc = i - m * kChunkPieces;   // kChunkPieces is a power of two
+      if (pc < pieces) {
+        const unsigned dst = (unsigned)__cvta_generic_to_shared(buf + xs_piece(pc, m));
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(p.x + (size_t)m * p.K + col0 + pc * 8));
       }
     }
+  };
+  // NBUF == 2: copy of the activations of this warp's step c (group warp + 8 c) into its buffer c & 1
+  const int tile_pieces = p.M * kTilePitch;
+  uint4* wtile = sm_x + warp * 2 * tile_pieces;
+  auto stage_tile = [&](int c) {
+    if (c < nsteps) {
+      const uint16_t* src = p.x + (size_t)(warp + kWarps * c) * 128;
+      uint4* buf = wtile + (c & 1) * tile_pieces;
+      for (int i = lane; i < p.M * 16; i += 32) {
+        const int m = i >> 4, pc = i & 15;
+        const unsigned dst = (unsigned)__cvta_generic_to_shared(buf + m * kTilePitch + pc + (pc >> 3) + ((m & 1) << 1));
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src + (size_t)m * p.K + pc * 8));
+      }
+    }
+  };
+  if (NBUF == 0) {
+    for (int c = 0; c < nchunks; ++c) stage_chunk(c);
+  } else {
+    stage_tile(0);
   }
-  // outlier payload of the two owned rows (needs the row extents: the one load awaited here)
+  asm volatile("cp.async.commit_group;" ::: "memory");   // also carries the scale / zero-point tables
+
+  // outlier payload of the two owned rows.  With everything staged (NBUF == 0) entry lane + 32 e of a
+  // row is loaded into cv[row][e] now (up to 96 per row; all ones = no entry) and meets the staged
+  // activations after the loop; in ring mode the entries are read after the loop.
   const int j0 = __shfl_sync(0xFFFFFFFFu, rp, 0), j1 = __shfl_sync(0xFFFFFFFFu, rp, 1),
             j2 = __shfl_sync(0xFFFFFFFFu, rp, 2);
   unsigned cv[2][kOutSlots];
+  if (NBUF == 0) {
 #pragma unroll
-  for (int e = 0; e < kOutSlots; ++e) {
-    const int ja = j0 + lane + 32 * e, jb = j1 + lane + 32 * e;
-    cv[0][e] = ja < j1 ? __ldcs(p.cv + ja) : 0u;  // value 0 contributes nothing
-    cv[1][e] = jb < j2 ? __ldcs(p.cv + jb) : 0u;
+    for (int e = 0; e < kOutSlots; ++e) {
+      const int ja = j0 + lane + 32 * e, jb = j1 + lane + 32 * e;
+      cv[0][e] = ja < j1 ? __ldcs(p.cv + ja) : 0xFFFFFFFFu;
+      cv[1][e] = jb < j2 ? __ldcs(p.cv + jb) : 0xFFFFFFFFu;
+    }
   }
-  asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;" ::: "memory");
+
+  if (NBUF != 0) {
+    // ring mode: the outliers are done now, while the first codes are still on their way.  The
+    // activations come from the token-major copy xt[K][TP] (one short contiguous read per entry):
+    // lane = (entry, group of VT tokens), two batches of entries in flight.
+    constexpr int VT = TP < 8 ? TP : 8, TS = TP / VT, EPB = 32 / TS;
+    const uint16_t* xt = TP == 1 ? p.x : p.xt;
+    const int part = lane % TS;
+#pragma unroll
+    for (int rr = 0; rr < 2; ++rr) {
+      const int jb = rr == 0 ? j0 : j1, je = rr == 0 ? j1 : j2;
+      float v[VT];
+#pragma unroll
+      for (int i = 0; i < VT; ++i) v[i] = 0.f;
+      for (int jj = jb; jj < je; jj += 2 * EPB) {
+        unsigned e[2];
+        uint4 xq[2];
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+          const int j = jj + u * EPB + lane / TS;
+          e[u] = j < je ? __ldg(p.cv + j) : 0u;   // value 0, column 0
+        }
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+          const uint16_t* src = xt + (size_t)(e[u] & 0xFFFFu) * TP + part * VT;
+          if (VT == 8) xq[u] = __ldg(reinterpret_cast<const uint4*>(src));
+          else if (VT == 4) { const uint2 q = __ldg(reinterpret_cast<const uint2*>(src)); xq[u] = make_uint4(q.x, q.y, 0, 0); }
+          else xq[u] = make_uint4(__ldg(src), 0, 0, 0);
+        }
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+          const float wv = __half2float(__ushort_as_half((unsigned short)(e[u] >> 16)));
+          const unsigned w4[4] = {xq[u].x, xq[u].y, xq[u].z, xq[u].w};
+#pragma unroll
+          for (int i = 0; i < VT; ++i)
+            v[i] = fmaf(wv, act_to_float<BF16>((uint16_t)(w4[i >> 1] >> (16 * (i & 1)))), v[i]);
+        }
+      }
+      reduce_tokens<VT, TS>(v, lane);
+      constexpr int LPV = 32 / VT;   // lanes per value after the halving stages
+      const int tok = part * VT + lane / LPV;
+      if ((lane % LPV) / TS == 0) sm_out[(2 * warp + rr) * TP + tok] = v[0];
+    }
+  }
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
   __syncthreads();
 
-  // this lane's activation segment (64 bytes per group) for token gid of every token block;
-  // lanes without a token read the zero page and never advance
-  const uint4* xp[NB];
-  int xstep[NB];
+  // lane constants inside a chunk buffer: this lane's 64-byte segment of group `warp` for token gid
+  // of every token block (lanes without a token read the zero page), the scale tables, the x sums
+  int xoff[NB];
 #pragma unroll
   for (int nb = 0; nb < NB; ++nb) {
     const int m = nb * 8 + gid;
-    if (XS) {
-      const bool live = m < p.M;
-      xp[nb] = live ? sm_x + xs_chunk(warp * 16 + t * 4, m, pitch) : reinterpret_cast<const uint4*>(smem_raw);
-      xstep[nb] = live ? kWarps * 18 : 0;  // 8 groups ahead: 8 * (16 + 2 pad) chunks
-    } else {
-      const int mm = min(m, p.M - 1);
-      xp[nb] = reinterpret_cast<const uint4*>(p.x + (size_t)mm * p.K) + warp * 16 + t * 4;
-      xstep[nb] = kWarps * 16;
-    }
+    xoff[nb] = m >= p.M ? -1 : (NBUF == 0 ? xs_piece(warp * 16 + t * 4, m) : m * kTilePitch + 4 * t + (t >> 1) + ((m & 1) << 1));
   }
   const uint16_t* sp = sm_s + gid * ngroups + warp;   // scale / zero-point of row gid, group `warp`
   const uint8_t* zp = sm_z + gid * ngroups + warp;
   const int hi_row = 8 * ngroups;
-  // single staged token: its group sums come from shared memory, lane L adding columns 4L..4L+3
-  const uint2* xsum_p = reinterpret_cast<const uint2*>(sm_x + xs_chunk(warp * 16 + (lane >> 1), 0, pitch)) + (lane & 1);
+  const int xsum_off = (NBUF == 0 ? xs_piece(warp * 16 + (lane >> 1), 0) : (lane >> 1) + (lane >> 4)) * 2 + (lane & 1);   // 8-byte units, token 0
 
   float yacc[NB][4];
 #pragma unroll
@@ -371,87 +463,104 @@ __global__ void __launch_bounds__(kThreads, TP <= 8 ? 3 : (TP == 16 ? 2 : 1)) de
 #pragma unroll
     for (int i = 0; i < 4; ++i) yacc[nb][i] = 0.f;
 
-  for (int s0 = 0; s0 < nsteps; s0 += kDepth) {
+  // one chunk: stage the next one, this warp's group step (register slot D = c % kDepth), the owned
+  // rows' outliers of the chunk, then the hand-over barrier
+  auto do_chunk = [&](const int c, auto slot) {
+    constexpr int d = decltype(slot)::value;
+    if (NBUF != 0) {   // next step's activations on their way, this step's landed and visible to the warp
+      __syncwarp();
+      stage_tile(c + 1);
+      asm volatile("cp.async.commit_group;\ncp.async.wait_group 1;" ::: "memory");
+      __syncwarp();
+    }
+    const uint4* buf = NBUF == 0 ? sm_x + c * buf_pieces : wtile + (c & 1) * tile_pieces;
+    if (c < nsteps) {
+      unsigned xr[NB][16];
 #pragma unroll
-    for (int d = 0; d < kDepth; ++d) {
-      if (s0 + d < nsteps) {
-        unsigned xr[NB][16];
+      for (int nb = 0; nb < NB; ++nb) {
+        const uint4* seg = xoff[nb] >= 0 ? buf + xoff[nb] : reinterpret_cast<const uint4*>(smem_raw);
 #pragma unroll
-        for (int nb = 0; nb < NB; ++nb) {
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            uint4 v = XS ? xp[nb][i] : __ldg(xp[nb] + i);
-            if (!XS && nb * 8 + gid >= p.M) v = make_uint4(0, 0, 0, 0);  // token rows past M contribute nothing
-            xr[nb][4 * i] = v.x; xr[nb][4 * i + 1] = v.y; xr[nb][4 * i + 2] = v.z; xr[nb][4 * i + 3] = v.w;
-          }
-          xp[nb] += xstep[nb];
+        for (int i = 0; i < 4; ++i) {
+          const uint4 v = seg[i];
+          xr[nb][4 * i] = v.x; xr[nb][4 * i + 1] = v.y; xr[nb][4 * i + 2] = v.z; xr[nb][4 * i + 3] = v.w;
         }
-        // (s 2^24, s z) on the raw path, (s, magic | z) on the subtract path
-        float2 ta, tb;
-        {
-          const float sa = __half2float(__ushort_as_half(sp[0])), sb = __half2float(__ushort_as_half(sp[hi_row]));
-          const unsigned za = zp[0], zb = zp[hi_row];
-          sp += kWarps;
-          zp += kWarps;
-          if (BF16) {
-            ta = make_float2(sa, __uint_as_float(0x43004300u | (za * 0x00010001u)));
-            tb = make_float2(sb, __uint_as_float(0x43004300u | (zb * 0x00010001u)));
-          } else {
-            ta = make_float2(sa * 16777216.f, sa * (float)za);
-            tb = make_float2(sb * 16777216.f, sb * (float)zb);
-          }
-        }
-        float xsum1 = 0.f;
-        if (!BF16 && !ONES) {
-          const uint2 h4 = *xsum_p;
-          xsum_p += kWarps * 18 * 2;
-          const float2 f0 = __half22float2(*reinterpret_cast<const __half2*>(&h4.x));
-          const float2 f1 = __half22float2(*reinterpret_cast<const __half2*>(&h4.y));
-          xsum1 = (f0.x + f0.y) + (f1.x + f1.y);
-#pragma unroll
-          for (int o = 16; o > 0; o >>= 1) xsum1 += __shfl_xor_sync(0xFFFFFFFFu, xsum1, o);
-        }
-        typename StepAcc<BITS, NB, BF16>::type acc = {};
+      }
+      // (s 2^24, s z) on the raw path, (s, magic | z) on the subtract path
+      float2 ta, tb;
+      {
+        const float sa = __half2float(__ushort_as_half(sp[0])), sb = __half2float(__ushort_as_half(sp[hi_row]));
+        const unsigned za = zp[0], zb = zp[hi_row];
+        sp += kWarps;
+        zp += kWarps;
         if (BF16) {
-          step_sub<BITS, NB>(wa[d], wb[d], __float_as_uint(ta.y), __float_as_uint(tb.y), xr,
-                             reinterpret_cast<AccSub<NB>&>(acc));
-        } else if (BITS == 4) {
-          step_raw4<NB, ONES>(reinterpret_cast<const unsigned(&)[4]>(wa[d]), reinterpret_cast<const unsigned(&)[4]>(wb[d]), xr,
-                        reinterpret_cast<AccRaw4<NB>&>(acc));
+          ta = make_float2(sa, __uint_as_float(0x43004300u | (za * 0x00010001u)));
+          tb = make_float2(sb, __uint_as_float(0x43004300u | (zb * 0x00010001u)));
         } else {
-          step_raw3<NB, ONES>(reinterpret_cast<const unsigned(&)[3]>(wa[d]), reinterpret_cast<const unsigned(&)[3]>(wb[d]), xr,
-                        reinterpret_cast<AccRaw3<NB>&>(acc));
+          ta = make_float2(sa * 16777216.f, sa * (float)za);
+          tb = make_float2(sb * 16777216.f, sb * (float)zb);
         }
-        // refill this slot with the group kDepth steps ahead (its registers are dead now)
-        if (s0 + d + kDepth < nsteps) {
-          load_run<BITS>(p.codes, oa + kDepth * kStepWords, wa[d]);
-          load_run<BITS>(p.codes, ob + kDepth * kStepWords, wb[d]);
-        }
-        oa += kStepWords;
-        ob += kStepWords;
+      }
+      float xsum1 = 0.f;
+      if (!BF16 && !ONES) {   // one token: sum_k x_k of the group, lane L adding columns 4L..4L+3
+        const uint2 h4 = reinterpret_cast<const uint2*>(buf)[xsum_off];
+        const float2 f0 = __half22float2(*reinterpret_cast<const __half2*>(&h4.x));
+        const float2 f1 = __half22float2(*reinterpret_cast<const __half2*>(&h4.y));
+        xsum1 = (f0.x + f0.y) + (f1.x + f1.y);
 #pragma unroll
-        for (int nb = 0; nb < NB; ++nb) {
+        for (int o = 16; o > 0; o >>= 1) xsum1 += __shfl_xor_sync(0xFFFFFFFFu, xsum1, o);
+      }
+      typename StepAcc<BITS, NB, BF16>::type acc = {};
+      unsigned qa[BITS], qb[BITS];
 #pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const float2 tt = i < 2 ? ta : tb;
-            if (BF16) {
-              yacc[nb][i] = fmaf(tt.x, reinterpret_cast<AccSub<NB>&>(acc).c[nb][i], yacc[nb][i]);
-            } else if (BITS == 4) {
-              AccRaw4<NB>& a4 = reinterpret_cast<AccRaw4<NB>&>(acc);
-              const float code_sum = fmaf(a4.c4[nb][i], 0.0625f, a4.c0[nb][i]);         // units of 2^-24
-              const float xsum = ONES ? a4.xs[nb][i & 1] : ((i & 1) == 0 && t == 0 ? xsum1 : 0.f);  // token 0 only
-              yacc[nb][i] = fmaf(tt.x, code_sum, fmaf(-tt.y, xsum, yacc[nb][i]));
-            } else {
-              AccRaw3<NB>& a3 = reinterpret_cast<AccRaw3<NB>&>(acc);
-              const float code_sum = fmaf(a3.c6[nb][i], 0.015625f, fmaf(a3.c3[nb][i], 0.125f, a3.c0[nb][i]));
-              const float xsum = ONES ? a3.xs[nb][i & 1] : ((i & 1) == 0 && t == 0 ? xsum1 : 0.f);  // token 0 only
-              yacc[nb][i] = fmaf(tt.x, code_sum, fmaf(-tt.y, xsum, yacc[nb][i]));
-            }
+      for (int i = 0; i < BITS; ++i) {
+        qa[i] = wa[d][i];
+        qb[i] = wb[d][i];
+      }
+      if (BF16) {
+        step_sub<BITS, NB>(qa, qb, __float_as_uint(ta.y), __float_as_uint(tb.y), xr, reinterpret_cast<AccSub<NB>&>(acc));
+      } else if (BITS == 4) {
+        step_raw4<NB, ONES>(reinterpret_cast<const unsigned(&)[4]>(qa), reinterpret_cast<const unsigned(&)[4]>(qb), xr,
+                            reinterpret_cast<AccRaw4<NB>&>(acc));
+      } else {
+        step_raw3<NB, ONES>(reinterpret_cast<const unsigned(&)[3]>(qa), reinterpret_cast<const unsigned(&)[3]>(qb), xr,
+                            reinterpret_cast<AccRaw3<NB>&>(acc));
+      }
+      // refill the slot with the group kDepth steps ahead
+      const bool refill = c + kDepth < nsteps;
+      load_run_if<BITS>(p.codes, oa + kDepth * kStepWords, wa[d], refill);
+      load_run_if<BITS>(p.codes, ob + kDepth * kStepWords, wb[d], refill);
+      oa += kStepWords;
+      ob += kStepWords;
+#pragma unroll
+      for (int nb = 0; nb < NB; ++nb) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float2 tt = i < 2 ? ta : tb;
+          if (BF16) {
+            yacc[nb][i] = fmaf(tt.x, reinterpret_cast<AccSub<NB>&>(acc).c[nb][i], yacc[nb][i]);
+          } else if (BITS == 4) {
+            AccRaw4<NB>& a4 = reinterpret_cast<AccRaw4<NB>&>(acc);
+            const float code_sum = fmaf(a4.c4[nb][i], 0.0625f, a4.c0[nb][i]);  // units of 2^-24
+            const float xsum = ONES ? a4.xs[nb][i & 1] : ((i & 1) == 0 && t == 0 ? xsum1 : 0.f);  // token 0 only
+            yacc[nb][i] = fmaf(tt.x, code_sum, fmaf(-tt.y, xsum, yacc[nb][i]));
+          } else {
+            AccRaw3<NB>& a3 = reinterpret_cast<AccRaw3<NB>&>(acc);
+            const float code_sum = fmaf(a3.c6[nb][i], 0.015625f, fmaf(a3.c3[nb][i], 0.125f, a3.c0[nb][i]));
+            const float xsum = ONES ? a3.xs[nb][i & 1] : ((i & 1) == 0 && t == 0 ? xsum1 : 0.f);  // token 0 only
+            yacc[nb][i] = fmaf(tt.x, code_sum, fmaf(-tt.y, xsum, yacc[nb][i]));
           }
         }
       }
     }
+
+  };
+  for (int c0 = 0; c0 < nchunks; c0 += kDepth) {   // nchunks is uniform over the CTA: every warp meets every barrier
+    do_chunk(c0, std::integral_constant<int, 0>{});
+    if (c0 + 1 < nchunks) do_chunk(c0 + 1, std::integral_constant<int, 1>{});
+    if (c0 + 2 < nchunks) do_chunk(c0 + 2, std::integral_constant<int, 2>{});
+    if (c0 + 3 < nchunks) do_chunk(c0 + 3, std::integral_constant<int, 3>{});
   }
+  static_assert(kDepth == 4, "the chunk loop is written out for four register slots");
 
   // partial sums of the 8 warps: sm_red[warp][nb][row][token]
 #pragma unroll
@@ -460,46 +569,46 @@ __global__ void __launch_bounds__(kThreads, TP <= 8 ? 3 : (TP == 16 ? 2 : 1)) de
     *reinterpret_cast<float2*>(r + gid * 8 + 2 * t) = make_float2(yacc[nb][0], yacc[nb][1]);
     *reinterpret_cast<float2*>(r + (gid + 8) * 8 + 2 * t) = make_float2(yacc[nb][2], yacc[nb][3]);
   }
-
-  // CSR outliers of the two owned rows: lane = entry, every token per lane, then one
-  // transposing reduction over the lanes
-  auto x_at = [&](int m, unsigned col) -> float {
-    if (XS) {
-      const uint16_t* xs16 = reinterpret_cast<const uint16_t*>(sm_x);
-      return act_to_float<BF16>(xs16[(xs_chunk((int)(col >> 3), m, pitch) << 3) + (col & 7)]);
-    }
-    return act_to_float<BF16>(__ldg(p.x + (size_t)m * p.K + col));
-  };
+  // CSR outliers of the two owned rows
+  if (NBUF == 0) {
+    // every chunk is still in shared memory: lane = entry, every token per lane, one transposing
+    // reduction per row; entries beyond the 96 held in registers (rare) read x from global memory
+    const uint16_t* xs16 = reinterpret_cast<const uint16_t*>(sm_x);
 #pragma unroll
-  for (int rr = 0; rr < 2; ++rr) {
-    const int lr = 2 * warp + rr;
-    const int jb = rr == 0 ? j0 : j1, je = rr == 0 ? j1 : j2;
-    float v[TP];
+    for (int rr = 0; rr < 2; ++rr) {
+      const int lr = 2 * warp + rr;
+      const int jb = rr == 0 ? j0 : j1, je = rr == 0 ? j1 : j2;
+      float v[TP];
 #pragma unroll
-    for (int m = 0; m < TP; ++m) v[m] = 0.f;
-    if (r0 + lr < p.N && je > jb) {
-      const int ne = min(kOutSlots, (je - jb + 31) >> 5);  // warp-uniform
+      for (int m = 0; m < TP; ++m) v[m] = 0.f;
+      if (je > jb) {
+        const int ne = min(kOutSlots, (je - jb + 31) >> 5);   // warp-uniform
 #pragma unroll
-      for (int e = 0; e < kOutSlots; ++e) {
-        if (e < ne) {
-          const float wv = __half2float(__ushort_as_half((unsigned short)(cv[rr][e] >> 16)));
-          const unsigned col = cv[rr][e] & 0xFFFFu;
+        for (int e = 0; e < kOutSlots; ++e) {
+          if (e < ne && cv[rr][e] != 0xFFFFFFFFu) {
+            const float wv = __half2float(__ushort_as_half((unsigned short)(cv[rr][e] >> 16)));
+            const unsigned col = cv[rr][e] & 0xFFFFu;
+            const int base = (int)(col >> 10) * buf_pieces;            // chunk = col / 1024
+            const int pc = (int)((col & 1023u) >> 3), sub = (int)(col & 7u);
+#pragma unroll
+            for (int m = 0; m < TP; ++m)
+              if (TP == 1 || m < p.M)
+                v[m] = fmaf(wv, act_to_float<BF16>(xs16[((base + xs_piece(pc, m)) << 3) + sub]), v[m]);
+          }
+        }
+        for (int j = jb + 32 * kOutSlots + lane; j < je; j += 32) {
+          const unsigned e = __ldg(p.cv + j);
+          const float wv = __half2float(__ushort_as_half((unsigned short)(e >> 16)));
 #pragma unroll
           for (int m = 0; m < TP; ++m)
-            if (TP == 1 || m < p.M) v[m] = fmaf(wv, x_at(m, col), v[m]);
+            if (TP == 1 || m < p.M)
+              v[m] = fmaf(wv, act_to_float<BF16>(__ldg(p.x + (size_t)m * p.K + (e & 0xFFFFu))), v[m]);
         }
       }
-      for (int j = jb + 32 * kOutSlots + lane; j < je; j += 32) {  // rows with more than 96 outliers
-        const unsigned e = __ldg(p.cv + j);
-        const float wv = __half2float(__ushort_as_half((unsigned short)(e >> 16)));
-#pragma unroll
-        for (int m = 0; m < TP; ++m)
-          if (TP == 1 || m < p.M) v[m] = fmaf(wv, x_at(m, e & 0xFFFFu), v[m]);
-      }
+      reduce_tokens<TP, 1>(v, lane);
+      constexpr int LPT = 32 / TP;   // lanes per token after the reduction
+      if ((lane & (LPT - 1)) == 0) sm_out[lr * TP + lane / LPT] = v[0];
     }
-    reduce_across_lanes<TP>(v, lane);
-    constexpr int LPT = 32 / TP;  // lanes per token after the reduction
-    if ((lane & (LPT - 1)) == 0) sm_out[lr * TP + lane / LPT] = v[0];
   }
   __syncthreads();
 
@@ -517,16 +626,35 @@ __global__ void __launch_bounds__(kThreads, TP <= 8 ? 3 : (TP == 16 ? 2 : 1)) de
   }
 }
 
-constexpr size_t kXStageLimit = 72 * 1024;  // activations above this are read through L1 instead
+// xt[col][token] = x[token][col] for token < M (zero beyond), TP tokens per column.
+template <int TP>
+__global__ void __launch_bounds__(256) tokens_to_columns(const uint16_t* __restrict__ x, uint16_t* __restrict__ xt, int M, int K) {
+  constexpr int PARTS = TP >= 8 ? TP / 8 : 1, W = TP >= 8 ? 8 : TP;
+  const int id = blockIdx.x * 256 + threadIdx.x;
+  const int col = id / PARTS, part = id % PARTS;
+  if (col >= K) return;
+  uint16_t v[W];
+#pragma unroll
+  for (int i = 0; i < W; ++i) {
+    const int m = part * W + i;
+    v[i] = m < M ? __ldg(x + (size_t)m * K + col) : (uint16_t)0;
+  }
+  uint16_t* dst = xt + (size_t)col * TP + part * W;
+#pragma unroll
+  for (int i = 0; i < W; ++i) dst[i] = v[i];
+}
 
-template <int BITS, int TP, bool BF16, bool XS>
+constexpr size_t kStageAllLimit = 72 * 1024;   // stage every chunk up front when it fits in this much
+
+template <int BITS, int TP, bool BF16, int NBUF>
 cudaError_t launch(const DecodeArgs& a, cudaStream_t stream) {
   constexpr int NB = TP <= 8 ? 1 : TP / 8;
   const int ngroups = a.K / 128;
+  const int nchunks = (ngroups + kChunkGroups - 1) / kChunkGroups;
   const size_t smem = 64 + (size_t)kRows * ngroups * 3 + (size_t)kWarps * NB * 128 * 4 + (size_t)kRows * TP * 4 +
-                      (XS ? (size_t)a.M * xs_pitch_chunks(a.K) * 16 : 0);
+                      (NBUF == 0 ? (size_t)nchunks * a.M * kRowPitch : (size_t)kWarps * 2 * a.M * kTilePitch) * 16;
   if (smem > 48 * 1024) {
-    cudaError_t e = cudaFuncSetAttribute(decode_kernel<BITS, TP, BF16, XS>,
+    cudaError_t e = cudaFuncSetAttribute(decode_kernel<BITS, TP, BF16, NBUF>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
   }
@@ -540,22 +668,30 @@ cudaError_t launch(const DecodeArgs& a, cudaStream_t stream) {
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, decode_kernel<BITS, TP, BF16, XS>, a);
+  return cudaLaunchKernelEx(&cfg, decode_kernel<BITS, TP, BF16, NBUF>, a);
 }
 
-template <int BITS, bool BF16, bool XS>
-cudaError_t launch_tp(const DecodeArgs& a, cudaStream_t stream) {
-  if (a.M == 1) return launch<BITS, 1, BF16, XS>(a, stream);
-  if (a.M <= 4) return launch<BITS, 4, BF16, XS>(a, stream);
-  if (a.M <= 8) return launch<BITS, 8, BF16, XS>(a, stream);
-  if (a.M <= 16) return launch<BITS, 16, BF16, XS>(a, stream);
-  return launch<BITS, 32, BF16, XS>(a, stream);
+// ring depth used when the activations do not fit up front
+template <int BITS, int TP, bool BF16, int RING>
+cudaError_t launch_buf(const DecodeArgs& a, cudaStream_t stream) {
+  const int nchunks = (a.K / 128 + kChunkGroups - 1) / kChunkGroups;
+  if (TP <= 8 && (size_t)nchunks * a.M * kRowPitch * 16 <= kStageAllLimit) return launch<BITS, TP, BF16, 0>(a, stream);
+  if (TP > 1) {   // ring mode gathers the outliers' activations from a token-major copy
+    if (!a.xt) return cudaErrorInvalidValue;
+    tokens_to_columns<TP><<<(a.K * (TP >= 8 ? TP / 8 : 1) + 255) / 256, 256, 0, stream>>>(a.x, const_cast<uint16_t*>(a.xt), a.M, a.K);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+  }
+  return launch<BITS, TP, BF16, RING>(a, stream);
 }
 
 template <int BITS, bool BF16>
-cudaError_t launch_xs(const DecodeArgs& a, cudaStream_t stream) {
-  if ((size_t)a.M * xs_pitch_chunks(a.K) * 16 <= kXStageLimit) return launch_tp<BITS, BF16, true>(a, stream);
-  return launch_tp<BITS, BF16, false>(a, stream);
+cudaError_t launch_tp(const DecodeArgs& a, cudaStream_t stream) {
+  if (a.M == 1) return launch_buf<BITS, 1, BF16, 2>(a, stream);
+  if (a.M <= 4) return launch_buf<BITS, 4, BF16, 2>(a, stream);
+  if (a.M <= 8) return launch_buf<BITS, 8, BF16, 2>(a, stream);
+  if (a.M <= 16) return launch_buf<BITS, 16, BF16, 2>(a, stream);
+  return launch_buf<BITS, 32, BF16, 2>(a, stream);
 }
 
 }  // namespace
@@ -563,16 +699,32 @@ cudaError_t launch_xs(const DecodeArgs& a, cudaStream_t stream) {
 // Decode launcher: group size 128, M <= 32, K <= 65536.  Other shapes go to the general kernel.
 gwq_status gwq_launch_decode(const gwq_packed* P, const void* x, gwq_dtype xd, int M, void* y, gwq_dtype yd,
                              cudaStream_t stream) {
-  const gwq_priv* pv = static_cast<const gwq_priv*>(P->priv);
+  gwq_priv* pv = static_cast<gwq_priv*>(P->priv);
   if (P->group != 128 || M > 32 || !pv->cv) return gwq_launch_simt(P, x, xd, M, y, yd, stream);
   DecodeArgs a;
+  a.xt = nullptr;
+  if (M > 1) {   // scratch for the token-major copy (used when the activations are not staged up front)
+    const size_t need = (size_t)P->K * 32 * 2;
+    if (pv->xt_bytes < need) {
+      if (cudaStreamSynchronize(stream) != cudaSuccess) return GWQ_ERR_CUDA;
+      if (pv->xt) cudaFree(pv->xt);
+      pv->xt = nullptr;
+      pv->xt_bytes = 0;
+      if (cudaMalloc(&pv->xt, need) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return GWQ_ERR_ALLOC;
+      }
+      pv->xt_bytes = need;
+    }
+    a.xt = static_cast<const uint16_t*>(pv->xt);
+  }
   a.codes = P->codes; a.scales = P->scales; a.zeros = P->zeros;
   a.row_ptr = P->S->row_ptr; a.cv = pv->cv;
   a.x = static_cast<const uint16_t*>(x); a.y = y; a.yd = yd;
   a.N = P->N; a.K = P->K; a.M = M;
   cudaError_t e;
-  if (P->bits == 4) e = (xd == GWQ_BF16) ? launch_xs<4, true>(a, stream) : launch_xs<4, false>(a, stream);
-  else e = (xd == GWQ_BF16) ? launch_xs<3, true>(a, stream) : launch_xs<3, false>(a, stream);
+  if (P->bits == 4) e = (xd == GWQ_BF16) ? launch_tp<4, true>(a, stream) : launch_tp<4, false>(a, stream);
+  else e = (xd == GWQ_BF16) ? launch_tp<3, true>(a, stream) : launch_tp<3, false>(a, stream);
   if (e != cudaSuccess) {
     (void)cudaGetLastError();
     return GWQ_ERR_CUDA;

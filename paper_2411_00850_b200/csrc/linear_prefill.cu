@@ -28,7 +28,7 @@ namespace {
 constexpr int kTileN = 128;      // weight rows per CTA (UMMA M)
 constexpr int kBlockK = 64;      // k-block: 128 bytes of 16-bit operands
 constexpr int kDequantWarps = 4;   // warps of one dequantisation group (one thread per tile row)
-__host__ __device__ constexpr int dq_groups(int tok) { return tok >= 128 ? 4 : 2; }
+__host__ __device__ constexpr int dq_groups(int tok) { return 4; }
 __host__ __device__ constexpr int cta_threads(int tok) { return 32 * (2 + kDequantWarps * dq_groups(tok)); }
 constexpr int kMaxStages = 8;
 constexpr long long kSpinCycles = 1000LL * 1000LL * 1000LL;   // about half a second of SM clock
@@ -382,7 +382,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmx, const PrefillArgs p, con
     if (ok) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll 1
-      for (int c0 = gq * (TOK / G); c0 < (gq + 1) * (TOK / G); c0 += 32) {   // each group drains its share
+      constexpr int kShare = TOK / G >= 32 ? TOK / G : 32;   // token columns drained by one group
+      for (int c0 = gq * kShare; c0 < (gq + 1) * kShare && c0 < TOK; c0 += 32) {
         if (m0 + c0 >= p.M) break;             // warp-uniform
         unsigned v[32];
         tmem_ld32(tmem_acc + ((unsigned)(quad * 32) << 16) + (unsigned)c0, v);
@@ -478,6 +479,7 @@ gwq_status launch(const gwq_packed* P, const void* x, const float* tok_scale, in
 template <int BITS>
 gwq_status launch_tok(const gwq_packed* P, const void* x, const float* tok_scale, int M, void* y, gwq_dtype yd,
                       cudaStream_t stream) {
+  if (M <= 32) return launch<BITS, 32>(P, x, tok_scale, M, y, yd, stream);
   if (M <= 64) return launch<BITS, 64>(P, x, tok_scale, M, y, yd, stream);
   if (M <= 128) return launch<BITS, 128>(P, x, tok_scale, M, y, yd, stream);
   return launch<BITS, 256>(P, x, tok_scale, M, y, yd, stream);
