@@ -119,6 +119,24 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def max_over_ranks(ms_local: float, device=None) -> float:
+    """Slowest rank's time: the whole job is as slow as its slowest replica.  Works on any backend
+    (NCCL on the GPUs, gloo in the CPU test); a single process returns its own time."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(ms_local)
+    t = torch.tensor([float(ms_local)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_gbs(step_bytes: int, ms_step_max: float, world: int) -> float:
+    """Replicas only: every rank runs the same step on its own copy of the layer set, nothing is
+    exchanged; the job moved world * step_bytes in the time of the slowest rank."""
+    return world * step_bytes / (ms_step_max * 1e-3) / 1e9
+
+
 # ----------------------------------------------------------------------------- the CUDA arm
 def build_layer_set(torch, gwq, dev, replicas: int, keep_dense: bool):
     """Generate the 7 seeded layers, encode each to 4 and 3 bits on the GPU.
@@ -253,12 +271,10 @@ def run_cuda_arm(args):
         time.sleep(0.3)
     ms_step = time_region(torch, lambda i: graphs[i % replicas](), args.steps)
     if world > 1:
-        t = torch.tensor([ms_step], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_step = float(t.item())
+        ms_step = max_over_ranks(ms_step, dev)
         dist.barrier()
     clocks = sampler.stop() if rank == 0 else {}
-    value = world * step_bytes / (ms_step * 1e-3) / 1e9
+    value = whole_job_gbs(step_bytes, ms_step, world)
 
     out = {
         "metric": METRIC, "value": round(value, 1), "unit": "GB/s", "n_gpus": world, "steps": args.steps,
