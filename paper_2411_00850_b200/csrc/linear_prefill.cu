@@ -6,12 +6,14 @@
 // in the 128-byte-swizzled layout, the FP32 accumulator lives in tensor memory.
 //   warp 0, one thread : TMA loads of the activation tile (TOK x 64) per k-block
 //   warp 1, one thread : tcgen05.mma (4 x K=16 per k-block), tcgen05.commit frees the stage
-//   warps 2..          : G groups of 4 warps, group g taking the k-blocks g, g+G, ...; in a group
+//   warps 2..13        : 3 groups of 4 warps, group g taking the k-blocks g, g+3, ...; in a group
 //                        one thread per weight row: packed codes from global memory -> exact
 //                        q - z by a magic-number subtract -> times the group scale -> 128 bytes
 //                        of the swizzled A tile; the row's CSR outliers are written over their
 //                        (exactly zero) dense entries, so the tensor cores also do the SpMM;
-//                        afterwards the same warps drain the accumulator (tcgen05.ld) and store y
+//   warps 14..17       : epilogue, one thread per output feature: tcgen05.ld, conversion, stores
+// The CTAs are persistent (one per SM, tiles handed out round-robin) and keep two accumulators in
+// tensor memory, so the epilogue of a tile runs under the main loop of the next one.
 // The tensor cores always run in fp16: bf16 activations are first rewritten, one pass, as
 // fp16 x 2^-e with one power of two per token (exact for every element within 2^-14 of the
 // token's largest, i.e. for everything that matters), because weights rounded to bf16 (8 bits)
@@ -28,8 +30,9 @@ namespace {
 constexpr int kTileN = 128;      // weight rows per CTA (UMMA M)
 constexpr int kBlockK = 64;      // k-block: 128 bytes of 16-bit operands
 constexpr int kDequantWarps = 4;   // warps of one dequantisation group (one thread per tile row)
-__host__ __device__ constexpr int dq_groups(int tok) { return 4; }
-__host__ __device__ constexpr int cta_threads(int tok) { return 32 * (2 + kDequantWarps * dq_groups(tok)); }
+constexpr int kDequantGroups = 3;  // groups; group g takes the k-blocks g, g + 3, ... (numbered over all tiles)
+constexpr int kEpilogueWarps = 4;  // one thread per tile row
+constexpr int kCtaThreads = 32 * (2 + kDequantWarps * kDequantGroups + kEpilogueWarps);
 constexpr int kMaxStages = 8;
 constexpr long long kSpinCycles = 1000LL * 1000LL * 1000LL;   // about half a second of SM clock
 
@@ -200,28 +203,33 @@ __device__ __forceinline__ unsigned sub_magic(unsigned qm, unsigned zm) {
 }
 
 template <int BITS, int TOK, bool BF16>
-__global__ void __launch_bounds__(cta_threads(TOK), 1)
-prefill_kernel(const __grid_constant__ CUtensorMap tmx, const PrefillArgs p, const int stages) {
+__global__ void __launch_bounds__(kCtaThreads, 1)
+prefill_kernel(const __grid_constant__ CUtensorMap tmx, const PrefillArgs p, const int stages, const int ntn,
+               const int ntiles) {
   constexpr int kABytes = kTileN * kBlockK * 2;   // 16 KB
   constexpr int kBBytes = TOK * kBlockK * 2;
+  constexpr int kAccCols = TOK < 32 ? 32 : TOK;   // tensor-memory columns of one accumulator
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* tiles =
       reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
-  __shared__ __align__(8) unsigned long long bars[3 * kMaxStages + 1];
+  __shared__ __align__(8) unsigned long long bars[3 * kMaxStages + 4];
   __shared__ unsigned tmem_base_s;
   __shared__ int abort_s;
   volatile int* abort_flag = &abort_s;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int n0 = blockIdx.x * kTileN, m0 = blockIdx.y * TOK;
   const int nkb = p.K / kBlockK;
   const unsigned bar0 = smem_u32(bars);
   auto full_b = [&](int s) { return bar0 + 8u * s; };
   auto full_a = [&](int s) { return bar0 + 8u * (kMaxStages + s); };
   auto empty = [&](int s) { return bar0 + 8u * (2 * kMaxStages + s); };
-  const unsigned accum_bar = bar0 + 8u * (3 * kMaxStages);
+  auto acc_full = [&](int a) { return bar0 + 8u * (3 * kMaxStages + a); };
+  auto acc_empty = [&](int a) { return bar0 + 8u * (3 * kMaxStages + 2 + a); };
   auto a_tile = [&](int s) { return tiles + (size_t)s * (kABytes + kBBytes); };
   auto b_tile = [&](int s) { return tiles + (size_t)s * (kABytes + kBBytes) + kABytes; };
+  // this CTA's tiles: blockIdx.x, blockIdx.x + gridDim.x, ...; the feature tile runs fastest, so the CTAs
+  // that are busy at the same time share their activation rows in L2
+  const int my_tiles = blockIdx.x < ntiles ? (ntiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
 
   if (tid == 0) {
     abort_s = 0;
@@ -230,12 +238,15 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmx, const PrefillArgs p, con
       mbar_init(full_a(s), kDequantWarps);
       mbar_init(empty(s), 1);
     }
-    mbar_init(accum_bar, 1);
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(acc_full(a), 1);
+      mbar_init(acc_empty(a), kEpilogueWarps);
+    }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 1) {   // tensor memory for the accumulator: TOK columns of 128 lanes
+  if (warp == 1) {   // tensor memory: two accumulators of kAccCols columns x 128 lanes
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)),
-                 "r"(TOK)
+                 "r"(2 * kAccCols)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -244,18 +255,22 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmx, const PrefillArgs p, con
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const unsigned tmem_acc = tmem_base_s;
   bool ok = *reinterpret_cast<volatile int32_t*>(p.status) == 0;   // an earlier CTA gave up: do no work
-  int issued = 0;   // k-blocks whose activation copy was started (producer thread only)
+  int issued = 0;   // k-block copies started (producer thread only), counted over all tiles
 
   if (warp == 0) {
     // ------------------------------------------------------------------ activation tiles by TMA
     if (lane == 0) {
-      for (int kb = 0; kb < nkb && ok; ++kb) {
-        const int s = kb % stages, round = kb / stages;
-        if (round > 0) ok = mbar_wait(empty(s), (round - 1) & 1, abort_flag);
-        if (!ok) break;
-        mbar_expect_tx(full_b(s), kBBytes);
-        tma_load_2d(smem_u32(b_tile(s)), &tmx, kb * kBlockK, m0, full_b(s));
-        issued = kb + 1;
+      for (int ti = 0; ti < my_tiles && ok; ++ti) {
+        const int tile = blockIdx.x + ti * gridDim.x;
+        const int m0 = (tile / ntn) * TOK;
+        for (int kb = 0; kb < nkb && ok; ++kb) {
+          const int it = ti * nkb + kb, s = it % stages, round = it / stages;
+          if (round > 0) ok = mbar_wait(empty(s), (round - 1) & 1, abort_flag);
+          if (!ok) break;
+          mbar_expect_tx(full_b(s), kBBytes);
+          tma_load_2d(smem_u32(b_tile(s)), &tmx, kb * kBlockK, m0, full_b(s));
+          issued = it + 1;
+        }
       }
     }
   } else if (warp == 1) {
@@ -264,129 +279,146 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmx, const PrefillArgs p, con
       // instruction descriptor: FP32 accumulate, A and B both fp16 or both bf16, K-major, N = TOK, M = 128
       const unsigned idesc = (1u << 4) | ((BF16 ? 1u : 0u) << 7) | ((BF16 ? 1u : 0u) << 10) |
                              ((unsigned)(TOK >> 3) << 17) | ((unsigned)(kTileN >> 4) << 24);
-      for (int kb = 0; kb < nkb && ok; ++kb) {
-        const int s = kb % stages, round = kb / stages;
-        ok = mbar_wait(full_a(s), round & 1, abort_flag) && mbar_wait(full_b(s), round & 1, abort_flag);
+      for (int ti = 0; ti < my_tiles && ok; ++ti) {
+        const int a = ti & 1;
+        if (ti >= 2) ok = mbar_wait(acc_empty(a), ((ti >> 1) - 1) & 1, abort_flag);   // drained by the epilogue
         if (!ok) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint64_t da = umma_desc(smem_u32(a_tile(s))), db = umma_desc(smem_u32(b_tile(s)));
+        const unsigned acc = tmem_acc + (unsigned)(a * kAccCols);
+        for (int kb = 0; kb < nkb && ok; ++kb) {
+          const int it = ti * nkb + kb, s = it % stages, round = it / stages;
+          ok = mbar_wait(full_a(s), round & 1, abort_flag) && mbar_wait(full_b(s), round & 1, abort_flag);
+          if (!ok) break;
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          const uint64_t da = umma_desc(smem_u32(a_tile(s))), db = umma_desc(smem_u32(b_tile(s)));
 #pragma unroll
-        for (int k = 0; k < kBlockK / 16; ++k)   // 32 bytes further along K inside the swizzle atom
-          umma_f16(tmem_acc, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (kb | k) != 0);
-        umma_commit(empty(s));
+          for (int k = 0; k < kBlockK / 16; ++k)   // 32 bytes further along K inside the swizzle atom
+            umma_f16(acc, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (kb | k) != 0);
+          umma_commit(empty(s));
+        }
+        if (ok) umma_commit(acc_full(a));
       }
-      if (ok) umma_commit(accum_bar);
+    }
+  } else if (warp < 2 + kDequantWarps * kDequantGroups) {
+    // ------------------------------------------------------------------ dequantisation
+    constexpr int G = kDequantGroups;
+    const int gq = (warp - 2) >> 2;            // group: global k-block numbers gq, gq + G, ...
+    const int r = (warp & 3) * 32 + lane;      // row inside the tile
+    constexpr int WPB = kBlockK * BITS / 32;   // packed words per row per k-block (8 or 6)
+    constexpr unsigned MAGIC = BF16 ? 0x43004300u : 0x64006400u;   // 128.0 / 1024.0: ulp = 1
+    constexpr int kOutWin = 8;                 // outliers of the row kept this many entries ahead
+    for (int ti = 0; ti < my_tiles && ok; ++ti) {
+      const int tile = blockIdx.x + ti * gridDim.x;
+      const int row = (tile % ntn) * kTileN + r;
+      const bool live = row < p.N;
+      const int rowc = live ? row : p.N - 1;
+      const uint32_t* crow = p.codes + (size_t)rowc * (p.K / 32) * BITS;
+      const uint32_t* szcol = p.sz_t + rowc;   // [group][row] table: neighbouring rows are neighbouring words
+      int j = 0, je = 0;
+      if (live) {
+        j = p.row_ptr[row];
+        je = p.row_ptr[row + 1];
+      }
+      unsigned win[kOutWin];
+#pragma unroll
+      for (int i = 0; i < kOutWin; ++i) win[i] = j + i < je ? __ldg(p.cv + j + i) : 0xFFFFFFFFu;
+      // first k-block of this tile that belongs to the group
+      int kb = ((gq - ti * nkb) % G + G) % G;
+      unsigned wq[WPB];
+      unsigned sz_nx = 0;   // scale (fp16 bits) | zero-point << 16 of the group of the next k-block
+      if (kb < nkb) {
+        load_words<WPB>(crow + (size_t)kb * WPB, wq);
+        sz_nx = __ldg(szcol + (size_t)((kb * kBlockK) / p.group) * p.N);
+      }
+      for (; kb < nkb && ok; kb += G) {
+        const int it = ti * nkb + kb, s = it % stages, round = it / stages;
+        const float sc = live ? __half2float(__ushort_as_half((unsigned short)(sz_nx & 0xFFFFu))) : 0.f;
+        const unsigned z = sz_nx >> 16;
+        unsigned s_hi2, s_lo2 = 0;
+        if (BF16) {
+          const __nv_bfloat16 hi = __float2bfloat16_rn(sc);
+          const __nv_bfloat16 lo = __float2bfloat16_rn(sc - __bfloat162float(hi));
+          s_hi2 = (unsigned)__bfloat16_as_ushort(hi) * 0x00010001u;
+          s_lo2 = (unsigned)__bfloat16_as_ushort(lo) * 0x00010001u;
+        } else {
+          s_hi2 = (unsigned)__half_as_ushort(__float2half_rn(sc)) * 0x00010001u;
+        }
+        const unsigned zm = MAGIC | (z * 0x00010001u);
+        unsigned cur[WPB];
+#pragma unroll
+        for (int i = 0; i < WPB; ++i) cur[i] = wq[i];
+        if (kb + G < nkb) {   // codes, scale and zero-point of this group's next k-block
+          load_words<WPB>(crow + (size_t)(kb + G) * WPB, wq);
+          sz_nx = __ldg(szcol + (size_t)(((kb + G) * kBlockK) / p.group) * p.N);
+        }
+        // 64 codes -> 32 pairs (columns 2h, 2h+1) -> 8 chunks of 16 bytes
+        unsigned out[32];
+        if (BITS == 4) {
+#pragma unroll
+          for (int i = 0; i < 8; ++i)
+#pragma unroll
+            for (int q4 = 0; q4 < 4; ++q4)
+              out[4 * i + q4] = mul_scale<BF16>(
+                  sub_magic<BF16>(((cur[i % WPB] >> (4 * q4)) & 0x000F000Fu) | MAGIC, zm), s_hi2, s_lo2);
+        } else {
+#pragma unroll
+          for (int run = 0; run < 2; ++run) {
+            const unsigned* w3 = cur + (run * 3) % WPB;
+#pragma unroll
+            for (int i = 0; i < 3; ++i)
+#pragma unroll
+              for (int pp = 0; pp < 5; ++pp)
+                out[16 * run + 5 * i + pp] =
+                    mul_scale<BF16>(sub_magic<BF16>(((w3[i] >> (3 * pp)) & 0x00070007u) | MAGIC, zm), s_hi2, s_lo2);
+            const unsigned last =
+                ((w3[0] >> 15) & 0x00010001u) | ((w3[1] >> 14) & 0x00020002u) | ((w3[2] >> 13) & 0x00040004u);
+            out[16 * run + 15] = mul_scale<BF16>(sub_magic<BF16>(last | MAGIC, zm), s_hi2, s_lo2);
+          }
+        }
+        if (round > 0) ok = mbar_wait(empty(s), (round - 1) & 1, abort_flag);
+        if (!ok) break;
+        unsigned char* arow = a_tile(s) + r * 128;
+#pragma unroll
+        for (int c = 0; c < 8; ++c)
+          *reinterpret_cast<uint4*>(arow + ((c ^ (r & 7)) << 4)) =
+              make_uint4(out[4 * c], out[4 * c + 1], out[4 * c + 2], out[4 * c + 3]);
+        // the row's outliers inside this k-block replace their dense entries (which are exactly 0)
+        const unsigned k_end = (unsigned)(kb + 1) * kBlockK;
+        while (j < je && (win[0] & 0xFFFFu) < k_end) {   // entries of other groups' k-blocks are skipped
+          const unsigned e = win[0];
+          if ((e & 0xFFFFu) >= k_end - kBlockK) {
+            const unsigned col = (e & 0xFFFFu) - (unsigned)kb * kBlockK;
+            unsigned short v16 = (unsigned short)(e >> 16);
+            if (BF16) v16 = __bfloat16_as_ushort(__float2bfloat16_rn(__half2float(__ushort_as_half(v16))));
+            *reinterpret_cast<unsigned short*>(arow + ((((col >> 3) ^ (r & 7)) << 4) | ((col & 7) << 1))) = v16;
+          }
+          ++j;
+#pragma unroll
+          for (int i = 0; i + 1 < kOutWin; ++i) win[i] = win[i + 1];
+          win[kOutWin - 1] = j + kOutWin - 1 < je ? __ldg(p.cv + j + kOutWin - 1) : 0xFFFFFFFFu;
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to the MMA
+        __syncwarp();
+        if (lane == 0) mbar_arrive(full_a(s));
+      }
     }
   } else {
-    // ------------------------------------------------------------------ dequantization, then epilogue
-    constexpr int G = dq_groups(TOK);
-    const int gq = (warp - 2) >> 2;            // dequantisation group: k-blocks gq, gq + G, ...
+    // ------------------------------------------------------------------ epilogue: one thread per output feature
     const int quad = warp & 3;                 // tensor-memory lane quarter this warp may access
-    const int r = quad * 32 + lane;            // row inside the tile
-    const int row = n0 + r;
-    const bool live = row < p.N;
-    const int rowc = live ? row : p.N - 1;
-    constexpr int WPB = kBlockK * BITS / 32;   // packed words per row per k-block (8 or 6)
-    const uint32_t* crow = p.codes + (size_t)rowc * (p.K / 32) * BITS;
-    const uint32_t* szcol = p.sz_t + rowc;   // [group][row] table: neighbouring rows are neighbouring words
-    int j = 0, je = 0;
-    if (live) {
-      j = p.row_ptr[row];
-      je = p.row_ptr[row + 1];
-    }
-    // the row's next outliers, kept kOutWin entries ahead so that walking the list never waits on memory
-    constexpr int kOutWin = 8;
-    unsigned win[kOutWin];
-#pragma unroll
-    for (int i = 0; i < kOutWin; ++i) win[i] = j + i < je ? __ldg(p.cv + j + i) : 0xFFFFFFFFu;
-    constexpr unsigned MAGIC = BF16 ? 0x43004300u : 0x64006400u;   // 128.0 / 1024.0: ulp = 1
-    unsigned wq[WPB];
-    unsigned sz_nx = 0;   // scale (fp16 bits) | zero-point << 16 of the group of the next k-block
-    if (gq < nkb) {
-      load_words<WPB>(crow + (size_t)gq * WPB, wq);
-      sz_nx = __ldg(szcol + (size_t)((gq * kBlockK) / p.group) * p.N);
-    }
-    for (int kb = gq; kb < nkb && ok; kb += G) {
-      const int s = kb % stages, round = kb / stages;
-      const float sc = live ? __half2float(__ushort_as_half((unsigned short)(sz_nx & 0xFFFFu))) : 0.f;
-      const unsigned z = sz_nx >> 16;
-      unsigned s_hi2, s_lo2 = 0;
-      if (BF16) {
-        const __nv_bfloat16 hi = __float2bfloat16_rn(sc);
-        const __nv_bfloat16 lo = __float2bfloat16_rn(sc - __bfloat162float(hi));
-        s_hi2 = (unsigned)__bfloat16_as_ushort(hi) * 0x00010001u;
-        s_lo2 = (unsigned)__bfloat16_as_ushort(lo) * 0x00010001u;
-      } else {
-        s_hi2 = (unsigned)__half_as_ushort(__float2half_rn(sc)) * 0x00010001u;
-      }
-      const unsigned zm = MAGIC | (z * 0x00010001u);
-      unsigned cur[WPB];
-#pragma unroll
-      for (int i = 0; i < WPB; ++i) cur[i] = wq[i];
-      if (kb + G < nkb) {   // codes, scale and zero-point of this group's next k-block
-        load_words<WPB>(crow + (size_t)(kb + G) * WPB, wq);
-        sz_nx = __ldg(szcol + (size_t)(((kb + G) * kBlockK) / p.group) * p.N);
-      }
-      // 64 codes -> 32 pairs (columns 2h, 2h+1) -> 8 chunks of 16 bytes
-      unsigned out[32];
-      if (BITS == 4) {
-#pragma unroll
-        for (int i = 0; i < 8; ++i)
-#pragma unroll
-          for (int q4 = 0; q4 < 4; ++q4)
-            out[4 * i + q4] = mul_scale<BF16>(
-                sub_magic<BF16>(((cur[i % WPB] >> (4 * q4)) & 0x000F000Fu) | MAGIC, zm), s_hi2, s_lo2);
-      } else {
-#pragma unroll
-        for (int run = 0; run < 2; ++run) {
-          const unsigned* w3 = cur + (run * 3) % WPB;
-#pragma unroll
-          for (int i = 0; i < 3; ++i)
-#pragma unroll
-            for (int pp = 0; pp < 5; ++pp)
-              out[16 * run + 5 * i + pp] =
-                  mul_scale<BF16>(sub_magic<BF16>(((w3[i] >> (3 * pp)) & 0x00070007u) | MAGIC, zm), s_hi2, s_lo2);
-          const unsigned last =
-              ((w3[0] >> 15) & 0x00010001u) | ((w3[1] >> 14) & 0x00020002u) | ((w3[2] >> 13) & 0x00040004u);
-          out[16 * run + 15] = mul_scale<BF16>(sub_magic<BF16>(last | MAGIC, zm), s_hi2, s_lo2);
-        }
-      }
-      if (round > 0) ok = mbar_wait(empty(s), (round - 1) & 1, abort_flag);
+    const int r = quad * 32 + lane;
+    for (int ti = 0; ti < my_tiles && ok; ++ti) {
+      const int tile = blockIdx.x + ti * gridDim.x;
+      const int row = (tile % ntn) * kTileN + r, m0 = (tile / ntn) * TOK;
+      const bool live = row < p.N;
+      const int a = ti & 1;
+      ok = mbar_wait(acc_full(a), (ti >> 1) & 1, abort_flag);
       if (!ok) break;
-      unsigned char* arow = a_tile(s) + r * 128;
-#pragma unroll
-      for (int c = 0; c < 8; ++c)
-        *reinterpret_cast<uint4*>(arow + ((c ^ (r & 7)) << 4)) =
-            make_uint4(out[4 * c], out[4 * c + 1], out[4 * c + 2], out[4 * c + 3]);
-      // the row's outliers inside this k-block replace their dense entries (which are exactly 0)
-      const unsigned k_end = (unsigned)(kb + 1) * kBlockK;
-      while (j < je && (win[0] & 0xFFFFu) < k_end) {   // entries of other groups' k-blocks are skipped
-        const unsigned e = win[0];
-        if ((e & 0xFFFFu) >= k_end - kBlockK) {
-          const unsigned col = (e & 0xFFFFu) - (unsigned)kb * kBlockK;
-          unsigned short v16 = (unsigned short)(e >> 16);
-          if (BF16) v16 = __bfloat16_as_ushort(__float2bfloat16_rn(__half2float(__ushort_as_half(v16))));
-          *reinterpret_cast<unsigned short*>(arow + ((((col >> 3) ^ (r & 7)) << 4) | ((col & 7) << 1))) = v16;
-        }
-        ++j;
-#pragma unroll
-        for (int i = 0; i + 1 < kOutWin; ++i) win[i] = win[i + 1];
-        win[kOutWin - 1] = j + kOutWin - 1 < je ? __ldg(p.cv + j + kOutWin - 1) : 0xFFFFFFFFu;
-      }
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to the MMA
-      __syncwarp();
-      if (lane == 0) mbar_arrive(full_a(s));
-    }
-    // ---- epilogue: accumulator lane = output feature, column = token
-    if (ok) ok = mbar_wait(accum_bar, 0, abort_flag);
-    if (ok) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll 1
-      constexpr int kShare = TOK / G >= 32 ? TOK / G : 32;   // token columns drained by one group
-      for (int c0 = gq * kShare; c0 < (gq + 1) * kShare && c0 < TOK; c0 += 32) {
+      for (int c0 = 0; c0 < TOK; c0 += 32) {
         if (m0 + c0 >= p.M) break;             // warp-uniform
         unsigned v[32];
-        tmem_ld32(tmem_acc + ((unsigned)(quad * 32) << 16) + (unsigned)c0, v);
+        tmem_ld32(tmem_acc + ((unsigned)(quad * 32) << 16) + (unsigned)(a * kAccCols + c0), v);
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
         if (live) {
 #pragma unroll
@@ -403,6 +435,10 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmx, const PrefillArgs p, con
           }
         }
       }
+      // the accumulator may be overwritten by the tile after next
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) mbar_arrive(acc_empty(a));
     }
   }
   if (!ok) {
@@ -417,15 +453,15 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmx, const PrefillArgs p, con
     int zero = 0;
     for (int s = 0; s < stages; ++s) {
       if (issued > s) {
-        const int last_kb = ((issued - 1 - s) / stages) * stages + s;   // last k-block issued on stage s
-        (void)mbar_wait(full_b(s), (last_kb / stages) & 1, &zero);
+        const int last_it = ((issued - 1 - s) / stages) * stages + s;   // last copy issued on stage s
+        (void)mbar_wait(full_b(s), (last_it / stages) & 1, &zero);
       }
     }
   }
   __syncthreads();
   if (warp == 1) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(TOK) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(2 * kAccCols) : "memory");
   }
 }
 
@@ -471,8 +507,9 @@ gwq_status launch(const gwq_packed* P, const void* x, const float* tok_scale, in
   PrefillArgs a;
   a.codes = P->codes; a.scales = P->scales; a.zeros = P->zeros; a.row_ptr = P->S->row_ptr; a.cv = pv->cv; a.sz_t = pv->sz_t;
   a.y = y; a.yd = yd; a.status = pv->dev_status; a.tok_scale = tok_scale; a.N = P->N; a.K = P->K; a.M = M; a.group = P->group;
-  dim3 grid((unsigned)((P->N + kTileN - 1) / kTileN), (unsigned)((M + TOK - 1) / TOK));
-  prefill_kernel<BITS, TOK, BF16><<<grid, cta_threads(TOK), smem, stream>>>(tmx, a, stages);
+  const int ntn = (P->N + kTileN - 1) / kTileN, ntiles = ntn * ((M + TOK - 1) / TOK);
+  const int grid = ntiles < pv->sm_count ? ntiles : pv->sm_count;   // persistent: at most one CTA per SM
+  prefill_kernel<BITS, TOK, BF16><<<grid, kCtaThreads, smem, stream>>>(tmx, a, stages, ntn, ntiles);
   return cudaGetLastError() == cudaSuccess ? GWQ_OK : GWQ_ERR_CUDA;
 }
 
