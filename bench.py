@@ -61,6 +61,29 @@ def algorithmic_bytes(N: int, K: int, bits: int, group: int, nnz: int, M: int, c
     return codes + meta + csr + M * K * 2 + M * N * 2
 
 
+def kernels_per_linear(M: int, K: int) -> int:
+    """Kernels one gwq_linear call launches on the decode path: the product itself, plus the
+    token-major copy of x when M > 1 and the activations are not staged up front (M > 8, or
+    M K too large for 72 KB of staging)."""
+    nchunks = (K // 128 + 7) // 8
+    staged = M <= 8 and nchunks * M * 148 * 16 <= 72 * 1024
+    return 1 if (staged or M == 1) else 2
+
+
+def dominant_kernel_traffic():
+    """(dram bytes / algorithmic bytes) of the decode kernel from the committed ncu capture, or None when
+    the kernel source has changed since the capture was taken."""
+    import hashlib
+    try:
+        rec = json.load(open(os.path.join(ROOT, "profiles", "decode_kernel_traffic.json")))
+        src = open(os.path.join(ROOT, "paper_2411_00850_b200", "csrc", "linear_decode.cu"), "rb").read()
+        if hashlib.sha1(src).hexdigest() != rec["kernel_source_sha1"]:
+            return None
+        return float(rec["dram_bytes_per_launch"]) / float(rec["algorithmic_bytes_per_launch"])
+    except Exception:
+        return None
+
+
 def linear_flops(N: int, K: int, nnz: int, M: int) -> int:
     return 2 * M * (N * K + nnz)
 
@@ -286,7 +309,7 @@ def run_cuda_arm(args):
                    "launch_order": "per (M, bits): q|k|v concurrently, o, gate|up concurrently, down (decoder-block data flow)",
                    "l2": f"{replicas} rotating copies of the packed set ({replicas * step_bytes // 3 / 1e6:.0f} MB) "
                          "exceed the 126 MB L2 between reuses; one CUDA graph per copy"},
-        "gpu_launches": len(cases) * args.steps,
+        "gpu_launches": args.steps * sum(kernels_per_linear(M, layers[li]["K"]) for (li, bits, M) in cases),
         "clocks": clocks,
     }
     if rank != 0:
@@ -303,6 +326,10 @@ def run_cuda_arm(args):
         "frac_of_nominal_8TBs": round(step_bytes / (ms_step * 1e-3) / 1e9 / 8000.0, 4),
         "avg_launch_us": round(ms_step * 1e3 / len(cases), 3), "traffic": None,
     }
+    ratio = dominant_kernel_traffic()
+    if ratio is not None:   # DRAM bytes per launch, averaged like `achieved` (traffic scales with the bytes streamed)
+        out["roofline"]["traffic"] = round(ratio * step_bytes / len(cases))
+        out["roofline"]["traffic_source"] = "profiles/decode_kernel_traffic.json (ncu, 11008x4096 W4 M=1), scaled by algorithmic bytes"
     if world == 1 and not args.headline_only:
         out["decode_cases"] = bench_decode_detail(torch, gwq, layers, xs, ys, detail_iters, hbm_peak)
         out["cublas_fp16"] = bench_dense_library(torch, layers, xs, detail_iters, step_bytes, ms_step)
@@ -314,6 +341,13 @@ def run_cuda_arm(args):
         for L in layers:
             L["W"] = None
         out["prefill"] = bench_prefill(torch, gwq, dev, args, tf_burst, tf_sust)
+        best = max(out["prefill"], key=lambda r: r["tflops"])
+        out["prefill_roofline"] = {"bound": "tensor", "kernel": "gwq prefill linear (tcgen05)",
+                                   "case": f"{best['N']}x{best['K']} W4 g128 1% M={best['M']} bf16 in",
+                                   "achieved": best["tflops"], "peak": tf_burst, "unit": "TFLOP/s",
+                                   "frac": round(best["tflops"] / tf_burst, 4), "peak_source": peak_src,
+                                   "frac_of_sustained": round(best["tflops"] / tf_sust, 4),
+                                   "frac_of_nominal_2250": round(best["tflops"] / 2250.0, 4)}
         out["cpu_baseline"] = cpu_baseline(sample_seconds=args.cpu_seconds)
     else:
         out["e2e"] = bench_e2e(torch, gwq, layers, cases, detail_iters, step_bytes, world)
