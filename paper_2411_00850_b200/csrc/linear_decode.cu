@@ -227,6 +227,7 @@ struct DecodeArgs {
   const uint32_t* cv;  // per outlier: fp16 value << 16 | column
   const uint16_t* x;
   const uint16_t* xt;  // [K][TP] copy of x (ring mode with more than one token), else null
+  const float* xg;     // [K/128][TP] sums of x over each group of columns (same mode), else null
   void* y;
   gwq_dtype yd;
   int N, K, M;
@@ -288,7 +289,9 @@ template <int BITS, int TP, bool BF16, int NBUF>
 __global__ void __launch_bounds__(kThreads, TP <= 8 ? 3 : (TP == 16 ? 2 : 1)) decode_kernel(const DecodeArgs p) {
   constexpr int NB = TP <= 8 ? 1 : TP / 8;   // 8-token blocks of the MMA
   constexpr int WPR = BITS;                   // words per run of 32 columns
-  constexpr bool ONES = !BF16 && TP != 1;     // raw path: sum_k x_k by MMA unless there is one token
+  // raw path: sum_k x_k of a group from shared memory (one token), from the table that comes with the
+  // token-major copy (ring mode), else from a second MMA with an all-ones A operand
+  constexpr bool ONES = !BF16 && TP != 1 && NBUF == 0;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int ngroups = p.K >> 7;
   // shared: zero page 64 B | scales [16][ngroups] f16 | zeros [16][ngroups] u8 | red [kWarps][NB][16][8] f32 |
@@ -365,14 +368,20 @@ __global__ void __launch_bounds__(kThreads, TP <= 8 ? 3 : (TP == 16 ? 2 : 1)) de
   // NBUF == 2: copy of the activations of this warp's step c (group warp + 8 c) into its buffer c & 1
   const int tile_pieces = p.M * kTilePitch;
   uint4* wtile = sm_x + warp * 2 * tile_pieces;
+  // lane L copies piece L & 15 of the token rows (L >> 4), (L >> 4) + 2, ...: constant strides, three
+  // instructions per 16-byte piece
+  const int st_m0 = lane >> 4, st_pc = lane & 15;
+  const unsigned st_dst0 =
+      (unsigned)__cvta_generic_to_shared(wtile + st_m0 * kTilePitch + st_pc + (st_pc >> 3) + ((st_m0 & 1) << 1));
+  const uint16_t* st_src0 = p.x + (size_t)st_m0 * p.K + (size_t)warp * 128 + st_pc * 8;
   auto stage_tile = [&](int c) {
     if (c < nsteps) {
-      const uint16_t* src = p.x + (size_t)(warp + kWarps * c) * 128;
-      uint4* buf = wtile + (c & 1) * tile_pieces;
-      for (int i = lane; i < p.M * 16; i += 32) {
-        const int m = i >> 4, pc = i & 15;
-        const unsigned dst = (unsigned)__cvta_generic_to_shared(buf + m * kTilePitch + pc + (pc >> 3) + ((m & 1) << 1));
-        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src + (size_t)m * p.K + pc * 8));
+      const uint16_t* src = st_src0 + (size_t)c * (kWarps * 128);
+      unsigned dst = st_dst0 + (unsigned)((c & 1) * tile_pieces) * 16u;
+      for (int m = st_m0; m < p.M; m += 2) {
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src));
+        src += 2 * (size_t)p.K;
+        dst += 2 * kTilePitch * 16;
       }
     }
   };
@@ -465,8 +474,11 @@ __global__ void __launch_bounds__(kThreads, TP <= 8 ? 3 : (TP == 16 ? 2 : 1)) de
 
   // one chunk: stage the next one, this warp's group step (register slot D = c % kDepth), the owned
   // rows' outliers of the chunk, then the hand-over barrier
-  auto do_chunk = [&](const int c, auto slot) {
+  // `checked` = false promises c < nsteps (no branch, so that neighbouring steps can be interleaved);
+  // xsum_in carries the single token's group sum when the caller has already reduced it
+  auto do_chunk = [&](const int c, auto slot, auto checked_t, const float xsum_in) {
     constexpr int d = decltype(slot)::value;
+    constexpr bool checked = decltype(checked_t)::value;
     if (NBUF != 0) {   // next step's activations on their way, this step's landed and visible to the warp
       __syncwarp();
       stage_tile(c + 1);
@@ -474,7 +486,7 @@ __global__ void __launch_bounds__(kThreads, TP <= 8 ? 3 : (TP == 16 ? 2 : 1)) de
       __syncwarp();
     }
     const uint4* buf = NBUF == 0 ? sm_x + c * buf_pieces : wtile + (c & 1) * tile_pieces;
-    if (c < nsteps) {
+    if (!checked || c < nsteps) {
       unsigned xr[NB][16];
 #pragma unroll
       for (int nb = 0; nb < NB; ++nb) {
@@ -500,8 +512,16 @@ __global__ void __launch_bounds__(kThreads, TP <= 8 ? 3 : (TP == 16 ? 2 : 1)) de
           tb = make_float2(sb * 16777216.f, sb * (float)zb);
         }
       }
-      float xsum1 = 0.f;
-      if (!BF16 && !ONES) {   // one token: sum_k x_k of the group, lane L adding columns 4L..4L+3
+      float2 xg2[NB];
+#pragma unroll
+      for (int nb = 0; nb < NB; ++nb) xg2[nb] = make_float2(0.f, 0.f);
+      if (!BF16 && !ONES && TP != 1) {   // group sums of tokens 2t, 2t+1 of every token block
+#pragma unroll
+        for (int nb = 0; nb < NB; ++nb)
+          xg2[nb] = __ldg(reinterpret_cast<const float2*>(p.xg + (size_t)(warp + kWarps * c) * TP + nb * 8 + 2 * t));
+      }
+      float xsum1 = xsum_in;
+      if (!BF16 && TP == 1 && checked) {   // one token: sum_k x_k of the group, lane L adding columns 4L..4L+3
         const uint2 h4 = reinterpret_cast<const uint2*>(buf)[xsum_off];
         const float2 f0 = __half22float2(*reinterpret_cast<const __half2*>(&h4.x));
         const float2 f1 = __half22float2(*reinterpret_cast<const __half2*>(&h4.y));
@@ -541,12 +561,14 @@ __global__ void __launch_bounds__(kThreads, TP <= 8 ? 3 : (TP == 16 ? 2 : 1)) de
           } else if (BITS == 4) {
             AccRaw4<NB>& a4 = reinterpret_cast<AccRaw4<NB>&>(acc);
             const float code_sum = fmaf(a4.c4[nb][i], 0.0625f, a4.c0[nb][i]);  // units of 2^-24
-            const float xsum = ONES ? a4.xs[nb][i & 1] : ((i & 1) == 0 && t == 0 ? xsum1 : 0.f);  // token 0 only
+            const float xsum = ONES ? a4.xs[nb][i & 1]
+                                    : (TP == 1 ? ((i & 1) == 0 && t == 0 ? xsum1 : 0.f) : ((i & 1) ? xg2[nb].y : xg2[nb].x));
             yacc[nb][i] = fmaf(tt.x, code_sum, fmaf(-tt.y, xsum, yacc[nb][i]));
           } else {
             AccRaw3<NB>& a3 = reinterpret_cast<AccRaw3<NB>&>(acc);
             const float code_sum = fmaf(a3.c6[nb][i], 0.015625f, fmaf(a3.c3[nb][i], 0.125f, a3.c0[nb][i]));
-            const float xsum = ONES ? a3.xs[nb][i & 1] : ((i & 1) == 0 && t == 0 ? xsum1 : 0.f);  // token 0 only
+            const float xsum = ONES ? a3.xs[nb][i & 1]
+                                    : (TP == 1 ? ((i & 1) == 0 && t == 0 ? xsum1 : 0.f) : ((i & 1) ? xg2[nb].y : xg2[nb].x));
             yacc[nb][i] = fmaf(tt.x, code_sum, fmaf(-tt.y, xsum, yacc[nb][i]));
           }
         }
@@ -554,11 +576,43 @@ __global__ void __launch_bounds__(kThreads, TP <= 8 ? 3 : (TP == 16 ? 2 : 1)) de
     }
 
   };
-  for (int c0 = 0; c0 < nchunks; c0 += kDepth) {   // nchunks is uniform over the CTA: every warp meets every barrier
-    do_chunk(c0, std::integral_constant<int, 0>{});
-    if (c0 + 1 < nchunks) do_chunk(c0 + 1, std::integral_constant<int, 1>{});
-    if (c0 + 2 < nchunks) do_chunk(c0 + 2, std::integral_constant<int, 2>{});
-    if (c0 + 3 < nchunks) do_chunk(c0 + 3, std::integral_constant<int, 3>{});
+  using std::integral_constant;
+  for (int c0 = 0; c0 < nchunks; c0 += kDepth) {
+    if (c0 + kDepth <= nsteps) {
+      // four full steps of this warp: branch-free, the single token's four group sums reduced together
+      float xs4[kDepth] = {0.f, 0.f, 0.f, 0.f};
+      if (!BF16 && TP == 1) {
+#pragma unroll
+        for (int d = 0; d < kDepth; ++d) {
+          const uint4* buf = NBUF == 0 ? sm_x + (c0 + d) * buf_pieces : wtile + ((c0 + d) & 1) * tile_pieces;
+          if (NBUF == 0) {
+            const uint2 h4 = reinterpret_cast<const uint2*>(buf)[xsum_off];
+            const float2 f0 = __half22float2(*reinterpret_cast<const __half2*>(&h4.x));
+            const float2 f1 = __half22float2(*reinterpret_cast<const __half2*>(&h4.y));
+            xs4[d] = (f0.x + f0.y) + (f1.x + f1.y);
+          }
+        }
+        if (NBUF == 0) {
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+            for (int d = 0; d < kDepth; ++d) xs4[d] += __shfl_xor_sync(0xFFFFFFFFu, xs4[d], o);
+        }
+      }
+      if (NBUF == 0) {
+        do_chunk(c0, integral_constant<int, 0>{}, integral_constant<bool, false>{}, xs4[0]);
+        do_chunk(c0 + 1, integral_constant<int, 1>{}, integral_constant<bool, false>{}, xs4[1]);
+        do_chunk(c0 + 2, integral_constant<int, 2>{}, integral_constant<bool, false>{}, xs4[2]);
+        do_chunk(c0 + 3, integral_constant<int, 3>{}, integral_constant<bool, false>{}, xs4[3]);
+        continue;
+      }
+    }
+    // general path (a partial block of steps, or ring mode where the tile of a single token is not yet
+    // there when the block starts)
+    do_chunk(c0, integral_constant<int, 0>{}, integral_constant<bool, true>{}, 0.f);
+    if (c0 + 1 < nchunks) do_chunk(c0 + 1, integral_constant<int, 1>{}, integral_constant<bool, true>{}, 0.f);
+    if (c0 + 2 < nchunks) do_chunk(c0 + 2, integral_constant<int, 2>{}, integral_constant<bool, true>{}, 0.f);
+    if (c0 + 3 < nchunks) do_chunk(c0 + 3, integral_constant<int, 3>{}, integral_constant<bool, true>{}, 0.f);
   }
   static_assert(kDepth == 4, "the chunk loop is written out for four register slots");
 
@@ -626,22 +680,38 @@ __global__ void __launch_bounds__(kThreads, TP <= 8 ? 3 : (TP == 16 ? 2 : 1)) de
   }
 }
 
-// xt[col][token] = x[token][col] for token < M (zero beyond), TP tokens per column.
-template <int TP>
-__global__ void __launch_bounds__(256) tokens_to_columns(const uint16_t* __restrict__ x, uint16_t* __restrict__ xt, int M, int K) {
-  constexpr int PARTS = TP >= 8 ? TP / 8 : 1, W = TP >= 8 ? 8 : TP;
-  const int id = blockIdx.x * 256 + threadIdx.x;
-  const int col = id / PARTS, part = id % PARTS;
-  if (col >= K) return;
-  uint16_t v[W];
+// One CTA per group of 128 columns: xt[col][token] = x[token][col] for token < M (zero beyond), TP tokens
+// per column, and xg[group][token] = sum of x[token][col] over the group's columns (FP32).
+template <int TP, bool BF16>
+__global__ void __launch_bounds__(128) tokens_to_columns(const uint16_t* __restrict__ x, uint16_t* __restrict__ xt,
+                                                         float* __restrict__ xg, int M, int K) {
+  __shared__ float red[4][TP];
+  const int col = blockIdx.x * 128 + threadIdx.x;
+  uint16_t v[TP];
 #pragma unroll
-  for (int i = 0; i < W; ++i) {
-    const int m = part * W + i;
-    v[i] = m < M ? __ldg(x + (size_t)m * K + col) : (uint16_t)0;
+  for (int m = 0; m < TP; ++m) v[m] = m < M ? __ldg(x + (size_t)m * K + col) : (uint16_t)0;
+  if (TP % 8 == 0) {
+#pragma unroll
+    for (int q = 0; q < TP / 8; ++q) {
+      uint4 o;
+      o.x = v[8 * q] | ((unsigned)v[8 * q + 1] << 16);     o.y = v[8 * q + 2] | ((unsigned)v[8 * q + 3] << 16);
+      o.z = v[8 * q + 4] | ((unsigned)v[8 * q + 5] << 16); o.w = v[8 * q + 6] | ((unsigned)v[8 * q + 7] << 16);
+      reinterpret_cast<uint4*>(xt + (size_t)col * TP)[q] = o;
+    }
+  } else {
+#pragma unroll
+    for (int m = 0; m < TP; ++m) xt[(size_t)col * TP + m] = v[m];
   }
-  uint16_t* dst = xt + (size_t)col * TP + part * W;
 #pragma unroll
-  for (int i = 0; i < W; ++i) dst[i] = v[i];
+  for (int m = 0; m < TP; ++m) {
+    float f = act_to_float<BF16>(v[m]);
+    for (int o = 16; o > 0; o >>= 1) f += __shfl_xor_sync(0xFFFFFFFFu, f, o);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5][m] = f;
+  }
+  __syncthreads();
+  if (threadIdx.x < TP)
+    xg[(size_t)blockIdx.x * TP + threadIdx.x] =
+        (red[0][threadIdx.x] + red[1][threadIdx.x]) + (red[2][threadIdx.x] + red[3][threadIdx.x]);
 }
 
 constexpr size_t kStageAllLimit = 72 * 1024;   // stage every chunk up front when it fits in this much
@@ -677,8 +747,8 @@ cudaError_t launch_buf(const DecodeArgs& a, cudaStream_t stream) {
   const int nchunks = (a.K / 128 + kChunkGroups - 1) / kChunkGroups;
   if (TP <= 8 && (size_t)nchunks * a.M * kRowPitch * 16 <= kStageAllLimit) return launch<BITS, TP, BF16, 0>(a, stream);
   if (TP > 1) {   // ring mode gathers the outliers' activations from a token-major copy
-    if (!a.xt) return cudaErrorInvalidValue;
-    tokens_to_columns<TP><<<(a.K * (TP >= 8 ? TP / 8 : 1) + 255) / 256, 256, 0, stream>>>(a.x, const_cast<uint16_t*>(a.xt), a.M, a.K);
+    if (!a.xt || !a.xg) return cudaErrorInvalidValue;
+    tokens_to_columns<TP, BF16><<<a.K / 128, 128, 0, stream>>>(a.x, const_cast<uint16_t*>(a.xt), const_cast<float*>(a.xg), a.M, a.K);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
   }
@@ -703,8 +773,9 @@ gwq_status gwq_launch_decode(const gwq_packed* P, const void* x, gwq_dtype xd, i
   if (P->group != 128 || M > 32 || !pv->cv) return gwq_launch_simt(P, x, xd, M, y, yd, stream);
   DecodeArgs a;
   a.xt = nullptr;
-  if (M > 1) {   // scratch for the token-major copy (used when the activations are not staged up front)
-    const size_t need = (size_t)P->K * 32 * 2;
+  a.xg = nullptr;
+  if (M > 1) {   // scratch for the token-major copy and the group sums (used when x is not staged up front)
+    const size_t need = (size_t)P->K * 32 * 2 + (size_t)(P->K / 128) * 32 * 4;
     if (pv->xt_bytes < need) {
       if (cudaStreamSynchronize(stream) != cudaSuccess) return GWQ_ERR_CUDA;
       if (pv->xt) cudaFree(pv->xt);
@@ -717,6 +788,7 @@ gwq_status gwq_launch_decode(const gwq_packed* P, const void* x, gwq_dtype xd, i
       pv->xt_bytes = need;
     }
     a.xt = static_cast<const uint16_t*>(pv->xt);
+    a.xg = reinterpret_cast<const float*>(static_cast<const char*>(pv->xt) + (size_t)P->K * 32 * 2);
   }
   a.codes = P->codes; a.scales = P->scales; a.zeros = P->zeros;
   a.row_ptr = P->S->row_ptr; a.cv = pv->cv;
