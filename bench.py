@@ -38,6 +38,8 @@ BIT_WIDTHS = (4, 3)
 GROUP = 128
 FRAC = 0.01
 CONFIG_INDEX = 1
+# layers of the set (by index) in decoder-block data-flow order: q|k|v read the same x, then o, gate|up, down
+STAGES = ((0, 1, 2), (3,), (4, 5), (6,))
 PREFILL_SHAPES = ((11008, 4096), (4096, 11008))
 PREFILL_MS = (512, 2048, 8192)
 
@@ -253,6 +255,11 @@ def run_cuda_arm(args):
           for (li, bits, M) in cases}
 
     side = [torch.cuda.Stream(device=dev) for _ in range(2)]
+    fuse = not args.no_fuse
+    # kernel launches of one step: one call per stage when the siblings are fused, else one per layer
+    calls = [(lis if not fuse else lis[:1], M) for M in DECODE_MS for _b in BIT_WIDTHS for lis in STAGES]
+    launches_per_step = sum(kernels_per_linear(M, layers[li]["K"]) for (lis, M) in calls for li in lis)
+    calls_per_step = sum(len(lis) for (lis, M) in calls)
 
     def step_fn(rep):
         """The 7 linears of a decoder block in their data-flow order: q, k, v side by side, then o,
@@ -261,21 +268,23 @@ def run_cuda_arm(args):
             main = torch.cuda.current_stream()
 
             def stage(lis, bits, M):
+                if len(lis) > 1 and fuse:   # sibling projections read the same activations: one call, one launch
+                    gwq.gwq_linear_multi([layers[li]["packed"][bits][rep] for li in lis], xs[(lis[0], M)],
+                                         outs=[ys[(li, bits, M)] for li in lis])
+                    return
                 if len(lis) > 1:
                     for s_ in side[:len(lis) - 1]:
                         s_.wait_stream(main)
                 for k, li in enumerate(lis):
                     with torch.cuda.stream(main if k == 0 else side[k - 1]):
-                        gwq.gwq_linear(layers[li]["packed"][bits][rep], xs[(li, M)], out=ys[(li, bits, M)])
+                        gwq.gwq_linear(layers[li]["packed"][bits][rep], xs[(lis[0], M)], out=ys[(li, bits, M)])
                 if len(lis) > 1:
                     for s_ in side[:len(lis) - 1]:
                         main.wait_stream(s_)
             for M in DECODE_MS:
                 for bits in BIT_WIDTHS:
-                    stage([0, 1, 2], bits, M)
-                    stage([3], bits, M)
-                    stage([4, 5], bits, M)
-                    stage([6], bits, M)
+                    for lis in STAGES:
+                        stage(lis, bits, M)
         return run
 
     graphs = [capture(torch, step_fn(r)) for r in range(replicas)]
@@ -305,11 +314,14 @@ def run_cuda_arm(args):
         "vs_baseline": None, "dtype": "f16 x int4/int3 -> f32 accumulate", "data": "synthetic",
         "config": {"workload": WORKLOAD, "layers": [f"{n}:{N}x{K}" for n, N, K in synth.LLAMA7B_LAYER_SET],
                    "bits": list(BIT_WIDTHS), "group": GROUP, "outlier_frac": FRAC, "M": list(DECODE_MS),
-                   "launches_per_step": len(cases), "step_bytes": step_bytes,
-                   "launch_order": "per (M, bits): q|k|v concurrently, o, gate|up concurrently, down (decoder-block data flow)",
+                   "products_per_step": len(cases), "calls_per_step": calls_per_step,
+                   "kernel_launches_per_step": launches_per_step, "step_bytes": step_bytes, "fused_siblings": fuse,
+                   "launch_order": ("per (M, bits): q|k|v as one gwq_linear_multi launch, o, gate|up as one launch, down "
+                                    "(decoder-block data flow)") if fuse else
+                                   "per (M, bits): q|k|v concurrently, o, gate|up concurrently, down (decoder-block data flow)",
                    "l2": f"{replicas} rotating copies of the packed set ({replicas * step_bytes // 3 / 1e6:.0f} MB) "
                          "exceed the 126 MB L2 between reuses; one CUDA graph per copy"},
-        "gpu_launches": args.steps * sum(kernels_per_linear(M, layers[li]["K"]) for (li, bits, M) in cases),
+        "gpu_launches": args.steps * launches_per_step,
         "clocks": clocks,
     }
     if rank != 0:
@@ -320,15 +332,15 @@ def run_cuda_arm(args):
     # ---- everything below: rank 0 only, N = 1 detail
     detail_iters = max(5, min(args.steps, 20))
     out["roofline"] = {
-        "bound": "hbm", "kernel": "gwq decode linear (all 42 launches of the step)",
+        "bound": "hbm", "kernel": f"gwq decode linear (all {calls_per_step} calls = {len(cases)} products of the step)",
         "achieved": round(step_bytes / (ms_step * 1e-3) / 1e9, 1), "peak": hbm_peak, "unit": "GB/s",
         "frac": round(step_bytes / (ms_step * 1e-3) / 1e9 / hbm_peak, 4), "peak_source": peak_src,
         "frac_of_nominal_8TBs": round(step_bytes / (ms_step * 1e-3) / 1e9 / 8000.0, 4),
-        "avg_launch_us": round(ms_step * 1e3 / len(cases), 3), "traffic": None,
+        "avg_launch_us": round(ms_step * 1e3 / calls_per_step, 3), "traffic": None,
     }
     ratio = dominant_kernel_traffic()
     if ratio is not None:   # DRAM bytes per launch, averaged like `achieved` (traffic scales with the bytes streamed)
-        out["roofline"]["traffic"] = round(ratio * step_bytes / len(cases))
+        out["roofline"]["traffic"] = round(ratio * step_bytes / calls_per_step)
         out["roofline"]["traffic_source"] = "profiles/decode_kernel_traffic.json (ncu, 11008x4096 W4 M=1), scaled by algorithmic bytes"
     if world == 1 and not args.headline_only:
         out["decode_cases"] = bench_decode_detail(torch, gwq, layers, xs, ys, detail_iters, hbm_peak)
@@ -539,6 +551,8 @@ def main():
     ap.add_argument("--prefill-iters", type=int, default=5)
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--headline-only", action="store_true", help="skip the per-case detail sections")
+    ap.add_argument("--no-fuse", action="store_true",
+                    help="launch sibling projections as separate concurrent calls instead of one gwq_linear_multi")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     out = run_reference_arm(args) if args.impl == "reference" else run_cuda_arm(args)

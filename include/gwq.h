@@ -137,6 +137,20 @@ gwq_status gwq_pack(const uint16_t* W_f16, gwq_outliers* S, int32_t N, int32_t K
 gwq_status gwq_linear(const gwq_packed* P, const void* x, gwq_dtype x_dtype, int32_t M, void* y,
                       gwq_dtype y_dtype, void* stream);
 
+/* Several forward products that read the same activations, in one call: y[i] = x (deq(P[i]) + S_i)^T for
+ * i < count.  This is launch-level fusion of sibling projections (q | k | v, or gate | up, of a decoder
+ * block: Section 4.5 measures whole-model generation, where these run back to back); each product is
+ * exactly the one gwq_linear computes, bit for bit.
+ *   P: host array of `count` packed layers (1 <= count <= GWQ_MULTI_MAX) with the same K.
+ *   x: device [M, K]; y: host array of `count` device pointers, y[i] is [M, P[i]->N], all of y_dtype.
+ *   With M <= 32, group 128 and one bit width for all layers, the products run as ONE kernel launch
+ *   (layer 0 lends its scratch: do not overlap with another call that uses P[0]); otherwise the call is
+ *   the same as `count` calls of gwq_linear in order.  Asynchronous on `stream`.
+ * Errors: INVALID_ARG (count, null entries, differing K, alignment), otherwise as gwq_linear.          */
+#define GWQ_MULTI_MAX 4
+gwq_status gwq_linear_multi(const gwq_packed* const* P, int32_t count, const void* x, gwq_dtype x_dtype,
+                            int32_t M, void* const* y, gwq_dtype y_dtype, void* stream);
+
 /* Same product with HOST buffers: copies x_host [M,K] to a staging buffer kept inside P,
  * runs gwq_linear, copies y back into y_host [M,N] and synchronises `stream`.
  * For best copy speed the host buffers should be page-locked.  The staging buffers grow

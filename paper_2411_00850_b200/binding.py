@@ -16,13 +16,16 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libgwq.so")
 
 GWQ_OK = 0
+(GWQ_ERR_INVALID_ARG, GWQ_ERR_UNSUPPORTED, GWQ_ERR_ALLOC, GWQ_ERR_NONFINITE, GWQ_ERR_TIMEOUT,
+ GWQ_ERR_CUDA) = range(1, 7)
 GWQ_F16, GWQ_BF16, GWQ_F32 = 0, 1, 2
 STATUS_NAMES = {
     0: "GWQ_OK", 1: "GWQ_ERR_INVALID_ARG", 2: "GWQ_ERR_UNSUPPORTED", 3: "GWQ_ERR_ALLOC",
     4: "GWQ_ERR_NONFINITE", 5: "GWQ_ERR_TIMEOUT", 6: "GWQ_ERR_CUDA",
 }
-EXPORTS = ("gwq_select_outliers", "gwq_select_outliers_static", "gwq_pack", "gwq_linear", "gwq_linear_host", "gwq_device_status", "gwq_free",
-           "gwq_status_string")
+EXPORTS = ("gwq_select_outliers", "gwq_select_outliers_static", "gwq_pack", "gwq_linear", "gwq_linear_multi",
+           "gwq_linear_host", "gwq_device_status", "gwq_free", "gwq_status_string")
+GWQ_MULTI_MAX = 4
 
 
 class GwqError(RuntimeError):
@@ -67,6 +70,9 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     lib.gwq_linear.restype = C.c_int
     lib.gwq_linear.argtypes = [C.POINTER(gwq_packed), C.c_void_p, C.c_int, C.c_int32, C.c_void_p, C.c_int,
                                C.c_void_p]
+    lib.gwq_linear_multi.restype = C.c_int
+    lib.gwq_linear_multi.argtypes = [C.POINTER(C.POINTER(gwq_packed)), C.c_int32, C.c_void_p, C.c_int, C.c_int32,
+                                     C.POINTER(C.c_void_p), C.c_int, C.c_void_p]
     lib.gwq_linear_host.restype = C.c_int
     lib.gwq_linear_host.argtypes = lib.gwq_linear.argtypes
     lib.gwq_device_status.restype = C.c_int
@@ -289,6 +295,28 @@ def gwq_linear(P: Packed, x: torch.Tensor, out_dtype: torch.dtype | None = None,
                         _stream_ptr())
     _check(st, "gwq_linear")
     return out
+
+
+def gwq_linear_multi(Ps, x: torch.Tensor, out_dtype: torch.dtype | None = None, outs=None):
+    """[x (deq(P) + S_P)^T for P in Ps] for layers that read the same x [M,K]: one call, and for M <= 32 one launch."""
+    lib = load_library()
+    _require_cuda(x, "x")
+    n = len(Ps)
+    if x.dim() != 2 or any(P.K != x.shape[1] for P in Ps):
+        raise ValueError("x must be [M, K] with the K of every layer")
+    M = x.shape[0]
+    if outs is None:
+        outs = [torch.empty((M, P.N), dtype=out_dtype or x.dtype, device=x.device) for P in Ps]
+    for o in outs:
+        _require_cuda(o, "out")
+    if len(outs) != n or any(o.dtype != outs[0].dtype for o in outs):
+        raise ValueError("one output per layer, all of one dtype")
+    handles = (C.POINTER(gwq_packed) * max(n, 1))(*[P._h for P in Ps])
+    ys = (C.c_void_p * max(n, 1))(*[o.data_ptr() for o in outs])
+    st = lib.gwq_linear_multi(handles, n, x.data_ptr(), _dtype_code(x.dtype), M, ys,
+                              _dtype_code(outs[0].dtype) if outs else GWQ_F16, _stream_ptr())
+    _check(st, "gwq_linear_multi")
+    return outs
 
 
 def gwq_linear_host(P: Packed, x_host: torch.Tensor, y_host: torch.Tensor) -> torch.Tensor:

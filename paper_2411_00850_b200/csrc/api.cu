@@ -19,6 +19,29 @@ extern "C" gwq_status gwq_linear(const gwq_packed* P, const void* x, gwq_dtype x
   return gwq_launch_prefill(P, x, xd, M, y, yd, stream);
 }
 
+extern "C" gwq_status gwq_linear_multi(const gwq_packed* const* P, int32_t count, const void* x, gwq_dtype xd,
+                                       int32_t M, void* const* y, gwq_dtype yd, void* stream_) {
+  if (!P || !y || !x || count < 1 || count > GWQ_MULTI_MAX || M <= 0) return GWQ_ERR_INVALID_ARG;
+  if (xd != GWQ_F16 && xd != GWQ_BF16) return GWQ_ERR_UNSUPPORTED;
+  if (yd != GWQ_F16 && yd != GWQ_BF16 && yd != GWQ_F32) return GWQ_ERR_INVALID_ARG;
+  if (!gwq_aligned16(x)) return GWQ_ERR_INVALID_ARG;
+  for (int i = 0; i < count; ++i) {
+    if (!P[i] || P[i]->tag != GWQ_TAG_PACKED || !P[i]->S || !P[i]->priv || !y[i] || !gwq_aligned16(y[i]))
+      return GWQ_ERR_INVALID_ARG;
+    if (P[i]->K != P[0]->K) return GWQ_ERR_INVALID_ARG;
+  }
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  if (M <= GWQ_DECODE_MAX_M) {
+    const gwq_status st = gwq_launch_decode_multi(P, count, x, xd, M, y, yd, stream);
+    if (st != GWQ_ERR_UNSUPPORTED) return st;
+  }
+  for (int i = 0; i < count; ++i) {
+    const gwq_status st = gwq_linear(P[i], x, xd, M, y[i], yd, stream_);
+    if (st != GWQ_OK) return st;
+  }
+  return GWQ_OK;
+}
+
 extern "C" gwq_status gwq_linear_host(gwq_packed* P, const void* x_host, gwq_dtype xd, int32_t M,
                                       void* y_host, gwq_dtype yd, void* stream_) {
   if (!P || P->tag != GWQ_TAG_PACKED || !P->priv || !x_host || !y_host || M <= 0) return GWQ_ERR_INVALID_ARG;

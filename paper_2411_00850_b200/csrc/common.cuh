@@ -47,5 +47,7 @@ gwq_status gwq_launch_simt(const gwq_packed* P, const void* x, gwq_dtype xd, int
                            gwq_dtype yd, cudaStream_t stream);
 gwq_status gwq_launch_decode(const gwq_packed* P, const void* x, gwq_dtype xd, int M, void* y,
                              gwq_dtype yd, cudaStream_t stream);
+gwq_status gwq_launch_decode_multi(const gwq_packed* const* P, int count, const void* x, gwq_dtype xd, int M,
+                                   void* const* y, gwq_dtype yd, cudaStream_t stream);
 gwq_status gwq_launch_prefill(const gwq_packed* P, const void* x, gwq_dtype xd, int M, void* y,
                               gwq_dtype yd, cudaStream_t stream);

@@ -233,6 +233,29 @@ struct DecodeArgs {
   int N, K, M;
 };
 
+// One launch may serve several layers that read the same activations (sibling projections): the grid is the
+// concatenation of the layers' row blocks, layer l owning the blocks [first_block[l], first_block[l + 1]).
+constexpr int kMaxLayers = GWQ_MULTI_MAX;
+struct LayerArgs {
+  const uint32_t* codes;
+  const uint16_t* scales;
+  const uint8_t* zeros;
+  const int32_t* row_ptr;
+  const uint32_t* cv;
+  void* y;
+  int N;
+};
+struct MultiArgs {
+  LayerArgs layer[kMaxLayers];
+  int first_block[kMaxLayers + 1];
+  int count;
+  const uint16_t* x;
+  const uint16_t* xt;
+  const float* xg;
+  gwq_dtype yd;
+  int K, M;
+};
+
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
@@ -286,7 +309,25 @@ template <int BITS, int NB> struct StepAcc<BITS, NB, true> { using type = AccSub
 //           (M x 128 columns), copied one step ahead with cp.async; no CTA barrier in the K loop.
 constexpr int kTilePitch = 16 + 2 + 2;   // pieces per token row of a warp tile (same padding rule)
 template <int BITS, int TP, bool BF16, int NBUF>
-__global__ void __launch_bounds__(kThreads, TP <= 8 ? 3 : (TP == 16 ? 2 : 1)) decode_kernel(const DecodeArgs p) {
+__global__ void __launch_bounds__(kThreads, TP <= 8 ? 3 : (TP == 16 ? 2 : 1)) decode_kernel(const MultiArgs ma) {
+  // the layer this CTA works for and its row block inside that layer
+  DecodeArgs p;
+  int blk = blockIdx.x;
+  {
+    int l = 0;
+#pragma unroll
+    for (int i = 1; i < kMaxLayers; ++i)
+      if (i < ma.count && (int)blockIdx.x >= ma.first_block[i]) l = i;
+#pragma unroll
+    for (int i = 0; i < kMaxLayers; ++i) {
+      if (i == l) {
+        p.codes = ma.layer[i].codes; p.scales = ma.layer[i].scales; p.zeros = ma.layer[i].zeros;
+        p.row_ptr = ma.layer[i].row_ptr; p.cv = ma.layer[i].cv; p.y = ma.layer[i].y; p.N = ma.layer[i].N;
+        blk = (int)blockIdx.x - ma.first_block[i];
+      }
+    }
+    p.x = ma.x; p.xt = ma.xt; p.xg = ma.xg; p.yd = ma.yd; p.K = ma.K; p.M = ma.M;
+  }
   constexpr int NB = TP <= 8 ? 1 : TP / 8;   // 8-token blocks of the MMA
   constexpr int WPR = BITS;                   // words per run of 32 columns
   // raw path: sum_k x_k of a group from shared memory (one token), from the table that comes with the
@@ -305,7 +346,7 @@ __global__ void __launch_bounds__(kThreads, TP <= 8 ? 3 : (TP == 16 ? 2 : 1)) de
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int gid = lane >> 2, t = lane & 3;
-  const int r0 = blockIdx.x * kRows;
+  const int r0 = blk * kRows;
   const int ra = min(r0 + gid, p.N - 1), rb = min(r0 + gid + 8, p.N - 1);
   const unsigned row_words = (unsigned)(p.K >> 5) * WPR;
   constexpr unsigned kStepWords = kWarps * 4 * WPR;  // codes of 8 groups
@@ -717,7 +758,7 @@ __global__ void __launch_bounds__(128) tokens_to_columns(const uint16_t* __restr
 constexpr size_t kStageAllLimit = 72 * 1024;   // stage every chunk up front when it fits in this much
 
 template <int BITS, int TP, bool BF16, int NBUF>
-cudaError_t launch(const DecodeArgs& a, cudaStream_t stream) {
+cudaError_t launch(const MultiArgs& a, cudaStream_t stream) {
   constexpr int NB = TP <= 8 ? 1 : TP / 8;
   const int ngroups = a.K / 128;
   const int nchunks = (ngroups + kChunkGroups - 1) / kChunkGroups;
@@ -729,7 +770,7 @@ cudaError_t launch(const DecodeArgs& a, cudaStream_t stream) {
     if (e != cudaSuccess) return e;
   }
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)((a.N + kRows - 1) / kRows));
+  cfg.gridDim = dim3((unsigned)a.first_block[a.count]);
   cfg.blockDim = dim3(kThreads);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = stream;
@@ -743,7 +784,7 @@ cudaError_t launch(const DecodeArgs& a, cudaStream_t stream) {
 
 // ring depth used when the activations do not fit up front
 template <int BITS, int TP, bool BF16, int RING>
-cudaError_t launch_buf(const DecodeArgs& a, cudaStream_t stream) {
+cudaError_t launch_buf(const MultiArgs& a, cudaStream_t stream) {
   const int nchunks = (a.K / 128 + kChunkGroups - 1) / kChunkGroups;
   if (TP <= 8 && (size_t)nchunks * a.M * kRowPitch * 16 <= kStageAllLimit) return launch<BITS, TP, BF16, 0>(a, stream);
   if (TP > 1) {   // ring mode gathers the outliers' activations from a token-major copy
@@ -756,7 +797,7 @@ cudaError_t launch_buf(const DecodeArgs& a, cudaStream_t stream) {
 }
 
 template <int BITS, bool BF16>
-cudaError_t launch_tp(const DecodeArgs& a, cudaStream_t stream) {
+cudaError_t launch_tp(const MultiArgs& a, cudaStream_t stream) {
   if (a.M == 1) return launch_buf<BITS, 1, BF16, 2>(a, stream);
   if (a.M <= 4) return launch_buf<BITS, 4, BF16, 2>(a, stream);
   if (a.M <= 8) return launch_buf<BITS, 8, BF16, 2>(a, stream);
@@ -766,16 +807,23 @@ cudaError_t launch_tp(const DecodeArgs& a, cudaStream_t stream) {
 
 }  // namespace
 
-// Decode launcher: group size 128, M <= 32, K <= 65536.  Other shapes go to the general kernel.
-gwq_status gwq_launch_decode(const gwq_packed* P, const void* x, gwq_dtype xd, int M, void* y, gwq_dtype yd,
-                             cudaStream_t stream) {
-  gwq_priv* pv = static_cast<gwq_priv*>(P->priv);
-  if (P->group != 128 || M > 32 || !pv->cv) return gwq_launch_simt(P, x, xd, M, y, yd, stream);
-  DecodeArgs a;
+// Decode launcher for `count` layers that read the same x: group size 128, M <= 32, K <= 65536, same K and bit
+// width in every layer.  Returns GWQ_ERR_UNSUPPORTED for anything else (nothing has been launched then).
+// The scratch for the token-major copy of x is the first layer's.
+gwq_status gwq_launch_decode_multi(const gwq_packed* const* P, int count, const void* x, gwq_dtype xd, int M,
+                                   void* const* y, gwq_dtype yd, cudaStream_t stream) {
+  if (count < 1 || count > kMaxLayers || M > 32) return GWQ_ERR_UNSUPPORTED;
+  for (int i = 0; i < count; ++i) {
+    const gwq_priv* pvi = static_cast<const gwq_priv*>(P[i]->priv);
+    if (P[i]->group != 128 || !pvi->cv || P[i]->K != P[0]->K || P[i]->bits != P[0]->bits) return GWQ_ERR_UNSUPPORTED;
+  }
+  gwq_priv* pv = static_cast<gwq_priv*>(P[0]->priv);
+  MultiArgs a;
   a.xt = nullptr;
   a.xg = nullptr;
+  const int K = P[0]->K;
   if (M > 1) {   // scratch for the token-major copy and the group sums (used when x is not staged up front)
-    const size_t need = (size_t)P->K * 32 * 2 + (size_t)(P->K / 128) * 32 * 4;
+    const size_t need = (size_t)K * 32 * 2 + (size_t)(K / 128) * 32 * 4;
     if (pv->xt_bytes < need) {
       if (cudaStreamSynchronize(stream) != cudaSuccess) return GWQ_ERR_CUDA;
       if (pv->xt) cudaFree(pv->xt);
@@ -788,18 +836,35 @@ gwq_status gwq_launch_decode(const gwq_packed* P, const void* x, gwq_dtype xd, i
       pv->xt_bytes = need;
     }
     a.xt = static_cast<const uint16_t*>(pv->xt);
-    a.xg = reinterpret_cast<const float*>(static_cast<const char*>(pv->xt) + (size_t)P->K * 32 * 2);
+    a.xg = reinterpret_cast<const float*>(static_cast<const char*>(pv->xt) + (size_t)K * 32 * 2);
   }
-  a.codes = P->codes; a.scales = P->scales; a.zeros = P->zeros;
-  a.row_ptr = P->S->row_ptr; a.cv = pv->cv;
-  a.x = static_cast<const uint16_t*>(x); a.y = y; a.yd = yd;
-  a.N = P->N; a.K = P->K; a.M = M;
+  int blocks = 0;
+  for (int i = 0; i < kMaxLayers; ++i) {
+    const gwq_packed* Pi = P[i < count ? i : 0];
+    a.layer[i].codes = Pi->codes; a.layer[i].scales = Pi->scales; a.layer[i].zeros = Pi->zeros;
+    a.layer[i].row_ptr = Pi->S->row_ptr; a.layer[i].cv = static_cast<const gwq_priv*>(Pi->priv)->cv;
+    a.layer[i].y = y[i < count ? i : 0]; a.layer[i].N = Pi->N;
+    a.first_block[i] = blocks;
+    if (i < count) blocks += (Pi->N + kRows - 1) / kRows;
+  }
+  a.first_block[kMaxLayers] = blocks;
+  for (int i = count; i < kMaxLayers; ++i) a.first_block[i] = blocks;
+  a.count = count;
+  a.x = static_cast<const uint16_t*>(x); a.yd = yd; a.K = K; a.M = M;
   cudaError_t e;
-  if (P->bits == 4) e = (xd == GWQ_BF16) ? launch_tp<4, true>(a, stream) : launch_tp<4, false>(a, stream);
+  if (P[0]->bits == 4) e = (xd == GWQ_BF16) ? launch_tp<4, true>(a, stream) : launch_tp<4, false>(a, stream);
   else e = (xd == GWQ_BF16) ? launch_tp<3, true>(a, stream) : launch_tp<3, false>(a, stream);
   if (e != cudaSuccess) {
     (void)cudaGetLastError();
     return GWQ_ERR_CUDA;
   }
   return GWQ_OK;
+}
+
+// Decode launcher: group size 128, M <= 32, K <= 65536.  Other shapes go to the general kernel.
+gwq_status gwq_launch_decode(const gwq_packed* P, const void* x, gwq_dtype xd, int M, void* y, gwq_dtype yd,
+                             cudaStream_t stream) {
+  const gwq_status st = gwq_launch_decode_multi(&P, 1, x, xd, M, &y, yd, stream);
+  if (st != GWQ_ERR_UNSUPPORTED) return st;
+  return gwq_launch_simt(P, x, xd, M, y, yd, stream);
 }
