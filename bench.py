@@ -370,16 +370,34 @@ def run_cuda_arm(args):
 
 def bench_decode_detail(torch, gwq, layers, xs, ys, iters, hbm_peak):
     """Per (shape, bits, M): microseconds per launch with a cold L2 (the launches of one graph
-    cycle through the layers of equal shape in both copies and a 256 MB scrub precedes every timing)."""
+    cycle through the layers of equal shape in both copies and a 256 MB read-only scrub precedes every timing).
+    `read_only_launch_us` is the same loop with a kernel that only reads the layer's packed arrays: the
+    floor of a one-launch-per-layer product (launch, ramp-up and drain included)."""
     rows = []
-    scrub = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=xs[(0, 1)].device)
+    # L2 scrub: READ 256 MB, so that the cache is left full of clean lines (a written scrub would leave dirty
+    # lines whose write-back competes with the timed reads)
+    scrub = torch.zeros(64 * 1024 * 1024, dtype=torch.int32, device=xs[(0, 1)].device)
+
+    def scrub_l2():
+        return int(scrub.sum().item())
     shapes = {}
     for li, L in enumerate(layers):
         shapes.setdefault((L["N"], L["K"]), []).append(li)
     for (N, K), lis in shapes.items():
         for bits in BIT_WIDTHS:
+            members = [(li, r) for r in range(len(layers[lis[0]]["packed"][bits])) for li in lis]
+
+            def probe():
+                for (li, r) in members:
+                    gwq.gwq_read_probe(layers[li]["packed"][bits][r])
+            replay_probe = capture(torch, probe)
+            floor_ms = None
+            for _ in range(iters):
+                scrub_l2()
+                ms = time_region(torch, lambda i: replay_probe(), 1)
+                floor_ms = ms if floor_ms is None else min(floor_ms, ms)
+            floor_us = floor_ms * 1e3 / len(members)
             for M in DECODE_MS:
-                members = [(li, r) for r in range(len(layers[lis[0]]["packed"][bits])) for li in lis]
 
                 def run():
                     for (li, r) in members:
@@ -387,7 +405,7 @@ def bench_decode_detail(torch, gwq, layers, xs, ys, iters, hbm_peak):
                 replay = capture(torch, run)
                 best = None
                 for _ in range(iters):
-                    scrub.fill_(1)
+                    scrub_l2()
                     ms = time_region(torch, lambda i: replay(), 1)
                     best = ms if best is None else min(best, ms)
                 us = best * 1e3 / len(members)
@@ -395,7 +413,8 @@ def bench_decode_detail(torch, gwq, layers, xs, ys, iters, hbm_peak):
                 b = algorithmic_bytes(N, K, bits, GROUP, nnz, M)
                 rows.append({"N": N, "K": K, "bits": bits, "M": M, "us": round(us, 3), "bytes": b,
                              "gbs": round(b / us / 1e3, 1), "frac_measured_peak": round(b / us / 1e3 / hbm_peak, 4),
-                             "frac_8TBs": round(b / us / 1e3 / 8000.0, 4), "launches_in_graph": len(members)})
+                             "frac_8TBs": round(b / us / 1e3 / 8000.0, 4), "launches_in_graph": len(members),
+                             "read_only_launch_us": round(floor_us, 3), "x_read_only": round(us / floor_us, 2)})
     del scrub
     return rows
 

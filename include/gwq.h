@@ -151,6 +151,13 @@ gwq_status gwq_linear(const gwq_packed* P, const void* x, gwq_dtype x_dtype, int
 gwq_status gwq_linear_multi(const gwq_packed* const* P, int32_t count, const void* x, gwq_dtype x_dtype,
                             int32_t M, void* const* y, gwq_dtype y_dtype, void* stream);
 
+/* Measurement aid, no counterpart in the paper: one launch that reads, and only reads, the arrays a
+ * one-token gwq_linear reads of P (packed codes, scales, zero-points, CSR row pointers, outlier entries).
+ * Its duration is the floor for any forward product that is one kernel launch per layer; the benchmark
+ * prints it beside the decode timings.  *bytes_read (host, may be NULL) receives the bytes it reads.
+ * Asynchronous on `stream`.  Errors: INVALID_ARG, UNSUPPORTED (K > 65536), CUDA.                       */
+gwq_status gwq_read_probe(const gwq_packed* P, int64_t* bytes_read, void* stream);
+
 /* Same product with HOST buffers: copies x_host [M,K] to a staging buffer kept inside P,
  * runs gwq_linear, copies y back into y_host [M,N] and synchronises `stream`.
  * For best copy speed the host buffers should be page-locked.  The staging buffers grow

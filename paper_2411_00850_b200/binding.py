@@ -24,7 +24,7 @@ STATUS_NAMES = {
     4: "GWQ_ERR_NONFINITE", 5: "GWQ_ERR_TIMEOUT", 6: "GWQ_ERR_CUDA",
 }
 EXPORTS = ("gwq_select_outliers", "gwq_select_outliers_static", "gwq_pack", "gwq_linear", "gwq_linear_multi",
-           "gwq_linear_host", "gwq_device_status", "gwq_free", "gwq_status_string")
+           "gwq_read_probe", "gwq_linear_host", "gwq_device_status", "gwq_free", "gwq_status_string")
 GWQ_MULTI_MAX = 4
 
 
@@ -73,6 +73,8 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     lib.gwq_linear_multi.restype = C.c_int
     lib.gwq_linear_multi.argtypes = [C.POINTER(C.POINTER(gwq_packed)), C.c_int32, C.c_void_p, C.c_int, C.c_int32,
                                      C.POINTER(C.c_void_p), C.c_int, C.c_void_p]
+    lib.gwq_read_probe.restype = C.c_int
+    lib.gwq_read_probe.argtypes = [C.POINTER(gwq_packed), C.POINTER(C.c_int64), C.c_void_p]
     lib.gwq_linear_host.restype = C.c_int
     lib.gwq_linear_host.argtypes = lib.gwq_linear.argtypes
     lib.gwq_device_status.restype = C.c_int
@@ -317,6 +319,15 @@ def gwq_linear_multi(Ps, x: torch.Tensor, out_dtype: torch.dtype | None = None, 
                               _dtype_code(outs[0].dtype) if outs else GWQ_F16, _stream_ptr())
     _check(st, "gwq_linear_multi")
     return outs
+
+
+def gwq_read_probe(P: Packed) -> int:
+    """Launch the read-only probe on P (asynchronous on the current stream); returns the bytes it reads."""
+    n = C.c_int64(0)
+    with torch.cuda.device(P.device):
+        st = load_library().gwq_read_probe(P._h, C.byref(n), _stream_ptr())
+    _check(st, "gwq_read_probe")
+    return int(n.value)
 
 
 def gwq_linear_host(P: Packed, x_host: torch.Tensor, y_host: torch.Tensor) -> torch.Tensor:
