@@ -68,7 +68,7 @@ def kernels_per_linear(M: int, K: int) -> int:
     token-major copy of x when M > 1 and the activations are not staged up front (M > 8, or
     M K too large for 72 KB of staging)."""
     nchunks = (K // 128 + 7) // 8
-    staged = M <= 8 and nchunks * M * 148 * 16 <= 72 * 1024
+    staged = M <= 8 and nchunks * M * 148 * 16 <= 72 * 1024   # (80 KB for small grids: no case of this step)
     return 1 if (staged or M == 1) else 2
 
 
@@ -170,7 +170,7 @@ def build_layer_set(torch, gwq, dev, replicas: int, keep_dense: bool):
     for li, (name, N, K) in enumerate(synth.LLAMA7B_LAYER_SET):
         W, G = synth.make_weight_and_grad(N, K, synth.layer_seed(CONFIG_INDEX, li))
         Wd, Gd = torch.from_numpy(W).to(dev), torch.from_numpy(G).to(dev)
-        entry = dict(name=name, N=N, K=K, packed={}, W=Wd if keep_dense else None)
+        entry = dict(name=name, N=N, K=K, packed={}, W=Wd if keep_dense else None, G=Gd if keep_dense else None)
         for bits in BIT_WIDTHS:
             reps = []
             for r in range(replicas):
@@ -189,7 +189,8 @@ def build_layer_set(torch, gwq, dev, replicas: int, keep_dense: bool):
                 reps.append(P)
             entry["packed"][bits] = reps
         layers.append(entry)
-        del Gd
+        if not keep_dense:
+            del Gd
     return layers, enc
 
 
@@ -350,8 +351,10 @@ def run_cuda_arm(args):
                          "select_gbs_per_pass_of_G": round(enc["select_bytes"] / (enc["select_ms"] * 1e-3) / 1e9, 1),
                          "pack_gbs": round(enc["pack_bytes"] / (enc["pack_ms"] * 1e-3) / 1e9, 1),
                          "note": "14 encodes of the layer set (7 layers x 2 bit widths), first replica"}
+        out["decode_step_7b"] = bench_decode_step_7b(torch, gwq, layers, dev, detail_iters, hbm_peak)
         for L in layers:
             L["W"] = None
+            L["G"] = None
         out["prefill"] = bench_prefill(torch, gwq, dev, args, tf_burst, tf_sust)
         best = max(out["prefill"], key=lambda r: r["tflops"])
         out["prefill_roofline"] = {"bound": "tensor", "kernel": "gwq prefill linear (tcgen05)",
@@ -438,6 +441,66 @@ def bench_dense_library(torch, layers, xs, iters, step_bytes, ms_step):
             "gbs_on_dense_bytes": round(dense_bytes / (ms * 1e-3) / 1e9, 1),
             "gwq_speedup_over_library": round(ms / ms_step, 3),
             "note": "library call (torch.matmul fp16), same 42 (layer, M) products, CUDA graph"}
+
+
+def bench_decode_step_7b(torch, gwq, layers, dev, iters, hbm_peak, blocks: int = 32, bits: int = 4):
+    """Linear time of one whole decode step of a Llama-2-7B-shaped model: `blocks` decoder blocks x 7 projections,
+    every one its own packed copy (distinct addresses, ~3.8 GB at 4 bits: cold by construction), in data-flow
+    order with the sibling projections fused, one CUDA graph; the dense fp16 library product on as many
+    distinct dense copies beside it."""
+    packed = []
+    for b in range(blocks):
+        row = []
+        for L in layers:
+            S = gwq.gwq_select_outliers(L["W"], L["G"], FRAC)
+            row.append(gwq.gwq_pack(L["W"], S, bits, GROUP))
+        packed.append(row)
+    dense = [[L["W"].clone() for L in layers] for _ in range(blocks)]
+    torch.cuda.synchronize()
+    rows = []
+    for M in (1, 8):
+        xk = {}
+        for K in sorted({L["K"] for L in layers}):
+            bits16, _ = synth.make_activations(M, K, seed=synth.layer_seed(3, K % 97), dtype="f16")
+            xk[K] = torch.from_numpy(bits16.view(np.int16).copy()).to(dev).view(torch.float16)
+        ys = [torch.empty((M, L["N"]), dtype=torch.float16, device=dev) for L in layers]
+
+        def run_gwq():
+            for b in range(blocks):
+                for lis in STAGES:
+                    x = xk[layers[lis[0]]["K"]]
+                    if len(lis) > 1:
+                        gwq.gwq_linear_multi([packed[b][li] for li in lis], x, outs=[ys[li] for li in lis])
+                    else:
+                        gwq.gwq_linear(packed[b][lis[0]], x, out=ys[lis[0]])
+
+        def run_dense():
+            for b in range(blocks):
+                for li, L in enumerate(layers):
+                    torch.matmul(xk[L["K"]], dense[b][li].t())
+        t = {}
+        for name, fn in (("gwq", run_gwq), ("dense", run_dense)):
+            replay = capture(torch, fn)
+            for _ in range(2):
+                replay()
+            t[name] = time_region(torch, lambda i: replay(), iters)
+        step_bytes = blocks * sum(algorithmic_bytes(L["N"], L["K"], bits, GROUP, packed[0][li].nnz, M)
+                                  for li, L in enumerate(layers))
+        rows.append({"M": M, "us_per_step": round(t["gwq"] * 1e3, 1), "tokens_per_s": round(M / (t["gwq"] * 1e-3), 1),
+                     "step_bytes": step_bytes, "gbs": round(step_bytes / (t["gwq"] * 1e-3) / 1e9, 1),
+                     "frac_measured_peak": round(step_bytes / (t["gwq"] * 1e-3) / 1e9 / hbm_peak, 4),
+                     "library_fp16_us_per_step": round(t["dense"] * 1e3, 1),
+                     "speedup_over_library_fp16": round(t["dense"] / t["gwq"], 3)})
+    out = {"blocks": blocks, "bits": bits, "linears": blocks * len(layers),
+           "calls_per_step": blocks * len(STAGES), "cases": rows,
+           "note": f"{blocks} packed copies of the 7 synthetic layers at distinct addresses; q|k|v and gate|up fused; "
+                   "linear layers only (no attention, norms or sampling)"}
+    for row in packed:
+        for P in row:
+            P.free()
+    del dense
+    torch.cuda.empty_cache()
+    return out
 
 
 def bench_e2e(torch, gwq, layers, cases, iters, step_bytes, world=1):

@@ -256,6 +256,14 @@ def dequantize(codes, scales, zeros, group: int, row_ptr, col_idx, val) -> np.nd
     return w_hat + S
 
 
+def quality(W: np.ndarray, G: np.ndarray, w_hat: np.ndarray):
+    """The two objectives the method states for a quantized layer (Section 3.1):
+    the squared error ||W - W_Q||_2^2 (Eq. "Q") and the first-order change of the loss
+    g^T (W - W_Q) (Eq. "Taylor" / "final_OPO"), with W_Q = w_hat.  Plain float64 sums."""
+    d = W.astype(np.float64) - w_hat
+    return float(np.sum(d * d)), float(np.sum(G.astype(np.float64) * d))
+
+
 def linear(x: np.ndarray, w_hat: np.ndarray):
     """y = x w_hat^T in float64, and bound = |x| |w_hat|^T (the per-output sum
     of |x_k * w_hat_k| that the floating-point tolerance is stated against)."""

@@ -249,6 +249,7 @@ struct MultiArgs {
   LayerArgs layer[kMaxLayers];
   int first_block[kMaxLayers + 1];
   int count;
+  int sm_count;
   const uint16_t* x;
   const uint16_t* xt;
   const float* xg;
@@ -756,6 +757,7 @@ __global__ void __launch_bounds__(128) tokens_to_columns(const uint16_t* __restr
 }
 
 constexpr size_t kStageAllLimit = 72 * 1024;   // stage every chunk up front when it fits in this much
+constexpr size_t kStageAllLimitSmallGrid = 80 * 1024;   // the same for grids of at most two CTAs per SM
 
 template <int BITS, int TP, bool BF16, int NBUF>
 cudaError_t launch(const MultiArgs& a, cudaStream_t stream) {
@@ -786,7 +788,10 @@ cudaError_t launch(const MultiArgs& a, cudaStream_t stream) {
 template <int BITS, int TP, bool BF16, int RING>
 cudaError_t launch_buf(const MultiArgs& a, cudaStream_t stream) {
   const int nchunks = (a.K / 128 + kChunkGroups - 1) / kChunkGroups;
-  if (TP <= 8 && (size_t)nchunks * a.M * kRowPitch * 16 <= kStageAllLimit) return launch<BITS, TP, BF16, 0>(a, stream);
+  // staging everything up front costs shared memory, hence resident CTAs: beyond kStageAllLimit only two fit on an
+  // SM, which pays off as long as the whole grid is resident at that rate
+  const size_t lim = a.first_block[a.count] <= 2 * a.sm_count ? kStageAllLimitSmallGrid : kStageAllLimit;
+  if (TP <= 8 && (size_t)nchunks * a.M * kRowPitch * 16 <= lim) return launch<BITS, TP, BF16, 0>(a, stream);
   if (TP > 1) {   // ring mode gathers the outliers' activations from a token-major copy
     if (!a.xt || !a.xg) return cudaErrorInvalidValue;
     tokens_to_columns<TP, BF16><<<a.K / 128, 128, 0, stream>>>(a.x, const_cast<uint16_t*>(a.xt), const_cast<float*>(a.xg), a.M, a.K);
@@ -850,6 +855,7 @@ gwq_status gwq_launch_decode_multi(const gwq_packed* const* P, int count, const 
   a.first_block[kMaxLayers] = blocks;
   for (int i = count; i < kMaxLayers; ++i) a.first_block[i] = blocks;
   a.count = count;
+  a.sm_count = pv->sm_count > 0 ? pv->sm_count : 148;
   a.x = static_cast<const uint16_t*>(x); a.yd = yd; a.K = K; a.M = M;
   cudaError_t e;
   if (P[0]->bits == 4) e = (xd == GWQ_BF16) ? launch_tp<4, true>(a, stream) : launch_tp<4, false>(a, stream);

@@ -82,3 +82,48 @@ def test_outliers_enter_once():
     m = L["mask"]
     assert m.sum() == L["row_ptr"][-1] and m.sum() > 0
     assert np.array_equal(w_hat[m], W.astype(np.float64)[m])
+
+
+# ---------------------------------------------------------------- the method's objectives (Section 3.1)
+def test_quality_scalar_definition_and_special_cases():
+    # explicit loops over a tiny layer
+    W, G = synth.make_weight_and_grad(4, 64, seed=9)
+    L = orc.quantize_layer(W, G, 0.05, 4, 64)
+    w_hat = orc.dequantize(L["codes"], L["scales"], L["zeros"], 64, L["row_ptr"], L["col_idx"], L["val"])
+    sq, fo = orc.quality(W, G, w_hat)
+    a = b = 0.0
+    for n in range(4):
+        for k in range(64):
+            d = float(W[n, k]) - float(w_hat[n, k])
+            a += d * d
+            b += float(G[n, k]) * d
+    assert abs(sq - a) <= 1e-15 * max(1.0, a) and abs(fo - b) <= 1e-12 * max(1.0, abs(b))
+    assert sq > 0.0
+    # every weight kept as an outlier: nothing is lost
+    L1 = orc.quantize_layer(W, G, 1.0, 4, 64)
+    w1 = orc.dequantize(L1["codes"], L1["scales"], L1["zeros"], 64, L1["row_ptr"], L1["col_idx"], L1["val"])
+    assert orc.quality(W, G, w1) == (0.0, 0.0)
+    # with g = sign(W - W_Q) the first-order term is the L1 norm of the error, with g = 0 it vanishes
+    d = W.astype(np.float64) - w_hat
+    sq2, l1 = orc.quality(W, np.sign(d).astype(np.float32), w_hat)
+    assert sq2 == sq and abs(l1 - np.abs(d).sum()) <= 1e-12
+    assert orc.quality(W, np.zeros_like(G), w_hat)[1] == 0.0
+    # the squared error respects the rounding bound: at most (s / 2)^2 per non-outlier entry
+    s = np.repeat(L["scales"].astype(np.float64), 64, axis=1)
+    assert sq <= np.sum((0.5 * s[~L["mask"]]) ** 2) * (1 + 1e-12)
+
+
+def test_quality_closed_form_on_a_known_group():
+    # one group whose range fixes s = 2^-6, z = 8; entries a quarter step off the grid lose (s / 4)^2 each
+    base = np.zeros(64)
+    base[0], base[1] = -8, 7
+    base[2:12] = np.arange(10) - 4 + 0.25          # 10 entries, each 0.25 step above a grid point
+    W = (base * 2.0 ** -6).astype(np.float16).reshape(1, 64)
+    G = np.full((1, 64), 2.0, dtype=np.float32)
+    L = orc.quantize_layer(W, G * 0 + np.arange(64, dtype=np.float32)[::-1], 0.0, 4, 64)
+    assert float(L["scales"][0, 0]) == 2.0 ** -6 and int(L["zeros"][0, 0]) == 8
+    w_hat = orc.dequantize(L["codes"], L["scales"], L["zeros"], 64, L["row_ptr"], L["col_idx"], L["val"])
+    sq, fo = orc.quality(W, G, w_hat)
+    step = 2.0 ** -6
+    assert sq == 10 * (0.25 * step) ** 2
+    assert fo == 2.0 * 10 * 0.25 * step                # W - W_Q = +s/4 on those ten entries
