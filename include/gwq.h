@@ -151,6 +151,15 @@ gwq_status gwq_linear(const gwq_packed* P, const void* x, gwq_dtype x_dtype, int
 gwq_status gwq_linear_multi(const gwq_packed* const* P, int32_t count, const void* x, gwq_dtype x_dtype,
                             int32_t M, void* const* y, gwq_dtype y_dtype, void* stream);
 
+/* The two objectives the method states for a quantized layer (Section 3.1): the squared error
+ * ||W - W_Q||_2^2 (Eq. "Q") and the first-order change of the loss g^T (W - W_Q) (Eq. "Taylor",
+ * Eq. "final_OPO"), with W_Q = s (q - z) + S as gwq_linear uses it.  Terms and sums in FP64, in a fixed
+ * order.  W_f16 [N,K], G_f32 [N,K]: device, the arrays P was made from (any other pair of that shape gives
+ * the same formulas on them).  *sq_err, *first_order: host.  Allocates 16 N bytes for the call,
+ * synchronises `stream`.  Errors: INVALID_ARG, ALLOC, CUDA.                                             */
+gwq_status gwq_quality(const uint16_t* W_f16, const float* G_f32, const gwq_packed* P, double* sq_err,
+                       double* first_order, void* stream);
+
 /* Measurement aid, no counterpart in the paper: one launch that reads, and only reads, the arrays a
  * one-token gwq_linear reads of P (packed codes, scales, zero-points, CSR row pointers, outlier entries).
  * Its duration is the floor for any forward product that is one kernel launch per layer; the benchmark

@@ -24,7 +24,7 @@ STATUS_NAMES = {
     4: "GWQ_ERR_NONFINITE", 5: "GWQ_ERR_TIMEOUT", 6: "GWQ_ERR_CUDA",
 }
 EXPORTS = ("gwq_select_outliers", "gwq_select_outliers_static", "gwq_pack", "gwq_linear", "gwq_linear_multi",
-           "gwq_read_probe", "gwq_linear_host", "gwq_device_status", "gwq_free", "gwq_status_string")
+           "gwq_quality", "gwq_read_probe", "gwq_linear_host", "gwq_device_status", "gwq_free", "gwq_status_string")
 GWQ_MULTI_MAX = 4
 
 
@@ -73,6 +73,9 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     lib.gwq_linear_multi.restype = C.c_int
     lib.gwq_linear_multi.argtypes = [C.POINTER(C.POINTER(gwq_packed)), C.c_int32, C.c_void_p, C.c_int, C.c_int32,
                                      C.POINTER(C.c_void_p), C.c_int, C.c_void_p]
+    lib.gwq_quality.restype = C.c_int
+    lib.gwq_quality.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(gwq_packed), C.POINTER(C.c_double),
+                                C.POINTER(C.c_double), C.c_void_p]
     lib.gwq_read_probe.restype = C.c_int
     lib.gwq_read_probe.argtypes = [C.POINTER(gwq_packed), C.POINTER(C.c_int64), C.c_void_p]
     lib.gwq_linear_host.restype = C.c_int
@@ -319,6 +322,21 @@ def gwq_linear_multi(Ps, x: torch.Tensor, out_dtype: torch.dtype | None = None, 
                               _dtype_code(outs[0].dtype) if outs else GWQ_F16, _stream_ptr())
     _check(st, "gwq_linear_multi")
     return outs
+
+
+def gwq_quality(W: torch.Tensor, G: torch.Tensor, P: Packed):
+    """(||W - W_Q||^2, g^T (W - W_Q)) of the packed layer P against W fp16 [N,K] and G fp32 [N,K] on the GPU."""
+    _require_cuda(W, "W")
+    _require_cuda(G, "G")
+    if W.dtype != torch.float16 or G.dtype != torch.float32 or tuple(W.shape) != (P.N, P.K) or W.shape != G.shape:
+        raise ValueError("W must be fp16 [N,K] and G fp32 [N,K] of the layer's shape")
+    if not (W.is_contiguous() and G.is_contiguous()):
+        raise ValueError("W and G must be contiguous")
+    a, b = C.c_double(0.0), C.c_double(0.0)
+    with torch.cuda.device(P.device):
+        st = load_library().gwq_quality(W.data_ptr(), G.data_ptr(), P._h, C.byref(a), C.byref(b), _stream_ptr())
+    _check(st, "gwq_quality")
+    return float(a.value), float(b.value)
 
 
 def gwq_read_probe(P: Packed) -> int:
