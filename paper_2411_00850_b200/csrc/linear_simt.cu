@@ -48,36 +48,39 @@ linear_simt_kernel(const uint32_t* __restrict__ codes, const uint16_t* __restric
       float acc[MT];
 #pragma unroll
       for (int t = 0; t < MT; ++t) acc[t] = 0.f;
+      const int gsz = group < 32 ? group : 32;   // columns of a run that share one scale and zero-point
       for (int r = lane; r < nruns; r += 32) {
-        const int g = (r * 32) / group;
-        const float s = __half2float(__ushort_as_half(scales[(long long)row * ngroups + g]));
-        const float z = (float)zeros[(long long)row * ngroups + g];
         unsigned int w[4] = {0, 0, 0, 0};
         for (int j = 0; j < bits; ++j) w[j] = __ldg(crow + r * bits + j);
-        float part[MT];
+        for (int seg = 0; seg < 32; seg += gsz) {
+          const int g = (r * 32 + seg) / group;
+          const float s = __half2float(__ushort_as_half(scales[(long long)row * ngroups + g]));
+          const float z = (float)zeros[(long long)row * ngroups + g];
+          float part[MT];
 #pragma unroll
-        for (int t = 0; t < MT; ++t) part[t] = 0.f;
-        for (int i = 0; i < 32; ++i) {
-          // pair-interleaved packed order (see include/gwq.h)
-          unsigned int code;
-          const int e = i & 1;
-          if (bits == 4) {
-            code = (w[i >> 3] >> (16 * e + 4 * ((i & 7) >> 1))) & 15u;
-          } else if (i < 30) {
-            const int wi = i / 10, r10 = i - 10 * wi;
-            code = (w[wi] >> (16 * e + 3 * (r10 >> 1))) & 7u;
-          } else {
-            const int sh = 15 + 16 * e;
-            code = ((w[0] >> sh) & 1u) | (((w[1] >> sh) & 1u) << 1) | (((w[2] >> sh) & 1u) << 2);
-          }
-          const float qz = (float)(int)code - z;
+          for (int t = 0; t < MT; ++t) part[t] = 0.f;
+          for (int i = seg; i < seg + gsz; ++i) {
+            // pair-interleaved packed order (see include/gwq.h)
+            unsigned int code;
+            const int e = i & 1;
+            if (bits == 4) {
+              code = (w[i >> 3] >> (16 * e + 4 * ((i & 7) >> 1))) & 15u;
+            } else if (i < 30) {
+              const int wi = i / 10, r10 = i - 10 * wi;
+              code = (w[wi] >> (16 * e + 3 * (r10 >> 1))) & 7u;
+            } else {
+              const int sh = 15 + 16 * e;
+              code = ((w[0] >> sh) & 1u) | (((w[1] >> sh) & 1u) << 1) | (((w[2] >> sh) & 1u) << 2);
+            }
+            const float qz = (float)(int)code - z;
 #pragma unroll
-          for (int t = 0; t < MT; ++t) {
-            if (m0 + t < M) part[t] = fmaf(ld_act<BF16>(x + (long long)(m0 + t) * K + r * 32 + i), qz, part[t]);
+            for (int t = 0; t < MT; ++t) {
+              if (m0 + t < M) part[t] = fmaf(ld_act<BF16>(x + (long long)(m0 + t) * K + r * 32 + i), qz, part[t]);
+            }
           }
+#pragma unroll
+          for (int t = 0; t < MT; ++t) acc[t] = fmaf(s, part[t], acc[t]);
         }
-#pragma unroll
-        for (int t = 0; t < MT; ++t) acc[t] = fmaf(s, part[t], acc[t]);
       }
       for (int j = jb + lane; j < je; j += 32) {
         const float v = __half2float(__ushort_as_half(val[j]));

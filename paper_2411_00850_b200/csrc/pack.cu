@@ -34,20 +34,27 @@ pack_row_kernel(const uint16_t* __restrict__ W, const int32_t* __restrict__ row_
   }
   __syncthreads();
 
-  constexpr int EPL = GROUP / 32;  // consecutive elements per lane
+  // A warp takes one group per pass (GROUP >= 32: GROUP / 32 consecutive elements per lane) or 32 / GROUP
+  // neighbouring groups per pass (GROUP = 16: one element per lane, 16 lanes per group).
+  constexpr int LPG = GROUP >= 32 ? 32 : GROUP;   // lanes per group
+  constexpr int EPL = GROUP / LPG;                // consecutive elements per lane
+  constexpr int GPP = 32 / LPG;                   // groups per warp and pass
   const int ngroups = K / GROUP;
   const double qmax = (double)((1 << bits) - 1);
   const uint16_t* wrow = W + (long long)row * K;
   bool bad = false;
-  for (int g = warp; g < ngroups; g += kThreads / 32) {
-    const int c0 = g * GROUP + lane * EPL;
+  for (int g0 = warp * GPP; g0 < ngroups; g0 += (kThreads / 32) * GPP) {
+    const int g = min(g0 + lane / LPG, ngroups - 1);   // K is a multiple of 32, so every group of a pass exists
+    const int c0 = g * GROUP + (lane % LPG) * EPL;
     unsigned int hb[EPL];
     if (EPL == 4) {
       const uint2 v = *reinterpret_cast<const uint2*>(wrow + c0);
-      hb[0] = v.x & 0xFFFFu; hb[1] = v.x >> 16; hb[EPL - 2] = v.y & 0xFFFFu; hb[EPL - 1] = v.y >> 16;
-    } else {
+      hb[0] = v.x & 0xFFFFu; hb[1 % EPL] = v.x >> 16; hb[(EPL - 2 + EPL) % EPL] = v.y & 0xFFFFu; hb[EPL - 1] = v.y >> 16;
+    } else if (EPL == 2) {
       const unsigned int v = *reinterpret_cast<const unsigned int*>(wrow + c0);
-      hb[0] = v & 0xFFFFu; hb[1] = v >> 16;
+      hb[0] = v & 0xFFFFu; hb[EPL - 1] = v >> 16;
+    } else {
+      hb[0] = wrow[c0];
     }
     // this lane's EPL mask bits: c0 is a multiple of EPL, so they sit in one mask word
     const unsigned int mbits = (mask[c0 >> 5] >> (c0 & 31)) & ((1u << EPL) - 1u);
@@ -62,7 +69,8 @@ pack_row_kernel(const uint16_t* __restrict__ W, const int32_t* __restrict__ row_
         hi = fmaxf(hi, w[e]);
       }
     }
-    for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+    for (int o = LPG / 2; o > 0; o >>= 1) {
       lo = fminf(lo, __shfl_xor_sync(0xFFFFFFFFu, lo, o));
       hi = fmaxf(hi, __shfl_xor_sync(0xFFFFFFFFu, hi, o));
     }
@@ -82,7 +90,7 @@ pack_row_kernel(const uint16_t* __restrict__ W, const int32_t* __restrict__ row_
       if (!((mbits >> e) & 1u)) q = fmin(fmax(rint((double)w[e] / s) + z, 0.0), qmax);
       q8[c0 + e] = (unsigned char)(int)q;
     }
-    if (lane == 0) {
+    if (lane % LPG == 0) {
       scales[(long long)row * ngroups + g] = __half_as_ushort(sh);
       zeros[(long long)row * ngroups + g] = (uint8_t)(int)z;
     }
@@ -144,7 +152,7 @@ extern "C" gwq_status gwq_pack(const uint16_t* W, gwq_outliers* S, int32_t N, in
   if (S->tag != GWQ_TAG_OUTLIERS || S->N != N || S->K != K) return GWQ_ERR_INVALID_ARG;
   if (!gwq_aligned16(W)) return GWQ_ERR_INVALID_ARG;
   if (bits != 3 && bits != 4) return GWQ_ERR_UNSUPPORTED;
-  if (group != 64 && group != 128) return GWQ_ERR_UNSUPPORTED;
+  if (group != 16 && group != 32 && group != 64 && group != 128) return GWQ_ERR_UNSUPPORTED;
   if (K % group != 0 || K > 131072) return GWQ_ERR_UNSUPPORTED;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
 
@@ -172,15 +180,17 @@ extern "C" gwq_status gwq_pack(const uint16_t* W, gwq_outliers* S, int32_t N, in
   GWQ_CUDA_TRY(cudaMalloc(&P->zeros, ngroups + 16));
   GWQ_CUDA_TRY(cudaMalloc(&pv->dev_status, 64));
   GWQ_CUDA_TRY(cudaMemsetAsync(pv->dev_status, 0, 64, stream));
-  if (group == 128) {
-    GWQ_CUDA_TRY(cudaFuncSetAttribute(pack_row_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    pack_row_kernel<128><<<N, kThreads, smem, stream>>>(W, S->row_ptr, S->col_idx, K, bits, P->codes,
-                                                        P->scales, P->zeros, pv->dev_status);
-  } else {
-    GWQ_CUDA_TRY(cudaFuncSetAttribute(pack_row_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    pack_row_kernel<64><<<N, kThreads, smem, stream>>>(W, S->row_ptr, S->col_idx, K, bits, P->codes,
-                                                       P->scales, P->zeros, pv->dev_status);
-  }
+#define GWQ_PACK_LAUNCH(G)                                                                                              \
+  do {                                                                                                                  \
+    GWQ_CUDA_TRY(cudaFuncSetAttribute(pack_row_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));     \
+    pack_row_kernel<G><<<N, kThreads, smem, stream>>>(W, S->row_ptr, S->col_idx, K, bits, P->codes, P->scales,           \
+                                                      P->zeros, pv->dev_status);                                        \
+  } while (0)
+  if (group == 128) GWQ_PACK_LAUNCH(128);
+  else if (group == 64) GWQ_PACK_LAUNCH(64);
+  else if (group == 32) GWQ_PACK_LAUNCH(32);
+  else GWQ_PACK_LAUNCH(16);
+#undef GWQ_PACK_LAUNCH
   GWQ_CUDA_TRY(cudaGetLastError());
   if (K <= 65536) {
     const long long nnz = S->nnz;
@@ -190,10 +200,12 @@ extern "C" gwq_status gwq_pack(const uint16_t* W, gwq_outliers* S, int32_t N, in
       GWQ_CUDA_TRY(cudaGetLastError());
     }
   }
-  GWQ_CUDA_TRY(cudaMalloc(&pv->sz_t, ngroups * sizeof(uint32_t) + 16));
-  transpose_scale_zero_kernel<<<(unsigned)((ngroups + 255) / 256), 256, 0, stream>>>(P->scales, P->zeros, pv->sz_t, N,
-                                                                                     K / group);
-  GWQ_CUDA_TRY(cudaGetLastError());
+  if (group >= 64) {   // the tensor-core path (one scale per 64-column k-block) takes groups of 64 and 128 only
+    GWQ_CUDA_TRY(cudaMalloc(&pv->sz_t, ngroups * sizeof(uint32_t) + 16));
+    transpose_scale_zero_kernel<<<(unsigned)((ngroups + 255) / 256), 256, 0, stream>>>(P->scales, P->zeros, pv->sz_t,
+                                                                                       N, K / group);
+    GWQ_CUDA_TRY(cudaGetLastError());
+  }
   GWQ_CUDA_TRY(cudaMemcpyAsync(&host_status, pv->dev_status, sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
   GWQ_CUDA_TRY(cudaStreamSynchronize(stream));
   if (host_status != 0) {

@@ -37,9 +37,6 @@ quality_row_kernel(const uint16_t* __restrict__ W, const float* __restrict__ G, 
   }
   __syncthreads();
   for (int r = tid; r < nruns; r += kThreads) {
-    const int g = (r * 32) / group;
-    const double s = (double)__half2float(__ushort_as_half(scales[(size_t)n * ngroups + g]));
-    const int z = zeros[(size_t)n * ngroups + g];
     unsigned w[4] = {0, 0, 0, 0};
     for (int j = 0; j < bits; ++j) w[j] = __ldg(crow + r * bits + j);
     const unsigned m = mask[r];
@@ -57,7 +54,9 @@ quality_row_kernel(const uint16_t* __restrict__ W, const float* __restrict__ G, 
         const int sh = 15 + 16 * e;
         code = ((w[0] >> sh) & 1u) | (((w[1] >> sh) & 1u) << 1) | (((w[2] >> sh) & 1u) << 2);
       }
-      const int k = r * 32 + i;
+      const int k = r * 32 + i, g = k / group;
+      const double s = (double)__half2float(__ushort_as_half(scales[(size_t)n * ngroups + g]));
+      const int z = zeros[(size_t)n * ngroups + g];
       const double d = (double)__half2float(__ushort_as_half(wrow[k])) - s * (double)((int)code - z);
       sq += d * d;
       fo += (double)grow[k] * d;

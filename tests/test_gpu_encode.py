@@ -21,6 +21,10 @@ pytestmark = pytest.mark.gpu
     (1000, 2176, 0.01, 3, 64, 5),
     (64, 4096, 0.3, 4, 128, 6),        # dense outliers
     (2048, 2048, 0.01, 4, 128, 7),
+    (300, 1056, 0.01, 4, 16, 8),       # the paper's own group size (Section 3.2: beta = 16); K = 33 * 32
+    (300, 1056, 0.02, 3, 16, 9),
+    (192, 1024, 0.01, 4, 32, 10),
+    (192, 1024, 0.3, 3, 32, 11),
 ])
 def test_encode_matches_checker(N, K, frac, bits, group, seed):
     W, G = synth.make_weight_and_grad(N, K, seed)
@@ -107,7 +111,7 @@ def test_nonfinite_weight_is_an_error_and_bad_arguments():
         gwq.gwq_select_outliers(Wd, Gd, 1.5)
     assert e.value.status == 1
     S = gwq.gwq_select_outliers(Wd, Gd, 0.01)
-    for bits, group, want in ((5, 128, 2), (4, 32, 2), (4, 96, 2)):
+    for bits, group, want in ((5, 128, 2), (4, 8, 2), (4, 96, 2)):
         with pytest.raises(gwq.GwqError) as e:
             gwq.gwq_pack(Wd, S, bits, group)
         assert e.value.status == want

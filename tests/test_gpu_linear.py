@@ -102,6 +102,17 @@ def test_tensor_core_path_reads_back_columns_exactly_in_fp16():
     assert_linear_close(y, y_ref, bound)
 
 
+@pytest.mark.parametrize("layer", [(200, 1056, 0.01, 4, 16, 30), (200, 1056, 0.02, 3, 16, 31), (96, 1024, 0.01, 4, 32, 32)])
+@pytest.mark.parametrize("M,dtype", [(1, "f16"), (5, "bf16"), (16, "f16"), (40, "bf16"), (70, "f16")])
+def test_small_groups(layer, M, dtype):
+    # groups of 16 (the paper's own value, Section 3.2) and 32: the general kernel serves every M
+    P, L, w_hat = _layer(*layer)
+    bits16, xv = synth.make_activations(M, P.K, seed=60 + M, dtype=dtype)
+    y_ref, bound = orc.linear(xv, w_hat)
+    y = gwq.gwq_linear(P, x_tensor(bits16, dtype), out_dtype=torch.float32)
+    assert_linear_close(y, y_ref, bound)
+
+
 def test_all_outliers_is_the_dense_product():
     N, K = 128, 512
     W, G = synth.make_weight_and_grad(N, K, 30)

@@ -16,6 +16,7 @@ pytestmark = pytest.mark.gpu
 @pytest.mark.parametrize("N,K,frac,bits,group,seed", [
     (64, 512, 0.01, 4, 128, 60), (100, 2176, 0.02, 3, 64, 61), (528, 4096, 0.01, 4, 128, 62),
     (33, 1024, 0.0, 3, 128, 63), (16, 256, 1.0, 4, 64, 64), (1000, 2176, 0.3, 4, 64, 65),
+    (100, 1056, 0.01, 4, 16, 66), (64, 1024, 0.02, 3, 32, 67),
 ])
 def test_quality_matches_checker(N, K, frac, bits, group, seed):
     W, G = synth.make_weight_and_grad(N, K, seed)

@@ -66,7 +66,7 @@ def test_degenerate_groups():
 
 # ---------------------------------------------------------------- properties
 @pytest.mark.parametrize("bits,group,frac,seed", [(4, 128, 0.01, 0), (3, 64, 0.02, 1), (4, 64, 0.0, 2),
-                                                   (3, 128, 0.3, 3)])
+                                                   (3, 128, 0.3, 3), (4, 16, 0.01, 4), (3, 32, 0.02, 5)])
 def test_scale_covers_range_and_is_minimal(bits, group, frac, seed):
     N, K = 64, 512
     W, G = synth.make_weight_and_grad(N, K, seed)
@@ -90,7 +90,8 @@ def test_scale_covers_range_and_is_minimal(bits, group, frac, seed):
     assert np.all(np.abs(lo / s + z)[live] <= 0.5)
 
 
-@pytest.mark.parametrize("bits,group,frac", [(4, 128, 0.01), (3, 128, 0.01), (4, 64, 0.005), (3, 64, 0.02)])
+@pytest.mark.parametrize("bits,group,frac", [(4, 128, 0.01), (3, 128, 0.01), (4, 64, 0.005), (3, 64, 0.02),
+                                             (4, 16, 0.01), (3, 16, 0.01), (4, 32, 0.02)])
 def test_error_bound_and_outlier_codes(bits, group, frac):
     N, K = 128, 1024
     W, G = synth.make_weight_and_grad(N, K, seed=4)
