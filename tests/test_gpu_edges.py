@@ -1,0 +1,58 @@
+"""Edge cases of the forward product on the GPU against the CPU checker: the largest K each path
+takes, layers smaller than one tile, no outliers at all, rows with more outliers than a warp keeps
+in registers, and all of them through both the streaming and the tensor-core path where they apply."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import gwq_oracle as orc
+from paper_2411_00850_b200 import binding as gwq
+from paper_2411_00850_b200 import synth
+from tests.gpu_util import (assert_linear_close, assert_packed_equal, oracle_w_hat, quantize_on_gpu, x_tensor)
+
+pytestmark = pytest.mark.gpu
+
+
+def _check(N, K, frac, bits, group, seed, cases):
+    W, G = synth.make_weight_and_grad(N, K, seed)
+    L = orc.quantize_layer(W, G, frac, bits, group)
+    P = quantize_on_gpu(W, G, frac, bits, group)
+    assert_packed_equal(P, L)
+    w_hat = oracle_w_hat(L)
+    for M, dtype in cases:
+        bits16, xv = synth.make_activations(M, K, seed=seed + M, dtype=dtype)
+        y_ref, bound = orc.linear(xv, w_hat)
+        y = gwq.gwq_linear(P, x_tensor(bits16, dtype), out_dtype=torch.float32)
+        assert_linear_close(y, y_ref, bound)
+    assert gwq.gwq_device_status(P) == 0
+    P.free()
+
+
+def test_largest_k_with_16_bit_outlier_columns():
+    # K = 65536: the last K the streaming and tensor-core kernels take (outlier columns in 16 bits)
+    _check(40, 65536, 0.01, 4, 128, 70, [(1, "f16"), (16, "bf16"), (64, "f16")])
+
+
+def test_k_beyond_16_bit_columns_takes_the_general_kernel():
+    _check(16, 131072, 0.005, 3, 128, 71, [(1, "f16"), (40, "bf16")])
+
+
+@pytest.mark.parametrize("N", [1, 15, 17])
+def test_fewer_rows_than_a_tile(N):
+    _check(N, 1024, 0.02, 4, 128, 72 + N, [(1, "f16"), (32, "bf16"), (33, "f16"), (300, "bf16")])
+
+
+@pytest.mark.parametrize("bits", [4, 3])
+def test_no_outliers(bits):
+    _check(272, 2048, 0.0, bits, 128, 75, [(1, "f16"), (4, "bf16"), (16, "f16"), (128, "bf16")])
+
+
+def test_rows_with_hundreds_of_outliers():
+    # 30 % outliers: ~1200 per row, far more than the 96 entries a warp keeps in registers on the streaming
+    # path and than the look-ahead window of the tensor-core path
+    _check(64, 4096, 0.3, 3, 128, 76, [(1, "f16"), (8, "bf16"), (16, "f16"), (17, "bf16"), (96, "f16")])
+
+
+def test_one_group_per_row():
+    # K = 128: a single group, seven of the eight warps of a streaming CTA have nothing to do
+    _check(96, 128, 0.05, 4, 128, 77, [(1, "f16"), (16, "f16"), (64, "bf16")])
