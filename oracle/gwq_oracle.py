@@ -72,6 +72,15 @@ __all__ = [
 # --------------------------------------------------------------------------
 # Eq. "o": outlier location
 # --------------------------------------------------------------------------
+def gradient_mean(G_list) -> np.ndarray:
+    """Gradient mean over calibration samples (Section 4.5, "Effect on Number of Calibration"):
+    float32 additions in list order, then one float32 division by the count."""
+    acc = np.array(G_list[0], dtype=np.float32, copy=True)
+    for G in G_list[1:]:
+        acc = (acc + np.asarray(G, dtype=np.float32)).astype(np.float32)
+    return (acc / np.float32(len(G_list))).astype(np.float32)
+
+
 def outlier_count(frac: float, numel: int) -> int:
     """Number of kept outliers: ceil(frac * numel) in IEEE double, clamped."""
     if not (0.0 <= frac <= 1.0):

@@ -121,3 +121,22 @@ def test_select_special_values_order():
     _, ci, _ = orc.select_outliers(W, G, 26 / 32)
     zero_cols_taken = [c for c in ci.tolist() if c % 8 in (0, 1)]
     assert len(ci) == 26 and zero_cols_taken == [0, 1]
+
+
+# ---------------------------------------------------------------- gradient mean over calibration samples (Section 4.5)
+def test_gradient_mean_pins():
+    rng = np.random.default_rng(21)
+    G = rng.normal(size=(6, 8, 32)).astype(np.float32)
+    # one sample: the gradient itself
+    assert np.array_equal(orc.gradient_mean([G[0]]), G[0])
+    # small integers: every float32 sum is exact, so the mean is the exact quotient rounded once
+    I = rng.integers(-50, 50, size=(5, 4, 16)).astype(np.float32)
+    want = (I.astype(np.float64).sum(axis=0) / 5.0).astype(np.float32)
+    assert np.array_equal(orc.gradient_mean(list(I)), want)
+    # general values: within count roundings of the float64 mean
+    m = orc.gradient_mean(list(G))
+    ref = G.astype(np.float64).mean(axis=0)
+    assert m.dtype == np.float32
+    assert np.all(np.abs(m - ref) <= 6 * 2.0 ** -24 * np.abs(G).astype(np.float64).sum(axis=0) / 6 + 1e-45)
+    # a power-of-two count of equal samples returns the sample (doubling and halving are exact)
+    assert np.array_equal(orc.gradient_mean([G[1]] * 4), G[1])
