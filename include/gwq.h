@@ -154,6 +154,17 @@ gwq_status gwq_linear(const gwq_packed* P, const void* x, gwq_dtype x_dtype, int
 gwq_status gwq_linear_multi(const gwq_packed* const* P, int32_t count, const void* x, gwq_dtype x_dtype,
                             int32_t M, void* const* y, gwq_dtype y_dtype, void* stream);
 
+/* Mean of the gradients of `count` calibration samples (Section 4.5, "Effect on Number of Calibration":
+ * the outliers are located on the gradient mean); the result feeds gwq_select_outliers.
+ * G_mean[i] = (((G_0[i] + G_1[i]) + G_2[i]) + ...) / count, FP32, additions in sample order, round to
+ * nearest, one division: reproducible bit for bit.
+ *   G_list: host array of `count` device pointers (1 <= count <= GWQ_GRAD_SAMPLES_MAX), each [numel] fp32.
+ *   G_mean: device [numel] fp32, caller-owned; may be one of the inputs.  Asynchronous on `stream`.
+ * Errors: INVALID_ARG, CUDA.                                                                          */
+#define GWQ_GRAD_SAMPLES_MAX 16
+gwq_status gwq_gradient_mean(const float* const* G_list, int32_t count, int64_t numel, float* G_mean,
+                             void* stream);
+
 /* The two objectives the method states for a quantized layer (Section 3.1): the squared error
  * ||W - W_Q||_2^2 (Eq. "Q") and the first-order change of the loss g^T (W - W_Q) (Eq. "Taylor",
  * Eq. "final_OPO"), with W_Q = s (q - z) + S as gwq_linear uses it.  Terms and sums in FP64, in a fixed

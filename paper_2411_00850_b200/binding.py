@@ -24,7 +24,7 @@ STATUS_NAMES = {
     4: "GWQ_ERR_NONFINITE", 5: "GWQ_ERR_TIMEOUT", 6: "GWQ_ERR_CUDA",
 }
 EXPORTS = ("gwq_select_outliers", "gwq_select_outliers_static", "gwq_pack", "gwq_linear", "gwq_linear_multi",
-           "gwq_quality", "gwq_read_probe", "gwq_linear_host", "gwq_device_status", "gwq_free", "gwq_status_string")
+           "gwq_gradient_mean", "gwq_quality", "gwq_read_probe", "gwq_linear_host", "gwq_device_status", "gwq_free", "gwq_status_string")
 GWQ_MULTI_MAX = 4
 
 
@@ -73,6 +73,8 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     lib.gwq_linear_multi.restype = C.c_int
     lib.gwq_linear_multi.argtypes = [C.POINTER(C.POINTER(gwq_packed)), C.c_int32, C.c_void_p, C.c_int, C.c_int32,
                                      C.POINTER(C.c_void_p), C.c_int, C.c_void_p]
+    lib.gwq_gradient_mean.restype = C.c_int
+    lib.gwq_gradient_mean.argtypes = [C.POINTER(C.c_void_p), C.c_int32, C.c_int64, C.c_void_p, C.c_void_p]
     lib.gwq_quality.restype = C.c_int
     lib.gwq_quality.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(gwq_packed), C.POINTER(C.c_double),
                                 C.POINTER(C.c_double), C.c_void_p]
@@ -322,6 +324,23 @@ def gwq_linear_multi(Ps, x: torch.Tensor, out_dtype: torch.dtype | None = None, 
                               _dtype_code(outs[0].dtype) if outs else GWQ_F16, _stream_ptr())
     _check(st, "gwq_linear_multi")
     return outs
+
+
+def gwq_gradient_mean(Gs, out: torch.Tensor | None = None) -> torch.Tensor:
+    """FP32 mean of the gradients of several calibration samples (same shape, on the GPU), added in list order."""
+    if len(Gs) < 1:
+        raise ValueError("at least one gradient")
+    for G in Gs:
+        _require_cuda(G, "G")
+        if G.dtype != torch.float32 or G.shape != Gs[0].shape or not G.is_contiguous():
+            raise ValueError("gradients must be contiguous fp32 tensors of one shape")
+    if out is None:
+        out = torch.empty_like(Gs[0])
+    ptrs = (C.c_void_p * len(Gs))(*[G.data_ptr() for G in Gs])
+    with torch.cuda.device(Gs[0].device):
+        st = load_library().gwq_gradient_mean(ptrs, len(Gs), Gs[0].numel(), out.data_ptr(), _stream_ptr())
+    _check(st, "gwq_gradient_mean")
+    return out
 
 
 def gwq_quality(W: torch.Tensor, G: torch.Tensor, P: Packed):

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libgwq.so")
-SOURCES = ("select.cu", "select_static.cu", "pack.cu", "linear_simt.cu", "linear_decode.cu", "linear_prefill.cu", "probe.cu", "quality.cu", "api.cu")
+SOURCES = ("select.cu", "select_static.cu", "pack.cu", "linear_simt.cu", "linear_decode.cu", "linear_prefill.cu", "probe.cu", "quality.cu", "gradmean.cu", "api.cu")
 NVCC_FLAGS = (
     "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
     "-Xcompiler", "-fPIC", "-shared",
