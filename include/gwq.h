@@ -188,6 +188,15 @@ gwq_status gwq_read_probe(const gwq_packed* P, int64_t* bytes_read, void* stream
 gwq_status gwq_linear_host(gwq_packed* P, const void* x_host, gwq_dtype x_dtype, int32_t M,
                            void* y_host, gwq_dtype y_dtype, void* stream);
 
+/* gwq_linear_host without the final synchronisation: the copy of x, the product and the copy of y are
+ * enqueued on `stream` and the call returns; y_host is valid, and x_host may be reused, once the caller
+ * has synchronised the stream (one synchronisation can serve many calls).  Calls that share P must be
+ * on one stream (they share P's staging buffers, and stream order keeps them apart).  Use page-locked
+ * host buffers, or the copies are not asynchronous.  A call that has to grow the staging buffers
+ * synchronises the stream and allocates.  Errors: as gwq_linear_host.                              */
+gwq_status gwq_linear_host_async(gwq_packed* P, const void* x_host, gwq_dtype x_dtype, int32_t M,
+                                 void* y_host, gwq_dtype y_dtype, void* stream);
+
 /* Device-side status of the gwq_linear calls made on P so far: synchronises `stream`, returns
  * GWQ_OK or the error a kernel recorded (GWQ_ERR_TIMEOUT when a bounded wait inside the
  * tensor-core path ran out and the kernel returned early; y is then undefined, and later

@@ -24,7 +24,7 @@ STATUS_NAMES = {
     4: "GWQ_ERR_NONFINITE", 5: "GWQ_ERR_TIMEOUT", 6: "GWQ_ERR_CUDA",
 }
 EXPORTS = ("gwq_select_outliers", "gwq_select_outliers_static", "gwq_pack", "gwq_linear", "gwq_linear_multi",
-           "gwq_gradient_mean", "gwq_quality", "gwq_read_probe", "gwq_linear_host", "gwq_device_status", "gwq_free", "gwq_status_string")
+           "gwq_gradient_mean", "gwq_quality", "gwq_read_probe", "gwq_linear_host", "gwq_linear_host_async", "gwq_device_status", "gwq_free", "gwq_status_string")
 GWQ_MULTI_MAX = 4
 
 
@@ -82,6 +82,8 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     lib.gwq_read_probe.argtypes = [C.POINTER(gwq_packed), C.POINTER(C.c_int64), C.c_void_p]
     lib.gwq_linear_host.restype = C.c_int
     lib.gwq_linear_host.argtypes = lib.gwq_linear.argtypes
+    lib.gwq_linear_host_async.restype = C.c_int
+    lib.gwq_linear_host_async.argtypes = lib.gwq_linear.argtypes
     lib.gwq_device_status.restype = C.c_int
     lib.gwq_device_status.argtypes = [C.POINTER(gwq_packed), C.c_void_p]
     lib.gwq_free.restype = None
@@ -377,6 +379,19 @@ def gwq_linear_host(P: Packed, x_host: torch.Tensor, y_host: torch.Tensor) -> to
         st = lib.gwq_linear_host(P._h, x_host.data_ptr(), _dtype_code(x_host.dtype), M, y_host.data_ptr(),
                                  _dtype_code(y_host.dtype), _stream_ptr())
     _check(st, "gwq_linear_host")
+    return y_host
+
+
+def gwq_linear_host_async(P: Packed, x_host: torch.Tensor, y_host: torch.Tensor) -> torch.Tensor:
+    """gwq_linear_host without the synchronisation: y_host is valid after the current stream has been synchronised."""
+    lib = load_library()
+    if x_host.is_cuda or y_host.is_cuda:
+        raise ValueError("gwq_linear_host_async takes host tensors")
+    M = x_host.shape[0]
+    with torch.cuda.device(P.device):
+        st = lib.gwq_linear_host_async(P._h, x_host.data_ptr(), _dtype_code(x_host.dtype), M, y_host.data_ptr(),
+                                       _dtype_code(y_host.dtype), _stream_ptr())
+    _check(st, "gwq_linear_host_async")
     return y_host
 
 

@@ -42,8 +42,8 @@ extern "C" gwq_status gwq_linear_multi(const gwq_packed* const* P, int32_t count
   return GWQ_OK;
 }
 
-extern "C" gwq_status gwq_linear_host(gwq_packed* P, const void* x_host, gwq_dtype xd, int32_t M,
-                                      void* y_host, gwq_dtype yd, void* stream_) {
+static gwq_status linear_host(gwq_packed* P, const void* x_host, gwq_dtype xd, int32_t M, void* y_host, gwq_dtype yd,
+                              void* stream_, bool synchronise) {
   if (!P || P->tag != GWQ_TAG_PACKED || !P->priv || !x_host || !y_host || M <= 0) return GWQ_ERR_INVALID_ARG;
   if (xd != GWQ_F16 && xd != GWQ_BF16) return GWQ_ERR_UNSUPPORTED;
   if (yd != GWQ_F16 && yd != GWQ_BF16 && yd != GWQ_F32) return GWQ_ERR_INVALID_ARG;
@@ -71,10 +71,20 @@ extern "C" gwq_status gwq_linear_host(gwq_packed* P, const void* x_host, gwq_dty
   st = gwq_linear(P, pv->x_stage, xd, M, pv->y_stage, yd, stream);
   if (st != GWQ_OK) return st;
   GWQ_CUDA_TRY(cudaMemcpyAsync(y_host, pv->y_stage, yb, cudaMemcpyDeviceToHost, stream));
-  GWQ_CUDA_TRY(cudaStreamSynchronize(stream));
+  if (synchronise) GWQ_CUDA_TRY(cudaStreamSynchronize(stream));
   return GWQ_OK;
 fail:
   return st;
+}
+
+extern "C" gwq_status gwq_linear_host(gwq_packed* P, const void* x_host, gwq_dtype xd, int32_t M,
+                                      void* y_host, gwq_dtype yd, void* stream_) {
+  return linear_host(P, x_host, xd, M, y_host, yd, stream_, true);
+}
+
+extern "C" gwq_status gwq_linear_host_async(gwq_packed* P, const void* x_host, gwq_dtype xd, int32_t M,
+                                            void* y_host, gwq_dtype yd, void* stream_) {
+  return linear_host(P, x_host, xd, M, y_host, yd, stream_, false);
 }
 
 extern "C" gwq_status gwq_device_status(const gwq_packed* P, void* stream_) {

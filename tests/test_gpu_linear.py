@@ -133,6 +133,13 @@ def test_host_buffer_entry_point_and_argument_errors():
     yh = torch.empty((4, P.N), dtype=torch.float32).pin_memory()
     gwq.gwq_linear_host(P, xh, yh)
     assert_linear_close(yh, y_ref, bound)
+    # the asynchronous variant: two calls in a row on the same layer, results valid after one synchronisation
+    ya, yb = (torch.zeros((4, P.N), dtype=torch.float32).pin_memory() for _ in range(2))
+    gwq.gwq_linear_host_async(P, xh, ya)
+    gwq.gwq_linear_host_async(P, xh, yb)
+    torch.cuda.synchronize()
+    assert_linear_close(ya, y_ref, bound)
+    assert torch.equal(ya, yb)
     with pytest.raises(gwq.GwqError) as e:
         gwq.gwq_linear(P, torch.zeros((2, P.K), dtype=torch.float32, device="cuda:0"))
     assert e.value.status == 2
