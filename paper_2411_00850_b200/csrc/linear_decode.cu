@@ -392,6 +392,24 @@ __global__ void __launch_bounds__(kThreads, TP <= 8 ? 3 : (TP == 16 ? 2 : 1)) de
   }
   if (tid < 16) reinterpret_cast<unsigned*>(smem_raw)[tid] = 0u;
 
+  const int j0 = __shfl_sync(0xFFFFFFFFu, rp, 0), j1 = __shfl_sync(0xFFFFFFFFu, rp, 1),
+            j2 = __shfl_sync(0xFFFFFFFFu, rp, 2);
+  // ring mode: lane = (entry, group of VT tokens); the first kPre batches of outlier entries of both owned rows
+  // are requested now (they are weights: no need to wait for the previous kernel)
+  constexpr int VT = TP < 8 ? TP : 8, TS = TP / VT, EPB = 32 / TS;
+  constexpr int kPre = TP <= 8 ? 2 : 3;   // batches of EPB entries per row: 64 entries up to 8 tokens, 48 / 24 beyond
+  unsigned epre[2][kPre];
+  if (NBUF != 0) {
+#pragma unroll
+    for (int rr = 0; rr < 2; ++rr) {
+      const int jb = rr == 0 ? j0 : j1, je = rr == 0 ? j1 : j2;
+#pragma unroll
+      for (int u = 0; u < kPre; ++u) {
+        const int j = jb + u * EPB + lane / TS;
+        epre[rr][u] = j < je ? __ldg(p.cv + j) : 0u;   // value 0, column 0
+      }
+    }
+  }
   // ---- from here on x is read
   pdl_wait();
   // NBUF == 0: copy of chunk c of the activations into its buffer, by the whole CTA
@@ -437,8 +455,6 @@ __global__ void __launch_bounds__(kThreads, TP <= 8 ? 3 : (TP == 16 ? 2 : 1)) de
   // outlier payload of the two owned rows.  With everything staged (NBUF == 0) entry lane + 32 e of a
   // row is loaded into cv[row][e] now (up to 96 per row; all ones = no entry) and meets the staged
   // activations after the loop; in ring mode the entries are read after the loop.
-  const int j0 = __shfl_sync(0xFFFFFFFFu, rp, 0), j1 = __shfl_sync(0xFFFFFFFFu, rp, 1),
-            j2 = __shfl_sync(0xFFFFFFFFu, rp, 2);
   unsigned cv[2][kOutSlots];
   if (NBUF == 0) {
 #pragma unroll
@@ -451,40 +467,49 @@ __global__ void __launch_bounds__(kThreads, TP <= 8 ? 3 : (TP == 16 ? 2 : 1)) de
 
   if (NBUF != 0) {
     // ring mode: the outliers are done now, while the first codes are still on their way.  The
-    // activations come from the token-major copy xt[K][TP] (one short contiguous read per entry):
-    // lane = (entry, group of VT tokens), two batches of entries in flight.
-    constexpr int VT = TP < 8 ? TP : 8, TS = TP / VT, EPB = 32 / TS;
+    // activations come from the token-major copy xt[K][TP] (one short contiguous read per entry).
+    // All reads for the entries requested above are issued before any is used; longer rows continue
+    // with two batches of entries in flight.
     const uint16_t* xt = TP == 1 ? p.x : p.xt;
     const int part = lane % TS;
+    auto xt_load = [&](unsigned ent) {
+      const uint16_t* src = xt + (size_t)(ent & 0xFFFFu) * TP + part * VT;
+      if (VT == 8) return __ldg(reinterpret_cast<const uint4*>(src));
+      if (VT == 4) { const uint2 q = __ldg(reinterpret_cast<const uint2*>(src)); return make_uint4(q.x, q.y, 0, 0); }
+      return make_uint4(__ldg(src), 0, 0, 0);
+    };
+    uint4 xpre[2][kPre];
+#pragma unroll
+    for (int rr = 0; rr < 2; ++rr)
+#pragma unroll
+      for (int u = 0; u < kPre; ++u) xpre[rr][u] = xt_load(epre[rr][u]);
 #pragma unroll
     for (int rr = 0; rr < 2; ++rr) {
       const int jb = rr == 0 ? j0 : j1, je = rr == 0 ? j1 : j2;
       float v[VT];
 #pragma unroll
       for (int i = 0; i < VT; ++i) v[i] = 0.f;
-      for (int jj = jb; jj < je; jj += 2 * EPB) {
+      auto add = [&](unsigned ent, const uint4& xq) {
+        const float wv = __half2float(__ushort_as_half((unsigned short)(ent >> 16)));
+        const unsigned w4[4] = {xq.x, xq.y, xq.z, xq.w};
+#pragma unroll
+        for (int i = 0; i < VT; ++i)
+          v[i] = fmaf(wv, act_to_float<BF16>((uint16_t)(w4[i >> 1] >> (16 * (i & 1)))), v[i]);
+      };
+#pragma unroll
+      for (int u = 0; u < kPre; ++u) add(epre[rr][u], xpre[rr][u]);
+      for (int jj = jb + kPre * EPB; jj < je; jj += 2 * EPB) {
         unsigned e[2];
         uint4 xq[2];
 #pragma unroll
         for (int u = 0; u < 2; ++u) {
           const int j = jj + u * EPB + lane / TS;
-          e[u] = j < je ? __ldg(p.cv + j) : 0u;   // value 0, column 0
+          e[u] = j < je ? __ldg(p.cv + j) : 0u;
         }
 #pragma unroll
-        for (int u = 0; u < 2; ++u) {
-          const uint16_t* src = xt + (size_t)(e[u] & 0xFFFFu) * TP + part * VT;
-          if (VT == 8) xq[u] = __ldg(reinterpret_cast<const uint4*>(src));
-          else if (VT == 4) { const uint2 q = __ldg(reinterpret_cast<const uint2*>(src)); xq[u] = make_uint4(q.x, q.y, 0, 0); }
-          else xq[u] = make_uint4(__ldg(src), 0, 0, 0);
-        }
+        for (int u = 0; u < 2; ++u) xq[u] = xt_load(e[u]);
 #pragma unroll
-        for (int u = 0; u < 2; ++u) {
-          const float wv = __half2float(__ushort_as_half((unsigned short)(e[u] >> 16)));
-          const unsigned w4[4] = {xq[u].x, xq[u].y, xq[u].z, xq[u].w};
-#pragma unroll
-          for (int i = 0; i < VT; ++i)
-            v[i] = fmaf(wv, act_to_float<BF16>((uint16_t)(w4[i >> 1] >> (16 * (i & 1)))), v[i]);
-        }
+        for (int u = 0; u < 2; ++u) add(e[u], xq[u]);
       }
       reduce_tokens<VT, TS>(v, lane);
       constexpr int LPV = 32 / VT;   // lanes per value after the halving stages
