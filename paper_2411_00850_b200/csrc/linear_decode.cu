@@ -392,10 +392,16 @@ __global__ void __launch_bounds__(kThreads, TP <= 8 ? 3 : (TP == 16 ? 2 : 1)) de
   }
   if (tid < 16) reinterpret_cast<unsigned*>(smem_raw)[tid] = 0u;
 
-  const int j0 = __shfl_sync(0xFFFFFFFFu, rp, 0), j1 = __shfl_sync(0xFFFFFFFFu, rp, 1),
-            j2 = __shfl_sync(0xFFFFFFFFu, rp, 2);
-  // ring mode: lane = (entry, group of VT tokens); the first kPre batches of outlier entries of both owned rows
-  // are requested now (they are weights: no need to wait for the previous kernel)
+  // CSR extents of the two owned rows.  Ring mode needs them now (lane = (entry, group of VT tokens): the first
+  // kPre batches of outlier entries of both rows are requested before the wait on the previous kernel, they are
+  // weights); with everything staged they are taken after the activations have been requested, so that waiting
+  // for the row pointers delays nothing.
+  int j0 = 0, j1 = 0, j2 = 0;
+  if (NBUF != 0) {
+    j0 = __shfl_sync(0xFFFFFFFFu, rp, 0);
+    j1 = __shfl_sync(0xFFFFFFFFu, rp, 1);
+    j2 = __shfl_sync(0xFFFFFFFFu, rp, 2);
+  }
   constexpr int VT = TP < 8 ? TP : 8, TS = TP / VT, EPB = 32 / TS;
   constexpr int kPre = TP <= 8 ? 2 : 3;   // batches of EPB entries per row: 64 entries up to 8 tokens, 48 / 24 beyond
   unsigned epre[2][kPre];
@@ -457,6 +463,9 @@ __global__ void __launch_bounds__(kThreads, TP <= 8 ? 3 : (TP == 16 ? 2 : 1)) de
   // activations after the loop; in ring mode the entries are read after the loop.
   unsigned cv[2][kOutSlots];
   if (NBUF == 0) {
+    j0 = __shfl_sync(0xFFFFFFFFu, rp, 0);
+    j1 = __shfl_sync(0xFFFFFFFFu, rp, 1);
+    j2 = __shfl_sync(0xFFFFFFFFu, rp, 2);
 #pragma unroll
     for (int e = 0; e < kOutSlots; ++e) {
       const int ja = j0 + lane + 32 * e, jb = j1 + lane + 32 * e;
