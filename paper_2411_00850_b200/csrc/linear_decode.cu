@@ -306,9 +306,12 @@ template <int BITS, int NB> struct StepAcc<BITS, NB, true> { using type = AccSub
 
 // TP = tokens rounded up to 1, 4, 8, 16 or 32.  Group size 128.
 // NBUF = 0: the activations of all chunks are staged up front by the whole CTA (small M K).
-// NBUF = 2: every warp keeps a private double buffer with the activations of its own group only
+// NBUF = 2, 3: every warp keeps a private ring of NBUF buffers with the activations of its own group only
 //           (M x 128 columns), copied one step ahead with cp.async; no CTA barrier in the K loop.
-constexpr int kTilePitch = 16 + 2 + 2;   // pieces per token row of a warp tile (same padding rule)
+constexpr int kTilePitch = 16;   // pieces per token row of a warp tile: no padding, the pieces of a row are permuted
+// piece p (16 bytes) of token row m of a warp tile: the XOR keeps the four lanes of a quad and four neighbouring
+// token rows in different 16-byte bank groups
+__device__ __forceinline__ int tile_piece(int pc, int m) { return m * kTilePitch + (pc ^ (pc >> 3) ^ ((m & 3) << 1)); }
 template <int BITS, int TP, bool BF16, int NBUF>
 __global__ void __launch_bounds__(kThreads, TP <= 8 ? 3 : (TP == 16 ? 2 : 1)) decode_kernel(const MultiArgs ma) {
   // the layer this CTA works for and its row block inside that layer
@@ -431,23 +434,23 @@ __global__ void __launch_bounds__(kThreads, TP <= 8 ? 3 : (TP == 16 ? 2 : 1)) de
       }
     }
   };
-  // NBUF == 2: copy of the activations of this warp's step c (group warp + 8 c) into its buffer c & 1
+  // ring mode: copy of the activations of this warp's step c (group warp + 8 c) into its buffer c % NBUF
+  constexpr int kBufs = NBUF == 0 ? 1 : NBUF;
   const int tile_pieces = p.M * kTilePitch;
-  uint4* wtile = sm_x + warp * 2 * tile_pieces;
+  uint4* wtile = sm_x + warp * kBufs * tile_pieces;
   // lane L copies piece L & 15 of the token rows (L >> 4), (L >> 4) + 2, ...: constant strides, three
   // instructions per 16-byte piece
   const int st_m0 = lane >> 4, st_pc = lane & 15;
-  const unsigned st_dst0 =
-      (unsigned)__cvta_generic_to_shared(wtile + st_m0 * kTilePitch + st_pc + (st_pc >> 3) + ((st_m0 & 1) << 1));
+  const unsigned st_dst0 = (unsigned)__cvta_generic_to_shared(wtile);
   const uint16_t* st_src0 = p.x + (size_t)st_m0 * p.K + (size_t)warp * 128 + st_pc * 8;
   auto stage_tile = [&](int c) {
     if (c < nsteps) {
       const uint16_t* src = st_src0 + (size_t)c * (kWarps * 128);
-      unsigned dst = st_dst0 + (unsigned)((c & 1) * tile_pieces) * 16u;
+      const unsigned dst = st_dst0 + (unsigned)((c % kBufs) * tile_pieces) * 16u;
       for (int m = st_m0; m < p.M; m += 2) {
-        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src));
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + (unsigned)tile_piece(st_pc, m) * 16u),
+                     "l"(src));
         src += 2 * (size_t)p.K;
-        dst += 2 * kTilePitch * 16;
       }
     }
   };
@@ -457,6 +460,13 @@ __global__ void __launch_bounds__(kThreads, TP <= 8 ? 3 : (TP == 16 ? 2 : 1)) de
     stage_tile(0);
   }
   asm volatile("cp.async.commit_group;" ::: "memory");   // also carries the scale / zero-point tables
+  if (NBUF != 0) {   // the tiles of the following steps, one group each
+#pragma unroll
+    for (int c = 1; c + 1 < kBufs; ++c) {
+      stage_tile(c);
+      asm volatile("cp.async.commit_group;" ::: "memory");
+    }
+  }
 
   // outlier payload of the two owned rows.  With everything staged (NBUF == 0) entry lane + 32 e of a
   // row is loaded into cv[row][e] now (up to 96 per row; all ones = no entry) and meets the staged
@@ -526,21 +536,23 @@ __global__ void __launch_bounds__(kThreads, TP <= 8 ? 3 : (TP == 16 ? 2 : 1)) de
       if ((lane % LPV) / TS == 0) sm_out[(2 * warp + rr) * TP + tok] = v[0];
     }
   }
-  asm volatile("cp.async.wait_group 0;" ::: "memory");
+  asm volatile("cp.async.wait_group %0;" ::"n"(NBUF == 0 ? 0 : NBUF - 2) : "memory");   // tables (and first tile) landed
   __syncthreads();
 
   // lane constants inside a chunk buffer: this lane's 64-byte segment of group `warp` for token gid
   // of every token block (lanes without a token read the zero page), the scale tables, the x sums
-  int xoff[NB];
+  // (ring mode: the four pieces of the segment sit in one aligned block of the permuted row, in the order i ^ xcx)
+  int xoff[NB], xcx[NB];
 #pragma unroll
   for (int nb = 0; nb < NB; ++nb) {
     const int m = nb * 8 + gid;
-    xoff[nb] = m >= p.M ? -1 : (NBUF == 0 ? xs_piece(warp * 16 + t * 4, m) : m * kTilePitch + 4 * t + (t >> 1) + ((m & 1) << 1));
+    xoff[nb] = m >= p.M ? -1 : (NBUF == 0 ? xs_piece(warp * 16 + t * 4, m) : m * kTilePitch + ((t ^ ((m >> 1) & 1)) << 2));
+    xcx[nb] = (NBUF == 0 || m >= p.M) ? 0 : ((t >> 1) ^ ((m & 1) << 1));
   }
   const uint16_t* sp = sm_s + gid * ngroups + warp;   // scale / zero-point of row gid, group `warp`
   const uint8_t* zp = sm_z + gid * ngroups + warp;
   const int hi_row = 8 * ngroups;
-  const int xsum_off = (NBUF == 0 ? xs_piece(warp * 16 + (lane >> 1), 0) : (lane >> 1) + (lane >> 4)) * 2 + (lane & 1);   // 8-byte units, token 0
+  const int xsum_off = (NBUF == 0 ? xs_piece(warp * 16 + (lane >> 1), 0) : ((lane >> 1) ^ (lane >> 4))) * 2 + (lane & 1);   // 8-byte units, token 0
 
   float yacc[NB][4];
 #pragma unroll
@@ -557,11 +569,11 @@ __global__ void __launch_bounds__(kThreads, TP <= 8 ? 3 : (TP == 16 ? 2 : 1)) de
     constexpr bool checked = decltype(checked_t)::value;
     if (NBUF != 0) {   // next step's activations on their way, this step's landed and visible to the warp
       __syncwarp();
-      stage_tile(c + 1);
-      asm volatile("cp.async.commit_group;\ncp.async.wait_group 1;" ::: "memory");
+      stage_tile(c + kBufs - 1);
+      asm volatile("cp.async.commit_group;\ncp.async.wait_group %0;" ::"n"(NBUF == 0 ? 0 : NBUF - 1) : "memory");
       __syncwarp();
     }
-    const uint4* buf = NBUF == 0 ? sm_x + c * buf_pieces : wtile + (c & 1) * tile_pieces;
+    const uint4* buf = NBUF == 0 ? sm_x + c * buf_pieces : wtile + (c % kBufs) * tile_pieces;
     if (!checked || c < nsteps) {
       unsigned xr[NB][16];
 #pragma unroll
@@ -569,7 +581,7 @@ __global__ void __launch_bounds__(kThreads, TP <= 8 ? 3 : (TP == 16 ? 2 : 1)) de
         const uint4* seg = xoff[nb] >= 0 ? buf + xoff[nb] : reinterpret_cast<const uint4*>(smem_raw);
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-          const uint4 v = seg[i];
+          const uint4 v = seg[i ^ xcx[nb]];
           xr[nb][4 * i] = v.x; xr[nb][4 * i + 1] = v.y; xr[nb][4 * i + 2] = v.z; xr[nb][4 * i + 3] = v.w;
         }
       }
@@ -660,7 +672,7 @@ __global__ void __launch_bounds__(kThreads, TP <= 8 ? 3 : (TP == 16 ? 2 : 1)) de
       if (!BF16 && TP == 1) {
 #pragma unroll
         for (int d = 0; d < kDepth; ++d) {
-          const uint4* buf = NBUF == 0 ? sm_x + (c0 + d) * buf_pieces : wtile + ((c0 + d) & 1) * tile_pieces;
+          const uint4* buf = NBUF == 0 ? sm_x + (c0 + d) * buf_pieces : wtile + ((c0 + d) % kBufs) * tile_pieces;
           if (NBUF == 0) {
             const uint2 h4 = reinterpret_cast<const uint2*>(buf)[xsum_off];
             const float2 f0 = __half22float2(*reinterpret_cast<const __half2*>(&h4.x));
@@ -799,7 +811,7 @@ cudaError_t launch(const MultiArgs& a, cudaStream_t stream) {
   const int ngroups = a.K / 128;
   const int nchunks = (ngroups + kChunkGroups - 1) / kChunkGroups;
   const size_t smem = 64 + (size_t)kRows * ngroups * 3 + (size_t)kWarps * NB * 128 * 4 + (size_t)kRows * TP * 4 +
-                      (NBUF == 0 ? (size_t)nchunks * a.M * kRowPitch : (size_t)kWarps * 2 * a.M * kTilePitch) * 16;
+                      (NBUF == 0 ? (size_t)nchunks * a.M * kRowPitch : (size_t)kWarps * NBUF * a.M * kTilePitch) * 16;
   if (smem > 48 * 1024) {
     cudaError_t e = cudaFuncSetAttribute(decode_kernel<BITS, TP, BF16, NBUF>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -840,8 +852,8 @@ cudaError_t launch_tp(const MultiArgs& a, cudaStream_t stream) {
   if (a.M == 1) return launch_buf<BITS, 1, BF16, 2>(a, stream);
   if (a.M <= 4) return launch_buf<BITS, 4, BF16, 2>(a, stream);
   if (a.M <= 8) return launch_buf<BITS, 8, BF16, 2>(a, stream);
-  if (a.M <= 16) return launch_buf<BITS, 16, BF16, 2>(a, stream);
-  return launch_buf<BITS, 32, BF16, 2>(a, stream);
+  if (a.M <= 16) return launch_buf<BITS, 16, BF16, 3>(a, stream);
+  return launch_buf<BITS, 32, BF16, 3>(a, stream);
 }
 
 }  // namespace
