@@ -830,7 +830,17 @@ cudaError_t launch(const MultiArgs& a, cudaStream_t stream) {
   return cudaLaunchKernelEx(&cfg, decode_kernel<BITS, TP, BF16, NBUF>, a);
 }
 
-// ring depth used when the activations do not fit up front
+// shared memory of a CTA with a ring of `bufs` activation tiles per warp
+template <int TP>
+size_t ring_smem(int K, int M, int bufs) {
+  constexpr int NB = TP <= 8 ? 1 : TP / 8;
+  return 64 + (size_t)kRows * (K / 128) * 3 + (size_t)kWarps * NB * 128 * 4 + (size_t)kRows * TP * 4 +
+         (size_t)kWarps * bufs * M * kTilePitch * 16;
+}
+constexpr size_t kSmemPerCta = 227 * 1024;
+
+// RING = ring depth used when the activations do not fit up front (one buffer less when the tables of a very wide
+// layer leave no room for it)
 template <int BITS, int TP, bool BF16, int RING>
 cudaError_t launch_buf(const MultiArgs& a, cudaStream_t stream) {
   const int nchunks = (a.K / 128 + kChunkGroups - 1) / kChunkGroups;
@@ -838,12 +848,14 @@ cudaError_t launch_buf(const MultiArgs& a, cudaStream_t stream) {
   // SM, which pays off as long as the whole grid is resident at that rate
   const size_t lim = a.first_block[a.count] <= 2 * a.sm_count ? kStageAllLimitSmallGrid : kStageAllLimit;
   if (TP <= 8 && (size_t)nchunks * a.M * kRowPitch * 16 <= lim) return launch<BITS, TP, BF16, 0>(a, stream);
+  if (ring_smem<TP>(a.K, a.M, 2) > kSmemPerCta) return cudaErrorInvalidConfiguration;   // nothing launched yet
   if (TP > 1) {   // ring mode gathers the outliers' activations from a token-major copy
     if (!a.xt || !a.xg) return cudaErrorInvalidValue;
     tokens_to_columns<TP, BF16><<<a.K / 128, 128, 0, stream>>>(a.x, const_cast<uint16_t*>(a.xt), const_cast<float*>(a.xg), a.M, a.K);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
   }
+  if (RING > 2 && ring_smem<TP>(a.K, a.M, RING) > kSmemPerCta) return launch<BITS, TP, BF16, 2>(a, stream);
   return launch<BITS, TP, BF16, RING>(a, stream);
 }
 
@@ -908,7 +920,7 @@ gwq_status gwq_launch_decode_multi(const gwq_packed* const* P, int count, const 
   else e = (xd == GWQ_BF16) ? launch_tp<3, true>(a, stream) : launch_tp<3, false>(a, stream);
   if (e != cudaSuccess) {
     (void)cudaGetLastError();
-    return GWQ_ERR_CUDA;
+    return e == cudaErrorInvalidConfiguration ? GWQ_ERR_UNSUPPORTED : GWQ_ERR_CUDA;   // too wide for shared memory
   }
   return GWQ_OK;
 }

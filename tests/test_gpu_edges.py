@@ -30,7 +30,13 @@ def _check(N, K, frac, bits, group, seed, cases):
 
 def test_largest_k_with_16_bit_outlier_columns():
     # K = 65536: the last K the streaming and tensor-core kernels take (outlier columns in 16 bits)
-    _check(40, 65536, 0.01, 4, 128, 70, [(1, "f16"), (16, "bf16"), (64, "f16")])
+    _check(40, 65536, 0.01, 4, 128, 70, [(1, "f16"), (16, "bf16"), (32, "f16"), (64, "f16")])
+
+
+def test_wide_layers_at_32_tokens():
+    # the tables of a wide layer and the activation tiles of 32 tokens compete for shared memory
+    _check(48, 16384, 0.01, 3, 128, 78, [(32, "f16"), (17, "bf16")])
+    _check(48, 32768, 0.01, 4, 128, 79, [(32, "bf16")])
 
 
 def test_k_beyond_16_bit_columns_takes_the_general_kernel():
