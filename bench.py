@@ -3,7 +3,8 @@
 
 One "step" is one pass of gwq_linear over the Llama-7B-shaped decode layer set
 (7 projections, each packed to 4 and to 3 bits, group 128, 1 % outliers) at
-M = 1, 4 and 16 tokens: 42 launches, replayed as one CUDA graph.  The headline
+M = 1, 4 and 16 tokens: 42 products in 24 calls (sibling projections share a call),
+replayed as one CUDA graph.  The headline
 value is the HBM rate over the algorithmic bytes of that step.  Beside it the
 line reports per-layer decode times, the tensor-core prefill cases, the encode
 kernels, a dense fp16 GEMM (torch.matmul, a library call) on the unquantized
