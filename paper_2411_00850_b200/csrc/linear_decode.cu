@@ -421,16 +421,18 @@ __global__ void __launch_bounds__(kThreads, TP <= 8 ? 3 : (TP == 16 ? 2 : 1)) de
   }
   // ---- from here on x is read
   pdl_wait();
-  // NBUF == 0: copy of chunk c of the activations into its buffer, by the whole CTA
-  auto stage_chunk = [&](int c) {
-    const int col0 = c * kChunkGroups * 128;
-    const int pieces = min(kChunkPieces, (p.K - col0) >> 3);
-    uint4* buf = sm_x + c * buf_pieces;
-    for (int i = tid; i < p.M * kChunkPieces; i += kThreads) {
-      const int m = i / kChunkPieces, pc = i - m * kChunkPieces;   // kChunkPieces is a power of two
-      if (pc < pieces) {
-        const unsigned dst = (unsigned)__cvta_generic_to_shared(buf + xs_piece(pc, m));
-        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(p.x + (size_t)m * p.K + col0 + pc * 8));
+  // NBUF == 0: copy of all activations into the chunk buffers, by the whole CTA: token row by token row, piece pc of a
+  // row goes to chunk pc / 128, place xs_piece(pc % 128, m) (few instructions per piece: this runs in every CTA)
+  auto stage_all = [&]() {
+    const int ppr = p.K >> 3;   // 16-byte pieces per token row
+    const unsigned base = (unsigned)__cvta_generic_to_shared(sm_x);
+    for (int m = 0; m < p.M; ++m) {
+      const uint16_t* src = p.x + (size_t)m * p.K;
+      const unsigned dst0 = base + (unsigned)(m * kRowPitch + ((m & 1) << 1)) * 16u;
+      for (int pc = tid; pc < ppr; pc += kThreads) {
+        const int c = pc >> 7, q = pc & (kChunkPieces - 1);
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst0 + (unsigned)(c * buf_pieces + q + (q >> 3)) * 16u),
+                     "l"(src + pc * 8));
       }
     }
   };
@@ -455,7 +457,7 @@ __global__ void __launch_bounds__(kThreads, TP <= 8 ? 3 : (TP == 16 ? 2 : 1)) de
     }
   };
   if (NBUF == 0) {
-    for (int c = 0; c < nchunks; ++c) stage_chunk(c);
+    stage_all();
   } else {
     stage_tile(0);
   }
