@@ -356,6 +356,8 @@ def run_cuda_arm(args):
         for L in layers:
             L["W"] = None
             L["G"] = None
+        if not args.skip_70b:
+            out["decode_cases_70b"] = bench_decode_70b(torch, gwq, dev, max(3, detail_iters // 2), hbm_peak)
         out["prefill"] = bench_prefill(torch, gwq, dev, args, tf_burst, tf_sust)
         best = max(out["prefill"], key=lambda r: r["tflops"])
         out["prefill_roofline"] = {"bound": "tensor", "kernel": "gwq prefill linear (tcgen05)",
@@ -419,6 +421,59 @@ def bench_decode_detail(torch, gwq, layers, xs, ys, iters, hbm_peak):
                              "gbs": round(b / us / 1e3, 1), "frac_measured_peak": round(b / us / 1e3 / hbm_peak, 4),
                              "frac_8TBs": round(b / us / 1e3 / 8000.0, 4), "launches_in_graph": len(members),
                              "read_only_launch_us": round(floor_us, 3), "x_read_only": round(us / floor_us, 2)})
+    del scrub
+    return rows
+
+
+def bench_decode_70b(torch, gwq, dev, iters, hbm_peak, Ms=(1, 8, 32)):
+    """Llama-70B-shaped layers (8192 x 8192, 28672 x 8192, 8192 x 28672), 4 and 3 bits, group 128, 1 % outliers:
+    microseconds per launch with a cold L2, as in `bench_decode_detail`.  A layer is 31 to 137 MB of packed data,
+    so the fixed cost of a launch weighs little here and the figure shows what the kernel itself sustains."""
+    rows = []
+    scrub = torch.zeros(64 * 1024 * 1024, dtype=torch.int32, device=dev)
+    for si, (N, K) in enumerate(synth.LLAMA70B_SHAPES):
+        W, G = synth.make_weight_and_grad(N, K, synth.layer_seed(4, si))
+        Wd, Gd = torch.from_numpy(W).to(dev), torch.from_numpy(G).to(dev)
+        del W, G
+        xs = {}
+        for M in Ms:
+            bits16, _ = synth.make_activations(M, K, seed=synth.layer_seed(4, si), dtype="f16")
+            xs[M] = torch.from_numpy(bits16.view(np.int16).copy()).to(dev).view(torch.float16)
+        for bits in BIT_WIDTHS:
+            copies = 4 if N * K < 100_000_000 else 2     # more than the 126 MB L2 between reuses
+            packed = [gwq.gwq_pack(Wd, gwq.gwq_select_outliers(Wd, Gd, FRAC), bits, GROUP) for _ in range(copies)]
+            nnz = packed[0].nnz
+
+            def probe():
+                for P in packed:
+                    gwq.gwq_read_probe(P)
+            replay_probe = capture(torch, probe)
+            floor_ms = None
+            for _ in range(iters):
+                int(scrub.sum().item())
+                ms = time_region(torch, lambda i: replay_probe(), 1)
+                floor_ms = ms if floor_ms is None else min(floor_ms, ms)
+            floor_us = floor_ms * 1e3 / copies
+            for M in Ms:
+                y = torch.empty((M, N), dtype=torch.float16, device=dev)
+
+                def run():
+                    for P in packed:
+                        gwq.gwq_linear(P, xs[M], out=y)
+                replay = capture(torch, run)
+                best = None
+                for _ in range(iters):
+                    int(scrub.sum().item())
+                    ms = time_region(torch, lambda i: replay(), 1)
+                    best = ms if best is None else min(best, ms)
+                us = best * 1e3 / copies
+                b = algorithmic_bytes(N, K, bits, GROUP, nnz, M)
+                rows.append({"N": N, "K": K, "bits": bits, "M": M, "us": round(us, 3), "bytes": b,
+                             "gbs": round(b / us / 1e3, 1), "frac_measured_peak": round(b / us / 1e3 / hbm_peak, 4),
+                             "frac_8TBs": round(b / us / 1e3 / 8000.0, 4), "launches_in_graph": copies,
+                             "read_only_launch_us": round(floor_us, 3), "x_read_only": round(us / floor_us, 2)})
+            del packed
+        del Wd, Gd
     del scrub
     return rows
 
@@ -643,6 +698,7 @@ def main():
     ap.add_argument("--prefill-iters", type=int, default=5)
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--headline-only", action="store_true", help="skip the per-case detail sections")
+    ap.add_argument("--skip-70b", action="store_true", help="skip the Llama-70B-shaped decode cases")
     ap.add_argument("--no-fuse", action="store_true",
                     help="launch sibling projections as separate concurrent calls instead of one gwq_linear_multi")
     args = ap.parse_args()
