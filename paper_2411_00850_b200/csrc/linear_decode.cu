@@ -30,6 +30,7 @@ constexpr int kWarps = 8;
 constexpr int kThreads = kWarps * 32;
 constexpr int kRows = 16;   // rows per CTA (one m16 tile)
 constexpr int kDepth = 4;   // groups of codes in flight per warp
+constexpr int kMaxTokens64 = 8;   // groups of 64: tokens one launch takes
 
 template <bool BF16>
 __device__ __forceinline__ void mma16816(float (&d)[4], unsigned a0, unsigned a1, unsigned a2, unsigned a3,
@@ -312,8 +313,18 @@ constexpr int kTilePitch = 16;   // pieces per token row of a warp tile: no padd
 // piece p (16 bytes) of token row m of a warp tile: the XOR keeps the four lanes of a quad and four neighbouring
 // token rows in different 16-byte bank groups
 __device__ __forceinline__ int tile_piece(int pc, int m) { return m * kTilePitch + (pc ^ (pc >> 3) ^ ((m & 3) << 1)); }
-template <int BITS, int TP, bool BF16, int NBUF>
-__global__ void __launch_bounds__(kThreads, TP <= 8 ? 3 : (TP == 16 ? 2 : 1)) decode_kernel(const MultiArgs ma) {
+// G64: groups of 64 columns.  A warp step still covers 128 columns, i.e. two groups: the runs of lanes t = 0, 1 belong
+// to the first, those of t = 2, 3 to the second.  An MMA sums over all four lanes, so the two groups are kept apart on
+// the token side: a token block holds 4 tokens, output column n < 4 is token n with the activations of the second
+// group replaced by zeros (lanes t >= 2 read the zero page), column n >= 4 is token n - 4 with those of the first
+// group replaced by zeros.  Accumulator columns 2t, 2t+1 of lane t then belong to the lane's own group (t >> 1), whose
+// scale and zero-point it applies; the two halves of a token meet in the final sum.  Sums of x always come from the
+// all-ones MMA here.  TP <= 8.
+template <int TP, bool G64>
+struct TokenBlocks { static constexpr int value = G64 ? (TP <= 4 ? 1 : TP / 4) : (TP <= 8 ? 1 : TP / 8); };
+template <int BITS, int TP, bool BF16, int NBUF, bool G64>
+__global__ void __launch_bounds__(kThreads, TokenBlocks<TP, G64>::value == 1 ? 3 : (TokenBlocks<TP, G64>::value == 2 ? 2 : 1))
+decode_kernel(const MultiArgs ma) {
   // the layer this CTA works for and its row block inside that layer
   DecodeArgs p;
   int blk = blockIdx.x;
@@ -332,18 +343,19 @@ __global__ void __launch_bounds__(kThreads, TP <= 8 ? 3 : (TP == 16 ? 2 : 1)) de
     }
     p.x = ma.x; p.xt = ma.xt; p.xg = ma.xg; p.yd = ma.yd; p.K = ma.K; p.M = ma.M;
   }
-  constexpr int NB = TP <= 8 ? 1 : TP / 8;   // 8-token blocks of the MMA
+  constexpr int NB = TokenBlocks<TP, G64>::value;   // token blocks of the MMA (8 tokens; 4 with groups of 64)
   constexpr int WPR = BITS;                   // words per run of 32 columns
   // raw path: sum_k x_k of a group from shared memory (one token), from the table that comes with the
   // token-major copy (ring mode), else from a second MMA with an all-ones A operand
-  constexpr bool ONES = !BF16 && TP != 1 && NBUF == 0;
+  constexpr bool ONES = !BF16 && (G64 || (TP != 1 && NBUF == 0));
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  const int ngroups = p.K >> 7;
+  const int ngroups = p.K >> 7;               // warp steps of 128 columns in a row
+  const int ntab = G64 ? 2 * ngroups : ngroups;   // scale / zero-point entries in a row
   // shared: zero page 64 B | scales [16][ngroups] f16 | zeros [16][ngroups] u8 | red [kWarps][NB][16][8] f32 |
   //         outl [16][TP] f32 | x chunk buffers 2 x [M][kRowPitch] pieces
   uint16_t* sm_s = reinterpret_cast<uint16_t*>(smem_raw + 64);
-  uint8_t* sm_z = reinterpret_cast<uint8_t*>(sm_s + kRows * ngroups);
-  float* sm_red = reinterpret_cast<float*>(sm_z + kRows * ngroups);
+  uint8_t* sm_z = reinterpret_cast<uint8_t*>(sm_s + kRows * ntab);
+  float* sm_red = reinterpret_cast<float*>(sm_z + kRows * ntab);
   float* sm_out = sm_red + kWarps * NB * 128;
   uint4* sm_x = reinterpret_cast<uint4*>(sm_out + kRows * TP);
   const int buf_pieces = p.M * kRowPitch;
@@ -368,20 +380,20 @@ __global__ void __launch_bounds__(kThreads, TP <= 8 ? 3 : (TP == 16 ? 2 : 1)) de
   {
     // scales and zero-points of the 16 rows: two contiguous, 16-byte aligned ranges
     const int rows_here = min(kRows, p.N - r0);
-    const char* gs = reinterpret_cast<const char*>(p.scales + (size_t)r0 * ngroups);
-    const char* gz = reinterpret_cast<const char*>(p.zeros + (size_t)r0 * ngroups);
+    const char* gs = reinterpret_cast<const char*>(p.scales + (size_t)r0 * ntab);
+    const char* gz = reinterpret_cast<const char*>(p.zeros + (size_t)r0 * ntab);
     if (rows_here == kRows) {
-      for (int c = tid; c < 3 * ngroups; c += kThreads) {   // 32 ng + 16 ng bytes = 3 ng pieces
-        const bool is_s = c < 2 * ngroups;
-        const char* src = is_s ? gs + c * 16 : gz + (c - 2 * ngroups) * 16;
+      for (int c = tid; c < 3 * ntab; c += kThreads) {   // 32 ng + 16 ng bytes = 3 ng pieces
+        const bool is_s = c < 2 * ntab;
+        const char* src = is_s ? gs + c * 16 : gz + (c - 2 * ntab) * 16;
         const unsigned dst = (unsigned)__cvta_generic_to_shared(reinterpret_cast<char*>(sm_s) + c * 16);
         asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src));
       }
     } else {   // last, partial CTA: rows past N read as scale 0
-      for (int i = tid; i < kRows * ngroups; i += kThreads) {
-        const bool live = i < rows_here * ngroups;
-        sm_s[i] = live ? p.scales[(size_t)r0 * ngroups + i] : (uint16_t)0;
-        sm_z[i] = live ? p.zeros[(size_t)r0 * ngroups + i] : (uint8_t)0;
+      for (int i = tid; i < kRows * ntab; i += kThreads) {
+        const bool live = i < rows_here * ntab;
+        sm_s[i] = live ? p.scales[(size_t)r0 * ntab + i] : (uint16_t)0;
+        sm_z[i] = live ? p.zeros[(size_t)r0 * ntab + i] : (uint8_t)0;
       }
     }
   }
@@ -547,13 +559,15 @@ __global__ void __launch_bounds__(kThreads, TP <= 8 ? 3 : (TP == 16 ? 2 : 1)) de
   int xoff[NB], xcx[NB];
 #pragma unroll
   for (int nb = 0; nb < NB; ++nb) {
-    const int m = nb * 8 + gid;
-    xoff[nb] = m >= p.M ? -1 : (NBUF == 0 ? xs_piece(warp * 16 + t * 4, m) : m * kTilePitch + ((t ^ ((m >> 1) & 1)) << 2));
-    xcx[nb] = (NBUF == 0 || m >= p.M) ? 0 : ((t >> 1) ^ ((m & 1) << 1));
+    const int m = G64 ? nb * 4 + (gid & 3) : nb * 8 + gid;
+    const bool live = m < p.M && (!G64 || (gid >> 2) == (t >> 1));   // groups of 64: the other group's columns read as zero
+    xoff[nb] = !live ? -1 : (NBUF == 0 ? xs_piece(warp * 16 + t * 4, m) : m * kTilePitch + ((t ^ ((m >> 1) & 1)) << 2));
+    xcx[nb] = (NBUF == 0 || !live) ? 0 : ((t >> 1) ^ ((m & 1) << 1));
   }
-  const uint16_t* sp = sm_s + gid * ngroups + warp;   // scale / zero-point of row gid, group `warp`
-  const uint8_t* zp = sm_z + gid * ngroups + warp;
-  const int hi_row = 8 * ngroups;
+  // scale / zero-point of row gid, group `warp` (groups of 64: the lane's own half of step `warp`)
+  const uint16_t* sp = sm_s + gid * ntab + (G64 ? 2 * warp + (t >> 1) : warp);
+  const uint8_t* zp = sm_z + gid * ntab + (G64 ? 2 * warp + (t >> 1) : warp);
+  const int hi_row = 8 * ntab;
   const int xsum_off = (NBUF == 0 ? xs_piece(warp * 16 + (lane >> 1), 0) : ((lane >> 1) ^ (lane >> 4))) * 2 + (lane & 1);   // 8-byte units, token 0
 
   float yacc[NB][4];
@@ -592,8 +606,8 @@ __global__ void __launch_bounds__(kThreads, TP <= 8 ? 3 : (TP == 16 ? 2 : 1)) de
       {
         const float sa = __half2float(__ushort_as_half(sp[0])), sb = __half2float(__ushort_as_half(sp[hi_row]));
         const unsigned za = zp[0], zb = zp[hi_row];
-        sp += kWarps;
-        zp += kWarps;
+        sp += G64 ? 2 * kWarps : kWarps;
+        zp += G64 ? 2 * kWarps : kWarps;
         if (BF16) {
           ta = make_float2(sa, __uint_as_float(0x43004300u | (za * 0x00010001u)));
           tb = make_float2(sb, __uint_as_float(0x43004300u | (zb * 0x00010001u)));
@@ -611,7 +625,7 @@ __global__ void __launch_bounds__(kThreads, TP <= 8 ? 3 : (TP == 16 ? 2 : 1)) de
           xg2[nb] = __ldg(reinterpret_cast<const float2*>(p.xg + (size_t)(warp + kWarps * c) * TP + nb * 8 + 2 * t));
       }
       float xsum1 = xsum_in;
-      if (!BF16 && TP == 1 && checked) {   // one token: sum_k x_k of the group, lane L adding columns 4L..4L+3
+      if (!BF16 && !ONES && TP == 1 && checked) {   // one token: sum_k x_k of the group, lane L adding columns 4L..4L+3
         const uint2 h4 = reinterpret_cast<const uint2*>(buf)[xsum_off];
         const float2 f0 = __half22float2(*reinterpret_cast<const __half2*>(&h4.x));
         const float2 f1 = __half22float2(*reinterpret_cast<const __half2*>(&h4.y));
@@ -671,7 +685,7 @@ __global__ void __launch_bounds__(kThreads, TP <= 8 ? 3 : (TP == 16 ? 2 : 1)) de
     if (c0 + kDepth <= nsteps) {
       // four full steps of this warp: branch-free, the single token's four group sums reduced together
       float xs4[kDepth] = {0.f, 0.f, 0.f, 0.f};
-      if (!BF16 && TP == 1) {
+      if (!BF16 && !ONES && TP == 1) {
 #pragma unroll
         for (int d = 0; d < kDepth; ++d) {
           const uint4* buf = NBUF == 0 ? sm_x + (c0 + d) * buf_pieces : wtile + ((c0 + d) % kBufs) * tile_pieces;
@@ -761,10 +775,13 @@ __global__ void __launch_bounds__(kThreads, TP <= 8 ? 3 : (TP == 16 ? 2 : 1)) de
     const int lr = o & 15, m = o >> 4;
     const int row = r0 + lr;
     if (row < p.N) {
-      const int nb = m >> 3, tk = m & 7;
+      const int nb = G64 ? m >> 2 : m >> 3, tk = G64 ? m & 3 : m & 7;
       float v = sm_out[lr * TP + m];
 #pragma unroll
-      for (int w = 0; w < kWarps; ++w) v += sm_red[(w * NB + nb) * 128 + lr * 8 + tk];
+      for (int w = 0; w < kWarps; ++w) {
+        v += sm_red[(w * NB + nb) * 128 + lr * 8 + tk];
+        if (G64) v += sm_red[(w * NB + nb) * 128 + lr * 8 + tk + 4];   // the token's second group of every step
+      }
       store_y(p.y, p.yd, (long long)m * p.N + row, v);
     }
   }
@@ -807,15 +824,15 @@ __global__ void __launch_bounds__(128) tokens_to_columns(const uint16_t* __restr
 constexpr size_t kStageAllLimit = 72 * 1024;   // stage every chunk up front when it fits in this much
 constexpr size_t kStageAllLimitSmallGrid = 80 * 1024;   // the same for grids of at most two CTAs per SM
 
-template <int BITS, int TP, bool BF16, int NBUF>
+template <int BITS, int TP, bool BF16, int NBUF, bool G64>
 cudaError_t launch(const MultiArgs& a, cudaStream_t stream) {
-  constexpr int NB = TP <= 8 ? 1 : TP / 8;
+  constexpr int NB = TokenBlocks<TP, G64>::value;
   const int ngroups = a.K / 128;
   const int nchunks = (ngroups + kChunkGroups - 1) / kChunkGroups;
-  const size_t smem = 64 + (size_t)kRows * ngroups * 3 + (size_t)kWarps * NB * 128 * 4 + (size_t)kRows * TP * 4 +
+  const size_t smem = 64 + (size_t)kRows * (G64 ? 2 * ngroups : ngroups) * 3 + (size_t)kWarps * NB * 128 * 4 + (size_t)kRows * TP * 4 +
                       (NBUF == 0 ? (size_t)nchunks * a.M * kRowPitch : (size_t)kWarps * NBUF * a.M * kTilePitch) * 16;
   if (smem > 48 * 1024) {
-    cudaError_t e = cudaFuncSetAttribute(decode_kernel<BITS, TP, BF16, NBUF>,
+    cudaError_t e = cudaFuncSetAttribute(decode_kernel<BITS, TP, BF16, NBUF, G64>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
   }
@@ -829,58 +846,68 @@ cudaError_t launch(const MultiArgs& a, cudaStream_t stream) {
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, decode_kernel<BITS, TP, BF16, NBUF>, a);
+  return cudaLaunchKernelEx(&cfg, decode_kernel<BITS, TP, BF16, NBUF, G64>, a);
 }
 
 // shared memory of a CTA with a ring of `bufs` activation tiles per warp
-template <int TP>
+template <int TP, bool G64>
 size_t ring_smem(int K, int M, int bufs) {
-  constexpr int NB = TP <= 8 ? 1 : TP / 8;
-  return 64 + (size_t)kRows * (K / 128) * 3 + (size_t)kWarps * NB * 128 * 4 + (size_t)kRows * TP * 4 +
+  constexpr int NB = TokenBlocks<TP, G64>::value;
+  return 64 + (size_t)kRows * (K / (G64 ? 64 : 128)) * 3 + (size_t)kWarps * NB * 128 * 4 + (size_t)kRows * TP * 4 +
          (size_t)kWarps * bufs * M * kTilePitch * 16;
 }
 constexpr size_t kSmemPerCta = 227 * 1024;
 
 // RING = ring depth used when the activations do not fit up front (one buffer less when the tables of a very wide
 // layer leave no room for it)
-template <int BITS, int TP, bool BF16, int RING>
+template <int BITS, int TP, bool BF16, int RING, bool G64>
 cudaError_t launch_buf(const MultiArgs& a, cudaStream_t stream) {
   const int nchunks = (a.K / 128 + kChunkGroups - 1) / kChunkGroups;
   // staging everything up front costs shared memory, hence resident CTAs: beyond kStageAllLimit only two fit on an
   // SM, which pays off as long as the whole grid is resident at that rate
   const size_t lim = a.first_block[a.count] <= 2 * a.sm_count ? kStageAllLimitSmallGrid : kStageAllLimit;
-  if (TP <= 8 && (size_t)nchunks * a.M * kRowPitch * 16 <= lim) return launch<BITS, TP, BF16, 0>(a, stream);
-  if (ring_smem<TP>(a.K, a.M, 2) > kSmemPerCta) return cudaErrorInvalidConfiguration;   // nothing launched yet
+  if (TP <= 8 && (size_t)nchunks * a.M * kRowPitch * 16 <= lim) return launch<BITS, TP, BF16, 0, G64>(a, stream);
+  if (ring_smem<TP, G64>(a.K, a.M, 2) > kSmemPerCta) return cudaErrorInvalidConfiguration;   // nothing launched yet
   if (TP > 1) {   // ring mode gathers the outliers' activations from a token-major copy
     if (!a.xt || !a.xg) return cudaErrorInvalidValue;
     tokens_to_columns<TP, BF16><<<a.K / 128, 128, 0, stream>>>(a.x, const_cast<uint16_t*>(a.xt), const_cast<float*>(a.xg), a.M, a.K);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
   }
-  if (RING > 2 && ring_smem<TP>(a.K, a.M, RING) > kSmemPerCta) return launch<BITS, TP, BF16, 2>(a, stream);
-  return launch<BITS, TP, BF16, RING>(a, stream);
+  if (RING > 2 && ring_smem<TP, G64>(a.K, a.M, RING) > kSmemPerCta) return launch<BITS, TP, BF16, 2, G64>(a, stream);
+  return launch<BITS, TP, BF16, RING, G64>(a, stream);
 }
 
 template <int BITS, bool BF16>
 cudaError_t launch_tp(const MultiArgs& a, cudaStream_t stream) {
-  if (a.M == 1) return launch_buf<BITS, 1, BF16, 2>(a, stream);
-  if (a.M <= 4) return launch_buf<BITS, 4, BF16, 2>(a, stream);
-  if (a.M <= 8) return launch_buf<BITS, 8, BF16, 2>(a, stream);
-  if (a.M <= 16) return launch_buf<BITS, 16, BF16, 3>(a, stream);
-  return launch_buf<BITS, 32, BF16, 3>(a, stream);
+  if (a.M == 1) return launch_buf<BITS, 1, BF16, 2, false>(a, stream);
+  if (a.M <= 4) return launch_buf<BITS, 4, BF16, 2, false>(a, stream);
+  if (a.M <= 8) return launch_buf<BITS, 8, BF16, 2, false>(a, stream);
+  if (a.M <= 16) return launch_buf<BITS, 16, BF16, 3, false>(a, stream);
+  return launch_buf<BITS, 32, BF16, 3, false>(a, stream);
+}
+
+// groups of 64: up to 8 tokens (two blocks of 4)
+template <int BITS, bool BF16>
+cudaError_t launch_tp64(const MultiArgs& a, cudaStream_t stream) {
+  if (a.M == 1) return launch_buf<BITS, 1, BF16, 2, true>(a, stream);
+  if (a.M <= 4) return launch_buf<BITS, 4, BF16, 2, true>(a, stream);
+  return launch_buf<BITS, 8, BF16, 2, true>(a, stream);
 }
 
 }  // namespace
 
-// Decode launcher for `count` layers that read the same x: group size 128, M <= 32, K <= 65536, same K and bit
+// Decode launcher for `count` layers that read the same x: group size 128 (M <= 32) or 64 (M <= 8), K <= 65536, same K and bit
 // width in every layer.  Returns GWQ_ERR_UNSUPPORTED for anything else (nothing has been launched then).
 // The scratch for the token-major copy of x is the first layer's.
 gwq_status gwq_launch_decode_multi(const gwq_packed* const* P, int count, const void* x, gwq_dtype xd, int M,
                                    void* const* y, gwq_dtype yd, cudaStream_t stream) {
   if (count < 1 || count > kMaxLayers || M > 32) return GWQ_ERR_UNSUPPORTED;
+  const bool g64 = P[0]->group == 64;
+  if (g64 && (M > kMaxTokens64 || P[0]->K % 128 != 0)) return GWQ_ERR_UNSUPPORTED;   // a warp step is 128 columns
   for (int i = 0; i < count; ++i) {
     const gwq_priv* pvi = static_cast<const gwq_priv*>(P[i]->priv);
-    if (P[i]->group != 128 || !pvi->cv || P[i]->K != P[0]->K || P[i]->bits != P[0]->bits) return GWQ_ERR_UNSUPPORTED;
+    if ((P[i]->group != 128 && P[i]->group != 64) || P[i]->group != P[0]->group || !pvi->cv || P[i]->K != P[0]->K || P[i]->bits != P[0]->bits) return GWQ_ERR_UNSUPPORTED;
   }
   gwq_priv* pv = static_cast<gwq_priv*>(P[0]->priv);
   MultiArgs a;
@@ -918,7 +945,10 @@ gwq_status gwq_launch_decode_multi(const gwq_packed* const* P, int count, const 
   a.sm_count = pv->sm_count > 0 ? pv->sm_count : 148;
   a.x = static_cast<const uint16_t*>(x); a.yd = yd; a.K = K; a.M = M;
   cudaError_t e;
-  if (P[0]->bits == 4) e = (xd == GWQ_BF16) ? launch_tp<4, true>(a, stream) : launch_tp<4, false>(a, stream);
+  if (g64) {
+    if (P[0]->bits == 4) e = (xd == GWQ_BF16) ? launch_tp64<4, true>(a, stream) : launch_tp64<4, false>(a, stream);
+    else e = (xd == GWQ_BF16) ? launch_tp64<3, true>(a, stream) : launch_tp64<3, false>(a, stream);
+  } else if (P[0]->bits == 4) e = (xd == GWQ_BF16) ? launch_tp<4, true>(a, stream) : launch_tp<4, false>(a, stream);
   else e = (xd == GWQ_BF16) ? launch_tp<3, true>(a, stream) : launch_tp<3, false>(a, stream);
   if (e != cudaSuccess) {
     (void)cudaGetLastError();
@@ -927,10 +957,13 @@ gwq_status gwq_launch_decode_multi(const gwq_packed* const* P, int count, const 
   return GWQ_OK;
 }
 
-// Decode launcher: group size 128, M <= 32, K <= 65536.  Other shapes go to the general kernel.
+// Decode launcher: group size 128 with M <= 32 or 64 with M <= 8, K <= 65536.  Groups of 64 with more tokens go to
+// the tensor-core kernel, other shapes to the general kernel.
 gwq_status gwq_launch_decode(const gwq_packed* P, const void* x, gwq_dtype xd, int M, void* y, gwq_dtype yd,
                              cudaStream_t stream) {
   const gwq_status st = gwq_launch_decode_multi(&P, 1, x, xd, M, &y, yd, stream);
   if (st != GWQ_ERR_UNSUPPORTED) return st;
+  // groups of 64 beyond the tokens the streaming kernel takes: the tensor-core kernel with its smallest token tile
+  if (P->group == 64 && M > kMaxTokens64) return gwq_launch_prefill(P, x, xd, M, y, yd, stream);
   return gwq_launch_simt(P, x, xd, M, y, yd, stream);
 }

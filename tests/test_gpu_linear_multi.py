@@ -52,6 +52,21 @@ def test_fused_siblings_match_checker_and_single_calls(bits, M, dtype):
         assert gwq.gwq_device_status(P) == 0
 
 
+@pytest.mark.parametrize("bits", [4, 3])
+@pytest.mark.parametrize("M,dtype", [(1, "f16"), (4, "bf16"), (8, "f16"), (12, "f16")])
+def test_fused_siblings_with_groups_of_64(bits, M, dtype):
+    # one launch up to 8 tokens; beyond, one launch per layer on the tensor-core kernel
+    sib = [_layer(N, 2176, 0.01, bits, 64, 50 + i) for i, N in enumerate((200, 72))]
+    Ps = [s[0] for s in sib]
+    bits16, xv = synth.make_activations(M, 2176, seed=200 + M, dtype=dtype)
+    x = x_tensor(bits16, dtype)
+    ys = gwq.gwq_linear_multi(Ps, x, out_dtype=torch.float32)
+    for (P, L, w_hat), y in zip(sib, ys):
+        y_ref, bound = orc.linear(xv, w_hat)
+        assert_linear_close(y, y_ref, bound)
+        assert torch.equal(y, gwq.gwq_linear(P, x, out_dtype=torch.float32))
+
+
 def test_two_and_four_layers_and_16_bit_outputs():
     sib = _siblings(4) + [_layer(48, 1024, 0.02, 4, 128, 47)]
     bits16, xv = synth.make_activations(4, 1024, seed=7, dtype="f16")
@@ -65,7 +80,7 @@ def test_two_and_four_layers_and_16_bit_outputs():
 
 
 def test_layers_that_cannot_share_a_launch_still_give_every_product():
-    # different bit widths, a group of 64, and M > 32: the call falls back to one launch per layer
+    # different bit widths, differing group sizes, and M > 32: the call falls back to one launch per layer
     a = _layer(200, 1024, 0.01, 4, 128, 40)
     b = _layer(72, 1024, 0.01, 3, 128, 41)
     c = _layer(96, 1024, 0.01, 4, 64, 48)
