@@ -222,8 +222,7 @@ __device__ __forceinline__ float act_to_float(uint16_t b) {
 
 struct DecodeArgs {
   const uint32_t* codes;
-  const uint16_t* scales;
-  const uint8_t* zeros;
+  const uint32_t* szt;   // [K / group][N]: scale (fp16 bits) | zero-point << 16
   const int32_t* row_ptr;
   const uint32_t* cv;  // per outlier: fp16 value << 16 | column
   const uint16_t* x;
@@ -239,8 +238,7 @@ struct DecodeArgs {
 constexpr int kMaxLayers = GWQ_MULTI_MAX;
 struct LayerArgs {
   const uint32_t* codes;
-  const uint16_t* scales;
-  const uint8_t* zeros;
+  const uint32_t* szt;
   const int32_t* row_ptr;
   const uint32_t* cv;
   void* y;
@@ -336,7 +334,7 @@ decode_kernel(const MultiArgs ma) {
 #pragma unroll
     for (int i = 0; i < kMaxLayers; ++i) {
       if (i == l) {
-        p.codes = ma.layer[i].codes; p.scales = ma.layer[i].scales; p.zeros = ma.layer[i].zeros;
+        p.codes = ma.layer[i].codes; p.szt = ma.layer[i].szt;
         p.row_ptr = ma.layer[i].row_ptr; p.cv = ma.layer[i].cv; p.y = ma.layer[i].y; p.N = ma.layer[i].N;
         blk = (int)blockIdx.x - ma.first_block[i];
       }
@@ -351,11 +349,12 @@ decode_kernel(const MultiArgs ma) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int ngroups = p.K >> 7;               // warp steps of 128 columns in a row
   const int ntab = G64 ? 2 * ngroups : ngroups;   // scale / zero-point entries in a row
-  // shared: zero page 64 B | scales [16][ngroups] f16 | zeros [16][ngroups] u8 | red [kWarps][NB][16][8] f32 |
+  // shared: zero page 64 B | scale and zero-point table [ntab][16 rows] u32 | red [kWarps][NB][16][8] f32 |
   //         outl [16][TP] f32 | x chunk buffers 2 x [M][kRowPitch] pieces
-  uint16_t* sm_s = reinterpret_cast<uint16_t*>(smem_raw + 64);
-  uint8_t* sm_z = reinterpret_cast<uint8_t*>(sm_s + kRows * ntab);
-  float* sm_red = reinterpret_cast<float*>(sm_z + kRows * ntab);
+  // (the table is group-major: the eight rows a load instruction asks for are eight neighbouring words, no bank
+  // conflicts however wide the layer is)
+  uint32_t* sm_tab = reinterpret_cast<uint32_t*>(smem_raw + 64);
+  float* sm_red = reinterpret_cast<float*>(sm_tab + kRows * ntab);
   float* sm_out = sm_red + kWarps * NB * 128;
   uint4* sm_x = reinterpret_cast<uint4*>(sm_out + kRows * TP);
   const int buf_pieces = p.M * kRowPitch;
@@ -378,22 +377,18 @@ decode_kernel(const MultiArgs ma) {
   int rp = 0;
   if (lane < 3) rp = __ldg(p.row_ptr + min(r0 + 2 * warp + lane, p.N));
   {
-    // scales and zero-points of the 16 rows: two contiguous, 16-byte aligned ranges
+    // scales and zero-points of the 16 rows: 64 contiguous bytes per group of the group-major table
     const int rows_here = min(kRows, p.N - r0);
-    const char* gs = reinterpret_cast<const char*>(p.scales + (size_t)r0 * ntab);
-    const char* gz = reinterpret_cast<const char*>(p.zeros + (size_t)r0 * ntab);
-    if (rows_here == kRows) {
-      for (int c = tid; c < 3 * ntab; c += kThreads) {   // 32 ng + 16 ng bytes = 3 ng pieces
-        const bool is_s = c < 2 * ntab;
-        const char* src = is_s ? gs + c * 16 : gz + (c - 2 * ntab) * 16;
-        const unsigned dst = (unsigned)__cvta_generic_to_shared(reinterpret_cast<char*>(sm_s) + c * 16);
-        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src));
+    if (rows_here == kRows && (p.N & 3) == 0) {
+      const unsigned dst0 = (unsigned)__cvta_generic_to_shared(sm_tab);
+      for (int c = tid; c < 4 * ntab; c += kThreads) {   // piece c: rows 4 (c & 3) .. + 3 of group c >> 2
+        const uint32_t* src = p.szt + (size_t)(c >> 2) * p.N + r0 + 4 * (c & 3);
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst0 + (unsigned)c * 16u), "l"(src));
       }
-    } else {   // last, partial CTA: rows past N read as scale 0
+    } else {   // partial last CTA, or rows that do not start on 16-byte boundaries: rows past N read as scale 0
       for (int i = tid; i < kRows * ntab; i += kThreads) {
-        const bool live = i < rows_here * ntab;
-        sm_s[i] = live ? p.scales[(size_t)r0 * ntab + i] : (uint16_t)0;
-        sm_z[i] = live ? p.zeros[(size_t)r0 * ntab + i] : (uint8_t)0;
+        const int r = i & 15, g = i >> 4;
+        sm_tab[i] = r < rows_here ? __ldg(p.szt + (size_t)g * p.N + r0 + r) : 0u;
       }
     }
   }
@@ -564,10 +559,8 @@ decode_kernel(const MultiArgs ma) {
     xoff[nb] = !live ? -1 : (NBUF == 0 ? xs_piece(warp * 16 + t * 4, m) : m * kTilePitch + ((t ^ ((m >> 1) & 1)) << 2));
     xcx[nb] = (NBUF == 0 || !live) ? 0 : ((t >> 1) ^ ((m & 1) << 1));
   }
-  // scale / zero-point of row gid, group `warp` (groups of 64: the lane's own half of step `warp`)
-  const uint16_t* sp = sm_s + gid * ntab + (G64 ? 2 * warp + (t >> 1) : warp);
-  const uint8_t* zp = sm_z + gid * ntab + (G64 ? 2 * warp + (t >> 1) : warp);
-  const int hi_row = 8 * ntab;
+  // scale | zero-point << 16 of row gid, group `warp` (groups of 64: the lane's own half of step `warp`)
+  const uint32_t* tp = sm_tab + (G64 ? 2 * warp + (t >> 1) : warp) * kRows + gid;
   const int xsum_off = (NBUF == 0 ? xs_piece(warp * 16 + (lane >> 1), 0) : ((lane >> 1) ^ (lane >> 4))) * 2 + (lane & 1);   // 8-byte units, token 0
 
   float yacc[NB][4];
@@ -604,10 +597,11 @@ decode_kernel(const MultiArgs ma) {
       // (s 2^24, s z) on the raw path, (s, magic | z) on the subtract path
       float2 ta, tb;
       {
-        const float sa = __half2float(__ushort_as_half(sp[0])), sb = __half2float(__ushort_as_half(sp[hi_row]));
-        const unsigned za = zp[0], zb = zp[hi_row];
-        sp += G64 ? 2 * kWarps : kWarps;
-        zp += G64 ? 2 * kWarps : kWarps;
+        const unsigned sza = tp[0], szb = tp[8];
+        tp += (G64 ? 2 * kWarps : kWarps) * kRows;
+        const float sa = __half2float(__ushort_as_half((unsigned short)sza));
+        const float sb = __half2float(__ushort_as_half((unsigned short)szb));
+        const unsigned za = sza >> 16, zb = szb >> 16;
         if (BF16) {
           ta = make_float2(sa, __uint_as_float(0x43004300u | (za * 0x00010001u)));
           tb = make_float2(sb, __uint_as_float(0x43004300u | (zb * 0x00010001u)));
@@ -829,7 +823,7 @@ cudaError_t launch(const MultiArgs& a, cudaStream_t stream) {
   constexpr int NB = TokenBlocks<TP, G64>::value;
   const int ngroups = a.K / 128;
   const int nchunks = (ngroups + kChunkGroups - 1) / kChunkGroups;
-  const size_t smem = 64 + (size_t)kRows * (G64 ? 2 * ngroups : ngroups) * 3 + (size_t)kWarps * NB * 128 * 4 + (size_t)kRows * TP * 4 +
+  const size_t smem = 64 + (size_t)kRows * (G64 ? 2 * ngroups : ngroups) * 4 + (size_t)kWarps * NB * 128 * 4 + (size_t)kRows * TP * 4 +
                       (NBUF == 0 ? (size_t)nchunks * a.M * kRowPitch : (size_t)kWarps * NBUF * a.M * kTilePitch) * 16;
   if (smem > 48 * 1024) {
     cudaError_t e = cudaFuncSetAttribute(decode_kernel<BITS, TP, BF16, NBUF, G64>,
@@ -853,7 +847,7 @@ cudaError_t launch(const MultiArgs& a, cudaStream_t stream) {
 template <int TP, bool G64>
 size_t ring_smem(int K, int M, int bufs) {
   constexpr int NB = TokenBlocks<TP, G64>::value;
-  return 64 + (size_t)kRows * (K / (G64 ? 64 : 128)) * 3 + (size_t)kWarps * NB * 128 * 4 + (size_t)kRows * TP * 4 +
+  return 64 + (size_t)kRows * (K / (G64 ? 64 : 128)) * 4 + (size_t)kWarps * NB * 128 * 4 + (size_t)kRows * TP * 4 +
          (size_t)kWarps * bufs * M * kTilePitch * 16;
 }
 constexpr size_t kSmemPerCta = 227 * 1024;
@@ -907,7 +901,7 @@ gwq_status gwq_launch_decode_multi(const gwq_packed* const* P, int count, const 
   if (g64 && (M > kMaxTokens64 || P[0]->K % 128 != 0)) return GWQ_ERR_UNSUPPORTED;   // a warp step is 128 columns
   for (int i = 0; i < count; ++i) {
     const gwq_priv* pvi = static_cast<const gwq_priv*>(P[i]->priv);
-    if ((P[i]->group != 128 && P[i]->group != 64) || P[i]->group != P[0]->group || !pvi->cv || P[i]->K != P[0]->K || P[i]->bits != P[0]->bits) return GWQ_ERR_UNSUPPORTED;
+    if ((P[i]->group != 128 && P[i]->group != 64) || P[i]->group != P[0]->group || !pvi->cv || !pvi->sz_t || P[i]->K != P[0]->K || P[i]->bits != P[0]->bits) return GWQ_ERR_UNSUPPORTED;
   }
   gwq_priv* pv = static_cast<gwq_priv*>(P[0]->priv);
   MultiArgs a;
@@ -933,7 +927,7 @@ gwq_status gwq_launch_decode_multi(const gwq_packed* const* P, int count, const 
   int blocks = 0;
   for (int i = 0; i < kMaxLayers; ++i) {
     const gwq_packed* Pi = P[i < count ? i : 0];
-    a.layer[i].codes = Pi->codes; a.layer[i].scales = Pi->scales; a.layer[i].zeros = Pi->zeros;
+    a.layer[i].codes = Pi->codes; a.layer[i].szt = static_cast<const gwq_priv*>(Pi->priv)->sz_t;
     a.layer[i].row_ptr = Pi->S->row_ptr; a.layer[i].cv = static_cast<const gwq_priv*>(Pi->priv)->cv;
     a.layer[i].y = y[i < count ? i : 0]; a.layer[i].N = Pi->N;
     a.first_block[i] = blocks;
