@@ -316,8 +316,9 @@ __device__ __forceinline__ int tile_piece(int pc, int m) { return m * kTilePitch
 // the token side: a token block holds 4 tokens, output column n < 4 is token n with the activations of the second
 // group replaced by zeros (lanes t >= 2 read the zero page), column n >= 4 is token n - 4 with those of the first
 // group replaced by zeros.  Accumulator columns 2t, 2t+1 of lane t then belong to the lane's own group (t >> 1), whose
-// scale and zero-point it applies; the two halves of a token meet in the final sum.  Sums of x always come from the
-// all-ones MMA here.  TP <= 8.
+// scale and zero-point it applies; the two halves of a token meet in the final sum.  With more than one token the sums
+// of x come from the all-ones MMA (which sees the same zeros); a single token's are reduced over half a warp each.
+// TP <= 8.
 template <int TP, bool G64>
 struct TokenBlocks { static constexpr int value = G64 ? (TP <= 4 ? 1 : TP / 4) : (TP <= 8 ? 1 : TP / 8); };
 template <int BITS, int TP, bool BF16, int NBUF, bool G64>
@@ -345,7 +346,7 @@ decode_kernel(const MultiArgs ma) {
   constexpr int WPR = BITS;                   // words per run of 32 columns
   // raw path: sum_k x_k of a group from shared memory (one token), from the table that comes with the
   // token-major copy (ring mode), else from a second MMA with an all-ones A operand
-  constexpr bool ONES = !BF16 && (G64 || (TP != 1 && NBUF == 0));
+  constexpr bool ONES = !BF16 && TP != 1 && (G64 || NBUF == 0);
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int ngroups = p.K >> 7;               // warp steps of 128 columns in a row
   const int ntab = G64 ? 2 * ngroups : ngroups;   // scale / zero-point entries in a row
@@ -625,7 +626,8 @@ decode_kernel(const MultiArgs ma) {
         const float2 f1 = __half22float2(*reinterpret_cast<const __half2*>(&h4.y));
         xsum1 = (f0.x + f0.y) + (f1.x + f1.y);
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) xsum1 += __shfl_xor_sync(0xFFFFFFFFu, xsum1, o);
+        for (int o = G64 ? 8 : 16; o > 0; o >>= 1) xsum1 += __shfl_xor_sync(0xFFFFFFFFu, xsum1, o);
+        if (G64) xsum1 = __shfl_sync(0xFFFFFFFFu, xsum1, (t >> 1) << 4);   // lanes 0-15 summed the first group, 16-31 the second
       }
       typename StepAcc<BITS, NB, BF16>::type acc = {};
       unsigned qa[BITS], qb[BITS];
@@ -660,13 +662,13 @@ decode_kernel(const MultiArgs ma) {
             AccRaw4<NB>& a4 = reinterpret_cast<AccRaw4<NB>&>(acc);
             const float code_sum = fmaf(a4.c4[nb][i], 0.0625f, a4.c0[nb][i]);  // units of 2^-24
             const float xsum = ONES ? a4.xs[nb][i & 1]
-                                    : (TP == 1 ? ((i & 1) == 0 && t == 0 ? xsum1 : 0.f) : ((i & 1) ? xg2[nb].y : xg2[nb].x));
+                                    : (TP == 1 ? ((i & 1) == 0 && (G64 ? (t & 1) == 0 : t == 0) ? xsum1 : 0.f) : ((i & 1) ? xg2[nb].y : xg2[nb].x));
             yacc[nb][i] = fmaf(tt.x, code_sum, fmaf(-tt.y, xsum, yacc[nb][i]));
           } else {
             AccRaw3<NB>& a3 = reinterpret_cast<AccRaw3<NB>&>(acc);
             const float code_sum = fmaf(a3.c6[nb][i], 0.015625f, fmaf(a3.c3[nb][i], 0.125f, a3.c0[nb][i]));
             const float xsum = ONES ? a3.xs[nb][i & 1]
-                                    : (TP == 1 ? ((i & 1) == 0 && t == 0 ? xsum1 : 0.f) : ((i & 1) ? xg2[nb].y : xg2[nb].x));
+                                    : (TP == 1 ? ((i & 1) == 0 && (G64 ? (t & 1) == 0 : t == 0) ? xsum1 : 0.f) : ((i & 1) ? xg2[nb].y : xg2[nb].x));
             yacc[nb][i] = fmaf(tt.x, code_sum, fmaf(-tt.y, xsum, yacc[nb][i]));
           }
         }
@@ -692,9 +694,13 @@ decode_kernel(const MultiArgs ma) {
         }
         if (NBUF == 0) {
 #pragma unroll
-          for (int o = 16; o > 0; o >>= 1)
+          for (int o = G64 ? 8 : 16; o > 0; o >>= 1)
 #pragma unroll
             for (int d = 0; d < kDepth; ++d) xs4[d] += __shfl_xor_sync(0xFFFFFFFFu, xs4[d], o);
+          if (G64) {
+#pragma unroll
+            for (int d = 0; d < kDepth; ++d) xs4[d] = __shfl_sync(0xFFFFFFFFu, xs4[d], (t >> 1) << 4);
+          }
         }
       }
       if (NBUF == 0) {

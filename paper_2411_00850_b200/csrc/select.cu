@@ -177,58 +177,71 @@ __global__ void __launch_bounds__(1024) sel_rowscan_kernel(int N, const SelState
   if (threadIdx.x == 0) row_ptr[N] = (int32_t)total;
 }
 
-// Emits one CSR row in column order: every entry above the threshold, and the first
-// take[row] entries equal to it.
-__global__ void __launch_bounds__(kThreads) sel_emit_kernel(const unsigned int* __restrict__ G,
-                                                            const uint16_t* __restrict__ W, int K,
+// Emits the CSR rows in column order, one warp per row: every entry above the threshold, and the first
+// take[row] entries equal to it.  A lane reads four consecutive columns (one 16-byte load, four loads in flight);
+// a 128-column slice without a candidate costs one ballot, the others a warp scan of the per-lane counts.
+constexpr int kEmitUnroll = 4;
+__global__ void __launch_bounds__(kThreads) sel_emit_kernel(const uint4* __restrict__ G4,
+                                                            const uint16_t* __restrict__ W, int N, int K,
                                                             const SelState* __restrict__ st,
                                                             const unsigned int* __restrict__ take,
                                                             const int32_t* __restrict__ row_ptr,
                                                             int32_t* __restrict__ col_idx,
                                                             uint16_t* __restrict__ val) {
-  __shared__ unsigned int sh_gt[kThreads / 32], sh_tie[kThreads / 32];
-  const int row = blockIdx.x;
+  const int lane = threadIdx.x & 31;
+  const int row = blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5);
+  if (row >= N) return;
   const int begin = row_ptr[row];
-  if (row_ptr[row + 1] == begin) return;
+  if (row_ptr[row + 1] == begin) return;   // the whole warp leaves
   const unsigned int thr = st->prefix;
   const unsigned int tk = take[row];
-  const unsigned int* g = G + (long long)row * K;
+  const int n4 = K >> 2;
+  const uint4* g = G4 + (long long)row * n4;
   const uint16_t* w = W + (long long)row * K;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const unsigned int lt = (1u << lane) - 1u;
   unsigned int run_gt = 0, run_tie = 0;
-  for (int c0 = 0; c0 < K; c0 += kThreads) {
-    const int col = c0 + threadIdx.x;
-    const bool valid = col < K;
-    const unsigned int key = valid ? abs_key(__ldg(g + col)) : 0u;
-    const bool is_gt = valid && key > thr;
-    const bool is_tie = valid && key == thr;
-    const unsigned int b_gt = __ballot_sync(0xFFFFFFFFu, is_gt);
-    const unsigned int b_tie = __ballot_sync(0xFFFFFFFFu, is_tie);
-    if (lane == 0) {
-      sh_gt[warp] = __popc(b_gt);
-      sh_tie[warp] = __popc(b_tie);
+  for (int c0 = 0; c0 < n4; c0 += 32 * kEmitUnroll) {
+    uint4 v[kEmitUnroll];
+#pragma unroll
+    for (int u = 0; u < kEmitUnroll; ++u) {
+      const int idx = c0 + u * 32 + lane;
+      v[u] = idx < n4 ? __ldg(g + idx) : make_uint4(0u, 0u, 0u, 0u);
     }
-    __syncthreads();
-    unsigned int gt_before = run_gt + __popc(b_gt & lt), tie_before = run_tie + __popc(b_tie & lt);
-    unsigned int tot_gt = 0, tot_tie = 0;
-    for (int i = 0; i < kThreads / 32; ++i) {
-      const unsigned int a = sh_gt[i], b = sh_tie[i];
-      if (i < warp) {
-        gt_before += a;
-        tie_before += b;
+#pragma unroll
+    for (int u = 0; u < kEmitUnroll; ++u) {
+      const int idx = c0 + u * 32 + lane;
+      const bool valid = idx < n4;
+      const unsigned int k4[4] = {abs_key(v[u].x), abs_key(v[u].y), abs_key(v[u].z), abs_key(v[u].w)};
+      unsigned int mg = 0, mt = 0;   // this lane's four columns: above / equal to the threshold
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        mg |= (valid && k4[e] > thr) ? (1u << e) : 0u;
+        mt |= (valid && k4[e] == thr) ? (1u << e) : 0u;
       }
-      tot_gt += a;
-      tot_tie += b;
+      if (__ballot_sync(0xFFFFFFFFu, (mg | mt) != 0u) == 0u) continue;
+      const unsigned int mine = (unsigned int)__popc(mg) | ((unsigned int)__popc(mt) << 16);
+      unsigned int scan = mine;   // inclusive scan over the lanes of both counts (at most 128 each)
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const unsigned int up = __shfl_up_sync(0xFFFFFFFFu, scan, o);
+        if (lane >= o) scan += up;
+      }
+      const unsigned int total = __shfl_sync(0xFFFFFFFFu, scan, 31);
+      unsigned int gt_before = run_gt + ((scan - mine) & 0xFFFFu), tie_before = run_tie + ((scan - mine) >> 16);
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const bool is_gt = (mg >> e) & 1u, is_tie = (mt >> e) & 1u;
+        if (is_gt || (is_tie && tie_before < tk)) {
+          const unsigned int pos = gt_before + min(tie_before, tk);
+          const int col = idx * 4 + e;
+          col_idx[begin + pos] = col;
+          val[begin + pos] = w[col];
+        }
+        gt_before += is_gt ? 1u : 0u;
+        tie_before += is_tie ? 1u : 0u;
+      }
+      run_gt += total & 0xFFFFu;
+      run_tie += total >> 16;
     }
-    __syncthreads();
-    if (is_gt || (is_tie && tie_before < tk)) {
-      const unsigned int pos = gt_before + min(tie_before, tk);
-      col_idx[begin + pos] = col;
-      val[begin + pos] = w[col];
-    }
-    run_gt += tot_gt;
-    run_tie += tot_tie;
   }
 }
 
@@ -263,8 +276,8 @@ cudaError_t gwq_select_run(const uint16_t* W, const float* G, int N, int K, unsi
   }
   sel_rowcount_kernel<<<N, kThreads, 0, stream>>>(reinterpret_cast<const uint4*>(G), K / 4, st, n_gt, n_tie);
   sel_rowscan_kernel<<<1, 1024, 0, stream>>>(N, st, n_gt, n_tie, take, row_ptr);
-  sel_emit_kernel<<<N, kThreads, 0, stream>>>(reinterpret_cast<const unsigned int*>(G), W, K, st, take,
-                                              row_ptr, col_idx, val);
+  sel_emit_kernel<<<(N + kThreads / 32 - 1) / (kThreads / 32), kThreads, 0, stream>>>(
+      reinterpret_cast<const uint4*>(G), W, N, K, st, take, row_ptr, col_idx, val);
   return cudaGetLastError();
 }
 
