@@ -121,7 +121,7 @@ gwq_status gwq_select_outliers_static(const uint16_t* W_f16, const float* G_f32,
  * round-half-to-even; outliers get q = z.  A group with hi == lo gets s = 1, z = 0.
  *   bits: 3 or 4.  group: 16 (the value Section 3.2 names), 32, 64 or 128; K a multiple of 32 and of
  *      group.  The streaming path of gwq_linear takes group 128 (up to 32 tokens) and group 64 (up to
- *      8 tokens, K a multiple of 128), the tensor-core path 64 and 128; the other groups are served by
+ *      16 tokens, K a multiple of 128), the tensor-core path 64 and 128; the other groups are served by
  *      the general kernel.
  *   W_f16: device, caller-owned, read only.
  *   S: from gwq_select_outliers with the same N, K; on success its ownership moves into

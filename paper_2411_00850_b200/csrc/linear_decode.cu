@@ -30,7 +30,11 @@ constexpr int kWarps = 8;
 constexpr int kThreads = kWarps * 32;
 constexpr int kRows = 16;   // rows per CTA (one m16 tile)
 constexpr int kDepth = 4;   // groups of codes in flight per warp
-constexpr int kMaxTokens64 = 8;   // groups of 64: tokens one launch takes
+constexpr int kMaxTokens64 = 16;  // groups of 64: tokens one launch takes
+// Groups of 64 with 9 to 16 tokens need four token blocks (184 to 229 registers, one CTA per SM): faster than the
+// tensor-core kernel's 32-token tile up to about this many weights (measured: 59.8 against 84.8 us on 8192 x 8192,
+// 184.5 against 163.1 us on 28672 x 8192), slower beyond.
+constexpr long long kMaxWeights64Wide = 160LL * 1000 * 1000;
 
 template <bool BF16>
 __device__ __forceinline__ void mma16816(float (&d)[4], unsigned a0, unsigned a1, unsigned a2, unsigned a3,
@@ -318,7 +322,7 @@ __device__ __forceinline__ int tile_piece(int pc, int m) { return m * kTilePitch
 // group replaced by zeros.  Accumulator columns 2t, 2t+1 of lane t then belong to the lane's own group (t >> 1), whose
 // scale and zero-point it applies; the two halves of a token meet in the final sum.  With more than one token the sums
 // of x come from the all-ones MMA (which sees the same zeros); a single token's are reduced over half a warp each.
-// TP <= 8.
+// TP <= 16.
 template <int TP, bool G64>
 struct TokenBlocks { static constexpr int value = G64 ? (TP <= 4 ? 1 : TP / 4) : (TP <= 8 ? 1 : TP / 8); };
 template <int BITS, int TP, bool BF16, int NBUF, bool G64>
@@ -887,17 +891,19 @@ cudaError_t launch_tp(const MultiArgs& a, cudaStream_t stream) {
   return launch_buf<BITS, 32, BF16, 3, false>(a, stream);
 }
 
-// groups of 64: up to 8 tokens (two blocks of 4)
+// groups of 64: up to 16 tokens (blocks of 4)
 template <int BITS, bool BF16>
 cudaError_t launch_tp64(const MultiArgs& a, cudaStream_t stream) {
   if (a.M == 1) return launch_buf<BITS, 1, BF16, 2, true>(a, stream);
   if (a.M <= 4) return launch_buf<BITS, 4, BF16, 2, true>(a, stream);
-  return launch_buf<BITS, 8, BF16, 2, true>(a, stream);
+  if (a.M <= 8) return launch_buf<BITS, 8, BF16, 2, true>(a, stream);
+  return launch_buf<BITS, 16, BF16, 3, true>(a, stream);
 }
 
 }  // namespace
 
-// Decode launcher for `count` layers that read the same x: group size 128 (M <= 32) or 64 (M <= 8), K <= 65536, same K and bit
+// Decode launcher for `count` layers that read the same x: group size 128 (M <= 32) or 64 (M <= 8; M <= 16 for
+// layers up to kMaxWeights64Wide weights), K <= 65536, same K and bit
 // width in every layer.  Returns GWQ_ERR_UNSUPPORTED for anything else (nothing has been launched then).
 // The scratch for the token-major copy of x is the first layer's.
 gwq_status gwq_launch_decode_multi(const gwq_packed* const* P, int count, const void* x, gwq_dtype xd, int M,
@@ -909,6 +915,9 @@ gwq_status gwq_launch_decode_multi(const gwq_packed* const* P, int count, const 
     const gwq_priv* pvi = static_cast<const gwq_priv*>(P[i]->priv);
     if ((P[i]->group != 128 && P[i]->group != 64) || P[i]->group != P[0]->group || !pvi->cv || !pvi->sz_t || P[i]->K != P[0]->K || P[i]->bits != P[0]->bits) return GWQ_ERR_UNSUPPORTED;
   }
+  if (g64 && M > 8)
+    for (int i = 0; i < count; ++i)
+      if ((long long)P[i]->N * P[i]->K > kMaxWeights64Wide) return GWQ_ERR_UNSUPPORTED;
   gwq_priv* pv = static_cast<gwq_priv*>(P[0]->priv);
   MultiArgs a;
   a.xt = nullptr;
@@ -957,13 +966,13 @@ gwq_status gwq_launch_decode_multi(const gwq_packed* const* P, int count, const 
   return GWQ_OK;
 }
 
-// Decode launcher: group size 128 with M <= 32 or 64 with M <= 8, K <= 65536.  Groups of 64 with more tokens go to
-// the tensor-core kernel, other shapes to the general kernel.
+// Decode launcher: group size 128 with M <= 32 or 64 with M <= 8 (16 for layers of moderate size), K <= 65536.
+// Groups of 64 with more tokens go to the tensor-core kernel, other shapes to the general kernel.
 gwq_status gwq_launch_decode(const gwq_packed* P, const void* x, gwq_dtype xd, int M, void* y, gwq_dtype yd,
                              cudaStream_t stream) {
   const gwq_status st = gwq_launch_decode_multi(&P, 1, x, xd, M, &y, yd, stream);
   if (st != GWQ_ERR_UNSUPPORTED) return st;
   // groups of 64 beyond the tokens the streaming kernel takes: the tensor-core kernel with its smallest token tile
-  if (P->group == 64 && M > kMaxTokens64) return gwq_launch_prefill(P, x, xd, M, y, yd, stream);
+  if (P->group == 64 && M > 8) return gwq_launch_prefill(P, x, xd, M, y, yd, stream);
   return gwq_launch_simt(P, x, xd, M, y, yd, stream);
 }
