@@ -82,9 +82,10 @@ def test_full_size_layer(N, K, bits, layer_index):
         assert gwq.gwq_device_status(P) == 0
 
     # tensor-core path: bf16 activations with 8 heavy channels, as in the prefill cases
-    for M in (512, 2048):
+    for M in (512, 2048, 8192):
         bits16, xv = synth.make_activations(M, K, seed=900 + M, dtype="bf16", heavy_channels=8)
         y = gwq.gwq_linear(P, x_tensor(bits16, "bf16"), out_dtype=torch.float32)
         y_ref, bound = orc.linear(xv, w_hat)
         assert_linear_close(y[:, rows], y_ref, bound)
+        del y
     assert gwq.gwq_device_status(P) == 0

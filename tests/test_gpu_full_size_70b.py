@@ -1,7 +1,7 @@
 """Parity on Llama-70B-shaped layers (8192 x 8192, 28672 x 8192, 8192 x 28672): both bit widths,
 groups of 64 and 128, outlier fractions 0.5 / 1 / 2 %, M in {1, 8, 32, 2048}.  As at the other full
 sizes the CPU checker selects the outliers of the whole matrix (compared in full, bit for bit) and
-encodes, reconstructs and multiplies sampled rows one by one."""
+encodes, reconstructs and multiplies ~250 sampled output rows one by one, for every token row."""
 import numpy as np
 import pytest
 import torch
@@ -14,10 +14,10 @@ from tests.gpu_util import assert_linear_close, to_dev, x_tensor
 pytestmark = pytest.mark.gpu
 
 
-def _sample_rows(N, seed):
+def _sample_rows(N, seed, extra=246):
     rng = np.random.default_rng(seed)
     rows = {0, 1, 7, 8, 15, 16, N - 17, N - 16, N - 2, N - 1}
-    rows.update(int(r) for r in rng.integers(0, N, size=10))
+    rows.update(int(r) for r in rng.integers(0, N, size=extra))
     return sorted(rows)
 
 
@@ -70,13 +70,8 @@ def test_llama70b_shaped_layer(shape_index, encodings, frac):
                                                 heavy_channels=8 if M == 2048 else 0)
             y = gwq.gwq_linear(P, x_tensor(bits16, dtype), out_dtype=torch.float32)
             torch.cuda.synchronize()
-            if M == 2048:   # checker on 64 seeded token rows (all sampled output rows)
-                tok = np.sort(np.random.default_rng(M + shape_index).choice(M, size=64, replace=False))
-                y_ref, bound = orc.linear(xv[tok], w_hat)
-                assert_linear_close(y[torch.from_numpy(tok).to(y.device)][:, rows], y_ref, bound)
-            else:
-                y_ref, bound = orc.linear(xv, w_hat)
-                assert_linear_close(y[:, rows], y_ref, bound)
+            y_ref, bound = orc.linear(xv, w_hat)       # every token row on ~250 sampled output rows
+            assert_linear_close(y[:, rows], y_ref, bound)
             del y
         assert gwq.gwq_device_status(P) == 0
         del P, S

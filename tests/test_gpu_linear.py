@@ -113,6 +113,18 @@ def test_small_groups(layer, M, dtype):
     assert_linear_close(y, y_ref, bound)
 
 
+@pytest.mark.parametrize("layer", [DECODE_LAYERS[0], DECODE_LAYERS[3]])
+@pytest.mark.parametrize("M", [1, 8, 16, 32, 200])
+def test_repeated_calls_give_the_same_bits(layer, M):
+    # fixed summation order everywhere (no floating-point atomics): the same call twice is bit-identical
+    P, L, w_hat = _layer(*layer)
+    bits16, _ = synth.make_activations(M, P.K, seed=300 + M, dtype="f16", heavy_channels=8 if M > 32 else 0)
+    x = x_tensor(bits16, "f16")
+    y1 = gwq.gwq_linear(P, x, out_dtype=torch.float32).clone()
+    y2 = gwq.gwq_linear(P, x, out_dtype=torch.float32)
+    assert torch.equal(y1, y2)
+
+
 def test_all_outliers_is_the_dense_product():
     N, K = 128, 512
     W, G = synth.make_weight_and_grad(N, K, 30)
