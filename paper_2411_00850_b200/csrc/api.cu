@@ -8,6 +8,15 @@
 
 static size_t dtype_bytes(gwq_dtype d) { return d == GWQ_F32 ? 4 : 2; }
 
+// With 17 to 32 tokens the streaming kernel needs four token blocks (one CTA of 8 warps per SM) and copies 8 KB of
+// activations per KB of codes; on tall layers the tensor-core kernel's 32-token tile is faster (measured, 4 bit,
+// M = 32: 44 against 52 us on 11008 x 4096, 161 against 215 us on 28672 x 8192), on layers with few 128-row tiles it
+// is not (84 against 70 us on 8192 x 8192, 287 against 213 us on 8192 x 28672).
+static bool prefers_tensor_core(const gwq_packed* P, int M) {
+  const gwq_priv* pv = static_cast<const gwq_priv*>(P->priv);
+  return M > 16 && M <= GWQ_DECODE_MAX_M && P->group == 128 && P->N >= 10240 && P->K % 64 == 0 && pv->cv && pv->sz_t;
+}
+
 extern "C" gwq_status gwq_linear(const gwq_packed* P, const void* x, gwq_dtype xd, int32_t M, void* y,
                                  gwq_dtype yd, void* stream_) {
   if (!P || P->tag != GWQ_TAG_PACKED || !P->S || !P->priv || !x || !y || M <= 0) return GWQ_ERR_INVALID_ARG;
@@ -15,7 +24,7 @@ extern "C" gwq_status gwq_linear(const gwq_packed* P, const void* x, gwq_dtype x
   if (yd != GWQ_F16 && yd != GWQ_BF16 && yd != GWQ_F32) return GWQ_ERR_INVALID_ARG;
   if (!gwq_aligned16(x) || !gwq_aligned16(y)) return GWQ_ERR_INVALID_ARG;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-  if (M <= GWQ_DECODE_MAX_M) return gwq_launch_decode(P, x, xd, M, y, yd, stream);
+  if (M <= GWQ_DECODE_MAX_M && !prefers_tensor_core(P, M)) return gwq_launch_decode(P, x, xd, M, y, yd, stream);
   return gwq_launch_prefill(P, x, xd, M, y, yd, stream);
 }
 
@@ -31,7 +40,9 @@ extern "C" gwq_status gwq_linear_multi(const gwq_packed* const* P, int32_t count
     if (P[i]->K != P[0]->K) return GWQ_ERR_INVALID_ARG;
   }
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-  if (M <= GWQ_DECODE_MAX_M) {
+  bool fused = M <= GWQ_DECODE_MAX_M;
+  for (int i = 0; i < count; ++i) fused = fused && !prefers_tensor_core(P[i], M);   // same kernels as gwq_linear
+  if (fused) {
     const gwq_status st = gwq_launch_decode_multi(P, count, x, xd, M, y, yd, stream);
     if (st != GWQ_ERR_UNSUPPORTED) return st;
   }

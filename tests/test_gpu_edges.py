@@ -77,3 +77,10 @@ def test_groups_of_64_on_the_streaming_path(bits):
 def test_groups_of_64_with_an_odd_number_of_groups():
     # K = 192 is not a whole number of 128-column steps: the general kernel
     _check(48, 192, 0.02, 4, 64, 88, [(1, "f16"), (3, "bf16"), (20, "f16")])
+
+
+def test_tall_layers_take_the_tensor_core_kernel_from_17_tokens():
+    # N >= 10240 with groups of 128: 17 to 32 tokens go to the tensor-core kernel's 32-token tile, fewer tokens
+    # and shorter layers stay on the streaming kernel; fused siblings follow the same rule
+    _check(10368, 512, 0.01, 4, 128, 90, [(16, "f16"), (17, "f16"), (24, "bf16"), (32, "f16"), (32, "bf16")])
+    _check(10240, 256, 0.01, 3, 128, 91, [(17, "bf16"), (32, "f16")])

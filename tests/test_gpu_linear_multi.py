@@ -67,6 +67,20 @@ def test_fused_siblings_with_groups_of_64(bits, M, dtype):
         assert torch.equal(y, gwq.gwq_linear(P, x, out_dtype=torch.float32))
 
 
+def test_tall_siblings_beyond_16_tokens_follow_the_single_call():
+    # layers of 10240 rows or more go to the tensor-core kernel from 17 tokens on, in the fused call too
+    sib = [_layer(10240, 256, 0.01, 4, 128, 52), _layer(10368, 256, 0.01, 4, 128, 53)]
+    for M in (16, 20):
+        bits16, xv = synth.make_activations(M, 256, seed=210 + M, dtype="f16")
+        x = x_tensor(bits16, "f16")
+        ys = gwq.gwq_linear_multi([s[0] for s in sib], x, out_dtype=torch.float32)
+        for (P, L, w_hat), y in zip(sib, ys):
+            y_ref, bound = orc.linear(xv, w_hat)
+            assert_linear_close(y, y_ref, bound)
+            assert torch.equal(y, gwq.gwq_linear(P, x, out_dtype=torch.float32))
+            assert gwq.gwq_device_status(P) == 0
+
+
 def test_two_and_four_layers_and_16_bit_outputs():
     sib = _siblings(4) + [_layer(48, 1024, 0.02, 4, 128, 47)]
     bits16, xv = synth.make_activations(4, 1024, seed=7, dtype="f16")
