@@ -135,7 +135,8 @@ gwq_status gwq_pack(const uint16_t* W_f16, gwq_outliers* S, int32_t N, int32_t K
 /* Forward product y = x (s (q - z) + S)^T (Section 3.2, Eq. "w", outliers in FP16).
  *   x: device [M, K], fp16 or bf16 (x_dtype).  y: device [M, N], y_dtype one of
  *   F16 / BF16 / F32.  Accumulation is FP32.  M >= 1; M <= 32 takes the bandwidth-bound
- *   streaming path, larger M the tensor-core path.
+ *   streaming path, larger M the tensor-core path (which also serves 17 to 32 tokens on
+ *   layers of 10240 rows or more, and groups of 64 beyond 16 tokens, where it is faster).
  *   Asynchronous on `stream`; argument errors are returned immediately.
  * Errors: INVALID_ARG, UNSUPPORTED (x_dtype F32), CUDA (launch failure).               */
 gwq_status gwq_linear(const gwq_packed* P, const void* x, gwq_dtype x_dtype, int32_t M, void* y,
