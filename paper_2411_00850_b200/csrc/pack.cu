@@ -1,7 +1,8 @@
 // Group-wise asymmetric quantization of the non-outliers and bit-packing
 // (Section 3.2, Eqs. "s", "z", "q"; outliers excluded from the group range).
 //
-// One CTA per output row.  The row's outlier columns are expanded into a bitmask in
+// One CTA per output row (the weights of a warp's first four passes are requested before
+// anything else).  The row's outlier columns are expanded into a bitmask in
 // shared memory, each warp then quantizes whole groups (min / max by shuffles, the
 // scale and zero-point in FP64 so that every rounding is fixed bit for bit), codes go
 // to shared memory as bytes and are finally packed into 32-bit words.
@@ -25,6 +26,31 @@ pack_row_kernel(const uint16_t* __restrict__ W, const int32_t* __restrict__ row_
   unsigned char* q8 = smem + (K / 32) * 4;                      // K bytes
   const int row = blockIdx.x;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  // A warp takes one group per pass (GROUP >= 32: GROUP / 32 consecutive elements per lane) or 32 / GROUP
+  // neighbouring groups per pass (GROUP = 16: one element per lane, 16 lanes per group).
+  constexpr int LPG = GROUP >= 32 ? 32 : GROUP;   // lanes per group
+  constexpr int EPL = GROUP / LPG;                // consecutive elements per lane
+  constexpr int GPP = 32 / LPG;                   // groups per warp and pass
+  constexpr int kAhead = 4;                       // passes whose weights are requested together
+  constexpr int kPassStride = (kThreads / 32) * GPP;
+  const int ngroups = K / GROUP;
+  const uint16_t* wrow = W + (long long)row * K;
+  auto load_raw = [&](int g0) {   // this lane's EPL weights of the pass that starts at group g0
+    const int g = min(g0 + lane / LPG, ngroups - 1);   // K is a multiple of 32, so every group of a pass exists
+    const int c0 = g * GROUP + (lane % LPG) * EPL;
+    uint2 v = make_uint2(0u, 0u);
+    if (EPL == 4) v = *reinterpret_cast<const uint2*>(wrow + c0);
+    else if (EPL == 2) v.x = *reinterpret_cast<const unsigned int*>(wrow + c0);
+    else v.x = wrow[c0];
+    return v;
+  };
+  // the first passes' weights are on their way while the mask is built
+  uint2 raw[kAhead];
+#pragma unroll
+  for (int u = 0; u < kAhead; ++u) {
+    const int g0 = warp * GPP + u * kPassStride;
+    raw[u] = g0 < ngroups ? load_raw(g0) : make_uint2(0u, 0u);
+  }
   for (int i = threadIdx.x; i < K / 32; i += kThreads) mask[i] = 0;
   __syncthreads();
   const int jb = row_ptr[row], je = row_ptr[row + 1];
@@ -34,27 +60,18 @@ pack_row_kernel(const uint16_t* __restrict__ W, const int32_t* __restrict__ row_
   }
   __syncthreads();
 
-  // A warp takes one group per pass (GROUP >= 32: GROUP / 32 consecutive elements per lane) or 32 / GROUP
-  // neighbouring groups per pass (GROUP = 16: one element per lane, 16 lanes per group).
-  constexpr int LPG = GROUP >= 32 ? 32 : GROUP;   // lanes per group
-  constexpr int EPL = GROUP / LPG;                // consecutive elements per lane
-  constexpr int GPP = 32 / LPG;                   // groups per warp and pass
-  const int ngroups = K / GROUP;
   const double qmax = (double)((1 << bits) - 1);
-  const uint16_t* wrow = W + (long long)row * K;
   bool bad = false;
-  for (int g0 = warp * GPP; g0 < ngroups; g0 += (kThreads / 32) * GPP) {
-    const int g = min(g0 + lane / LPG, ngroups - 1);   // K is a multiple of 32, so every group of a pass exists
+  auto quantize_pass = [&](const int g0, const uint2 v) {
+    const int g = min(g0 + lane / LPG, ngroups - 1);
     const int c0 = g * GROUP + (lane % LPG) * EPL;
     unsigned int hb[EPL];
     if (EPL == 4) {
-      const uint2 v = *reinterpret_cast<const uint2*>(wrow + c0);
       hb[0] = v.x & 0xFFFFu; hb[1 % EPL] = v.x >> 16; hb[(EPL - 2 + EPL) % EPL] = v.y & 0xFFFFu; hb[EPL - 1] = v.y >> 16;
     } else if (EPL == 2) {
-      const unsigned int v = *reinterpret_cast<const unsigned int*>(wrow + c0);
-      hb[0] = v & 0xFFFFu; hb[EPL - 1] = v >> 16;
+      hb[0] = v.x & 0xFFFFu; hb[EPL - 1] = v.x >> 16;
     } else {
-      hb[0] = wrow[c0];
+      hb[0] = v.x & 0xFFFFu;
     }
     // this lane's EPL mask bits: c0 is a multiple of EPL, so they sit in one mask word
     const unsigned int mbits = (mask[c0 >> 5] >> (c0 & 31)) & ((1u << EPL) - 1u);
@@ -98,6 +115,20 @@ pack_row_kernel(const uint16_t* __restrict__ W, const int32_t* __restrict__ row_
     if (lane % LPG == 0) {
       scales[(long long)row * ngroups + g] = __half_as_ushort(sh);
       zeros[(long long)row * ngroups + g] = (uint8_t)(int)z;
+    }
+  };
+  for (int gb = warp * GPP; gb < ngroups; gb += kAhead * kPassStride) {
+    if (gb != warp * GPP) {   // later batches (rows of more than kAhead passes per warp)
+#pragma unroll
+      for (int u = 0; u < kAhead; ++u) {
+        const int g0 = gb + u * kPassStride;
+        raw[u] = g0 < ngroups ? load_raw(g0) : make_uint2(0u, 0u);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < kAhead; ++u) {
+      const int g0 = gb + u * kPassStride;
+      if (g0 < ngroups) quantize_pass(g0, raw[u]);   // warp-uniform
     }
   }
   if (bad) atomicExch(status, (int32_t)GWQ_ERR_NONFINITE);
