@@ -303,16 +303,21 @@ def run_cuda_arm(args):
     if rank == 0:
         sampler.start()
         time.sleep(0.3)
-    ms_step = time_region(torch, lambda i: graphs[i % replicas](), args.steps)
+    # the timed block of exactly `steps` steps is repeated `repeats` times (each block bracketed by a synchronisation on
+    # both sides); the headline is the median block, the fastest one is reported beside it
+    blocks_ms = [time_region(torch, lambda i: graphs[i % replicas](), args.steps) for _ in range(max(1, args.repeats))]
+    ms_step, ms_step_min = float(np.median(blocks_ms)), float(min(blocks_ms))
     if world > 1:
         ms_step = max_over_ranks(ms_step, dev)
+        ms_step_min = max_over_ranks(ms_step_min, dev)
         dist.barrier()
     clocks = sampler.stop() if rank == 0 else {}
     value = whole_job_gbs(step_bytes, ms_step, world)
 
     out = {
         "metric": METRIC, "value": round(value, 1), "unit": "GB/s", "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": round(ms_step, 4), "higher_is_better": True, "scaling": "weak",
+        "warmup": args.warmup, "ms_per_step": round(ms_step, 4), "ms_per_step_min": round(ms_step_min, 4),
+        "timed_blocks": len(blocks_ms), "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f16 x int4/int3 -> f32 accumulate", "data": "synthetic",
         "config": {"workload": WORKLOAD, "layers": [f"{n}:{N}x{K}" for n, N, K in synth.LLAMA7B_LAYER_SET],
                    "bits": list(BIT_WIDTHS), "group": GROUP, "outlier_frac": FRAC, "M": list(DECODE_MS),
@@ -323,7 +328,7 @@ def run_cuda_arm(args):
                                    "per (M, bits): q|k|v concurrently, o, gate|up concurrently, down (decoder-block data flow)",
                    "l2": f"{replicas} rotating copies of the packed set ({replicas * step_bytes // 3 / 1e6:.0f} MB) "
                          "exceed the 126 MB L2 between reuses; one CUDA graph per copy"},
-        "gpu_launches": args.steps * launches_per_step,
+        "gpu_launches": args.steps * launches_per_step * len(blocks_ms),
         "clocks": clocks,
     }
     if rank != 0:
@@ -630,6 +635,73 @@ def bench_prefill(torch, gwq, dev, args, tf_burst, tf_sust):
     return rows
 
 
+# ----------------------------------------------------------------------------- single cases (profiling, sweeps)
+def run_cases(args):
+    """--case N,K,bits,group,M,dtype[,frac] (repeatable): one synthetic layer per case, `copies` packed copies
+    cycled through so that a launch does not find its weights in L2 (at least 256 MB between reuses unless
+    --case-copies says otherwise).  Per case: microseconds per gwq_linear call, cold L2, replayed from a CUDA
+    graph (min and median over --case-iters replays, a 256 MB read-only scrub before each), or in plain stream
+    order with --case-stream (the form the profiler captures are taken on: few launches, no graph)."""
+    import torch
+
+    from paper_2411_00850_b200 import binding as gwq
+    from paper_2411_00850_b200 import build as gbuild
+    gbuild.build()
+    gwq.load_library()
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    hbm_peak, tf_burst, _tf_sust, peak_src = measured_peaks()
+    scrub = torch.zeros(64 * 1024 * 1024, dtype=torch.int32, device=dev)
+    rows, cache = [], {}
+    for spec in args.case:
+        f = spec.split(",")
+        N, K, bits, group, M = (int(v) for v in f[:5])
+        dtype = f[5] if len(f) > 5 else "f16"
+        frac = float(f[6]) if len(f) > 6 else FRAC
+        key = (N, K, bits, group, frac)
+        if key not in cache:
+            cache.clear()
+            W, G = synth.make_weight_and_grad(N, K, 1)
+            Wd, Gd = torch.from_numpy(W).to(dev), torch.from_numpy(G).to(dev)
+            per_copy = N * K * bits // 8
+            copies = args.case_copies or max(2, min(32, -(-256 * 1024 * 1024 // per_copy)))
+            cache[key] = [gwq.gwq_pack(Wd, gwq.gwq_select_outliers(Wd, Gd, frac), bits, group) for _ in range(copies)]
+            del Wd, Gd
+        packed = cache[key]
+        bits16, _ = synth.make_activations(M, K, 1, dtype=dtype, heavy_channels=8 if M > 32 else 0)
+        x = torch.from_numpy(bits16.view(np.int16).copy()).to(dev).view(torch.float16 if dtype == "f16" else torch.bfloat16)
+        y = torch.empty((M, N), dtype=x.dtype, device=dev)
+        need = max(int(gwq.load_library().gwq_linear_workspace_bytes(P._h, gwq._dtype_code(x.dtype), M)) for P in packed)
+        ws = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
+
+        def run():
+            for P in packed:
+                gwq.gwq_linear(P, x, out=y, workspace=ws if need else None)
+        for _ in range(2):
+            run()
+        torch.cuda.synchronize()
+        times = []
+        if args.case_stream:
+            for _ in range(args.case_iters):
+                times.append(time_region(torch, lambda i: run(), 1))
+        else:
+            replay = capture(torch, run)
+            for _ in range(args.case_iters):
+                int(scrub.sum().item())
+                times.append(time_region(torch, lambda i: replay(), 1))
+        us_min, us_med = min(times) * 1e3 / len(packed), float(np.median(times)) * 1e3 / len(packed)
+        nnz = packed[0].nnz
+        b = algorithmic_bytes(N, K, bits, group, nnz, M)
+        fl = linear_flops(N, K, nnz, M)
+        rows.append({"N": N, "K": K, "bits": bits, "group": group, "M": M, "dtype": dtype, "frac": frac,
+                     "copies": len(packed), "us": round(us_min, 3), "us_median": round(us_med, 3), "bytes": b,
+                     "gbs": round(b / us_min / 1e3, 1), "frac_measured_peak": round(b / us_min / 1e3 / hbm_peak, 4),
+                     "tflops": round(fl / us_min / 1e6, 2), "status": gwq.gwq_device_status(packed[0])})
+        print(json.dumps(rows[-1]), file=sys.stderr, flush=True)
+    return {"mode": "cases", "order": "stream" if args.case_stream else "cuda graph, cold L2", "peak_source": peak_src,
+            "hbm_peak_gbs": hbm_peak, "cases": rows}
+
+
 # ----------------------------------------------------------------------------- the CPU checker, timed
 def cpu_baseline(sample_seconds: float = 20.0) -> dict:
     """Times the CPU checker's forward product (reconstruction + float64 product) as it stands, on a
@@ -696,14 +768,23 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=("ours", "reference"))
-    ap.add_argument("--prefill-iters", type=int, default=5)
+    ap.add_argument("--repeats", type=int, default=10, help="timed blocks of `steps` steps (median reported)")
+    ap.add_argument("--prefill-iters", type=int, default=20)
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--headline-only", action="store_true", help="skip the per-case detail sections")
     ap.add_argument("--skip-70b", action="store_true", help="skip the Llama-70B-shaped decode cases")
     ap.add_argument("--no-fuse", action="store_true",
                     help="launch sibling projections as separate concurrent calls instead of one gwq_linear_multi")
+    ap.add_argument("--case", action="append", default=[], metavar="N,K,bits,group,M,dtype[,frac]",
+                    help="time gwq_linear on one synthetic layer instead of the benchmark (repeatable)")
+    ap.add_argument("--case-copies", type=int, default=0, help="packed copies cycled through (default: 256 MB worth)")
+    ap.add_argument("--case-iters", type=int, default=10)
+    ap.add_argument("--case-stream", action="store_true", help="plain stream order instead of a CUDA graph, no L2 scrub")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.case:
+        print(json.dumps(run_cases(args), ensure_ascii=False))
+        return
     out = run_reference_arm(args) if args.impl == "reference" else run_cuda_arm(args)
     if out is not None:
         print(json.dumps(out, ensure_ascii=False))

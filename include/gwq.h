@@ -36,11 +36,12 @@ extern "C" {
 typedef enum {
   GWQ_OK = 0,
   GWQ_ERR_INVALID_ARG = 1, /* null or misaligned pointer, non-positive size, frac outside [0,1] */
-  GWQ_ERR_UNSUPPORTED = 2, /* bits not in {3,4}, group not in {64,128}, K % group != 0, ...    */
+  GWQ_ERR_UNSUPPORTED = 2, /* bits not in {3,4}, group not in {16,32,64,128}, K % group != 0 */
   GWQ_ERR_ALLOC = 3,       /* device or host allocation failed                                  */
   GWQ_ERR_NONFINITE = 4,   /* W holds an inf or NaN                                             */
   GWQ_ERR_TIMEOUT = 5,     /* a bounded device-side wait ran out (kernel returned early)        */
-  GWQ_ERR_CUDA = 6         /* a CUDA runtime call failed                                        */
+  GWQ_ERR_CUDA = 6,        /* a CUDA runtime call failed                                        */
+  GWQ_ERR_WORKSPACE = 7    /* the call needs scratch memory: see gwq_linear_ws                  */
 } gwq_status;
 
 typedef enum { GWQ_F16 = 0, GWQ_BF16 = 1, GWQ_F32 = 2 } gwq_dtype;
@@ -101,8 +102,9 @@ gwq_status gwq_select_outliers(const uint16_t* W_f16, const float* G_f32, int32_
  * This call performs no cudaMalloc / cudaFree and calls no allocating routine.
  *
  *   row_ptr [N+1], col_idx [capacity], val [capacity]: device buffers supplied by the
- *   caller; capacity must be >= ceil(frac * N*K), which is written to *nnz_host (host).
- *   The work area is a fixed ~386 KiB array inside the library image, present on every
+ *   caller; capacity must be >= ceil(frac * N*K), which is written to *nnz_host (host),
+ *   also when the call fails because capacity is too small (0 on every other failure).
+ *   The work area is a fixed 392 KiB array inside the library image, present on every
  *   GPU that loads the library; it bounds the row count: N <= 32768, otherwise
  *   GWQ_ERR_UNSUPPORTED.  All calls on one GPU share that array, so two calls that
  *   overlap on the GPU (different streams or threads) corrupt each other; serialise
@@ -135,28 +137,43 @@ gwq_status gwq_pack(const uint16_t* W_f16, gwq_outliers* S, int32_t N, int32_t K
 /* Forward product y = x (s (q - z) + S)^T (Section 3.2, Eq. "w", outliers in FP16).
  *   x: device [M, K], fp16 or bf16 (x_dtype).  y: device [M, N], y_dtype one of
  *   F16 / BF16 / F32.  Accumulation is FP32.  M >= 1; M <= 32 takes the bandwidth-bound
- *   streaming path, larger M the tensor-core path (which also serves 17 to 32 tokens on
- *   layers of 10240 rows or more, and groups of 64 beyond 16 tokens, where it is faster).
- *   Asynchronous on `stream`; argument errors are returned immediately.
- * Errors: INVALID_ARG, UNSUPPORTED (x_dtype F32), CUDA (launch failure).               */
+ *   streaming path, larger M the tensor-core path.
+ *   Asynchronous on `stream`: the call only enqueues kernels.  It never allocates and never
+ *   synchronises, so it may be captured into a CUDA graph from its first use.  Calls that share P
+ *   must be enqueued on one stream (or otherwise ordered): with 9 to 32 tokens they share a small
+ *   scratch buffer that gwq_pack created inside P.
+ *   A call that needs more scratch than P holds (bf16 activations on the tensor-core path: an fp16
+ *   copy of x) returns GWQ_ERR_WORKSPACE and does nothing: make it through gwq_linear_ws.
+ * Errors: INVALID_ARG, UNSUPPORTED (x_dtype F32), WORKSPACE, CUDA (launch failure).      */
 gwq_status gwq_linear(const gwq_packed* P, const void* x, gwq_dtype x_dtype, int32_t M, void* y,
                       gwq_dtype y_dtype, void* stream);
 
+/* gwq_linear with scratch memory supplied by the caller.  gwq_linear_workspace_bytes returns the bytes
+ * the product (P, x_dtype, M) needs (0 when it needs none); `workspace` must be a device buffer of at
+ * least that size, 256-byte aligned, and must not be used by anything else until the kernels enqueued by
+ * the call have finished (calls on one stream may share it).  Otherwise exactly gwq_linear.
+ * Errors: as gwq_linear; WORKSPACE when workspace_bytes is too small or the buffer is misaligned.  */
+size_t gwq_linear_workspace_bytes(const gwq_packed* P, gwq_dtype x_dtype, int32_t M);
+gwq_status gwq_linear_ws(const gwq_packed* P, const void* x, gwq_dtype x_dtype, int32_t M, void* y,
+                         gwq_dtype y_dtype, void* workspace, size_t workspace_bytes, void* stream);
+
 /* Several forward products that read the same activations, in one call: y[i] = x (deq(P[i]) + S_i)^T for
  * i < count.  This is launch-level fusion of sibling projections (q | k | v, or gate | up, of a decoder
- * block: Section 4.5 measures whole-model generation, where these run back to back); each product is
+ * block: Section 4.2, "Model Efficiency Comparison", times whole-model generation, where these run back to back); each product is
  * exactly the one gwq_linear computes, bit for bit.
  *   P: host array of `count` packed layers (1 <= count <= GWQ_MULTI_MAX) with the same K.
  *   x: device [M, K]; y: host array of `count` device pointers, y[i] is [M, P[i]->N], all of y_dtype.
- *   With M <= 32, group 128 and one bit width for all layers, the products run as ONE kernel launch
- *   (layer 0 lends its scratch: do not overlap with another call that uses P[0]); otherwise the call is
- *   the same as `count` calls of gwq_linear in order.  Asynchronous on `stream`.
+ *   With M <= 32, one group size (64 or 128) and one bit width for all layers, the products run as ONE kernel
+ *   launch wherever the streaming kernel takes that shape (layer 0 lends its scratch: do not overlap with
+ *   another call that uses P[0]); otherwise the call is the same as `count` calls of gwq_linear in order
+ *   (and like them returns GWQ_ERR_WORKSPACE where a product needs scratch: call gwq_linear_ws per layer
+ *   then).  Asynchronous on `stream`; never allocates, never synchronises.
  * Errors: INVALID_ARG (count, null entries, differing K, alignment), otherwise as gwq_linear.          */
 #define GWQ_MULTI_MAX 4
 gwq_status gwq_linear_multi(const gwq_packed* const* P, int32_t count, const void* x, gwq_dtype x_dtype,
                             int32_t M, void* const* y, gwq_dtype y_dtype, void* stream);
 
-/* Mean of the gradients of `count` calibration samples (Section 4.5, "Effect on Number of Calibration":
+/* Mean of the gradients of `count` calibration samples (Section 4.3, "Effect on Number of Calibration":
  * the outliers are located on the gradient mean); the result feeds gwq_select_outliers.
  * G_mean[i] = (((G_0[i] + G_1[i]) + G_2[i]) + ...) / count, FP32, additions in sample order, round to
  * nearest, one division: reproducible bit for bit.
@@ -185,8 +202,9 @@ gwq_status gwq_read_probe(const gwq_packed* P, int64_t* bytes_read, void* stream
 
 /* Same product with HOST buffers: copies x_host [M,K] to a staging buffer kept inside P,
  * runs gwq_linear, copies y back into y_host [M,N] and synchronises `stream`.
- * For best copy speed the host buffers should be page-locked.  The staging buffers grow
- * on demand (cudaMalloc) and are shared by all calls on P: not re-entrant per P.       */
+ * For best copy speed the host buffers should be page-locked.  The staging buffers (and the scratch
+ * of gwq_linear_ws, where needed) grow on demand (cudaMalloc) and are shared by all calls on P: not
+ * re-entrant per P.                                                                    */
 gwq_status gwq_linear_host(gwq_packed* P, const void* x_host, gwq_dtype x_dtype, int32_t M,
                            void* y_host, gwq_dtype y_dtype, void* stream);
 
@@ -204,6 +222,14 @@ gwq_status gwq_linear_host_async(gwq_packed* P, const void* x_host, gwq_dtype x_
  * tensor-core path ran out and the kernel returned early; y is then undefined, and later
  * tensor-core calls on P do no work until the status has been read) and clears it.            */
 gwq_status gwq_device_status(const gwq_packed* P, void* stream);
+
+/* Diagnostic, no counterpart in the paper: the number of SM clock cycles a bounded device-side wait of the
+ * tensor-core path may spin before the kernel gives up with GWQ_ERR_TIMEOUT (default: 10^9, about half a
+ * second).  cycles < 0 restores the default; 0 makes the first wait that is not satisfied at once give up,
+ * which lets a test walk the give-up path (the kernel drains what it has in flight, frees its tensor memory
+ * and returns) without any fault.  Takes effect for the calls on P made afterwards.
+ * Errors: INVALID_ARG.                                                                              */
+gwq_status gwq_set_wait_limit(gwq_packed* P, int64_t cycles);
 
 /* Releases a gwq_outliers* or a gwq_packed* (and everything it owns).  NULL is a no-op. */
 void gwq_free(void* obj);

@@ -56,6 +56,7 @@ import math
 import numpy as np
 
 __all__ = [
+    "gradient_mean",
     "outlier_count",
     "select_outliers",
     "outlier_mask",
@@ -64,6 +65,7 @@ __all__ = [
     "pack_codes",
     "unpack_codes",
     "dequantize",
+    "quality",
     "linear",
     "quantize_layer",
 ]
@@ -73,7 +75,7 @@ __all__ = [
 # Eq. "o": outlier location
 # --------------------------------------------------------------------------
 def gradient_mean(G_list) -> np.ndarray:
-    """Gradient mean over calibration samples (Section 4.5, "Effect on Number of Calibration"):
+    """Gradient mean over calibration samples (Section 4.3, "Effect on Number of Calibration"):
     float32 additions in list order, then one float32 division by the count."""
     acc = np.array(G_list[0], dtype=np.float32, copy=True)
     for G in G_list[1:]:

@@ -17,14 +17,15 @@ LIB_PATH = os.path.join(_HERE, "libgwq.so")
 
 GWQ_OK = 0
 (GWQ_ERR_INVALID_ARG, GWQ_ERR_UNSUPPORTED, GWQ_ERR_ALLOC, GWQ_ERR_NONFINITE, GWQ_ERR_TIMEOUT,
- GWQ_ERR_CUDA) = range(1, 7)
+ GWQ_ERR_CUDA, GWQ_ERR_WORKSPACE) = range(1, 8)
 GWQ_F16, GWQ_BF16, GWQ_F32 = 0, 1, 2
 STATUS_NAMES = {
     0: "GWQ_OK", 1: "GWQ_ERR_INVALID_ARG", 2: "GWQ_ERR_UNSUPPORTED", 3: "GWQ_ERR_ALLOC",
-    4: "GWQ_ERR_NONFINITE", 5: "GWQ_ERR_TIMEOUT", 6: "GWQ_ERR_CUDA",
+    4: "GWQ_ERR_NONFINITE", 5: "GWQ_ERR_TIMEOUT", 6: "GWQ_ERR_CUDA", 7: "GWQ_ERR_WORKSPACE",
 }
-EXPORTS = ("gwq_select_outliers", "gwq_select_outliers_static", "gwq_pack", "gwq_linear", "gwq_linear_multi",
-           "gwq_gradient_mean", "gwq_quality", "gwq_read_probe", "gwq_linear_host", "gwq_linear_host_async", "gwq_device_status", "gwq_free", "gwq_status_string")
+EXPORTS = ("gwq_select_outliers", "gwq_select_outliers_static", "gwq_pack", "gwq_linear", "gwq_linear_ws",
+           "gwq_linear_workspace_bytes", "gwq_linear_multi",
+           "gwq_gradient_mean", "gwq_quality", "gwq_read_probe", "gwq_linear_host", "gwq_linear_host_async", "gwq_device_status", "gwq_set_wait_limit", "gwq_free", "gwq_status_string")
 GWQ_MULTI_MAX = 4
 
 
@@ -70,6 +71,11 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     lib.gwq_linear.restype = C.c_int
     lib.gwq_linear.argtypes = [C.POINTER(gwq_packed), C.c_void_p, C.c_int, C.c_int32, C.c_void_p, C.c_int,
                                C.c_void_p]
+    lib.gwq_linear_ws.restype = C.c_int
+    lib.gwq_linear_ws.argtypes = [C.POINTER(gwq_packed), C.c_void_p, C.c_int, C.c_int32, C.c_void_p, C.c_int,
+                                  C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.gwq_linear_workspace_bytes.restype = C.c_size_t
+    lib.gwq_linear_workspace_bytes.argtypes = [C.POINTER(gwq_packed), C.c_int, C.c_int32]
     lib.gwq_linear_multi.restype = C.c_int
     lib.gwq_linear_multi.argtypes = [C.POINTER(C.POINTER(gwq_packed)), C.c_int32, C.c_void_p, C.c_int, C.c_int32,
                                      C.POINTER(C.c_void_p), C.c_int, C.c_void_p]
@@ -86,6 +92,8 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     lib.gwq_linear_host_async.argtypes = lib.gwq_linear.argtypes
     lib.gwq_device_status.restype = C.c_int
     lib.gwq_device_status.argtypes = [C.POINTER(gwq_packed), C.c_void_p]
+    lib.gwq_set_wait_limit.restype = C.c_int
+    lib.gwq_set_wait_limit.argtypes = [C.POINTER(gwq_packed), C.c_int64]
     lib.gwq_free.restype = None
     lib.gwq_free.argtypes = [C.c_void_p]
     lib.gwq_status_string.restype = C.c_char_p
@@ -289,8 +297,10 @@ def gwq_pack(W: torch.Tensor, S: Outliers, bits: int, group: int) -> Packed:
 
 
 def gwq_linear(P: Packed, x: torch.Tensor, out_dtype: torch.dtype | None = None,
-               out: torch.Tensor | None = None) -> torch.Tensor:
-    """y = x (deq(Wq) + S)^T for x [M,K] fp16/bf16 on the GPU; asynchronous on the current stream."""
+               out: torch.Tensor | None = None, workspace: torch.Tensor | None = None) -> torch.Tensor:
+    """y = x (deq(Wq) + S)^T for x [M,K] fp16/bf16 on the GPU; asynchronous on the current stream.
+    Where the product needs scratch memory (gwq_linear_workspace_bytes > 0) it is taken from `workspace`
+    (a CUDA uint8 tensor) or, by default, from a new torch tensor: the library itself never allocates here."""
     lib = load_library()
     _require_cuda(x, "x")
     if x.dim() != 2 or x.shape[1] != P.K:
@@ -300,8 +310,15 @@ def gwq_linear(P: Packed, x: torch.Tensor, out_dtype: torch.dtype | None = None,
         out = torch.empty((M, P.N), dtype=out_dtype or x.dtype, device=x.device)
     else:
         _require_cuda(out, "out")
-    st = lib.gwq_linear(P._h, x.data_ptr(), _dtype_code(x.dtype), M, out.data_ptr(), _dtype_code(out.dtype),
-                        _stream_ptr())
+    xd = _dtype_code(x.dtype)
+    need = 0 if xd == GWQ_F32 else int(lib.gwq_linear_workspace_bytes(P._h, xd, M))
+    if need > 0 and (workspace is None or workspace.numel() * workspace.element_size() < need):
+        workspace = torch.empty(need, dtype=torch.uint8, device=x.device)
+    if workspace is not None:
+        st = lib.gwq_linear_ws(P._h, x.data_ptr(), xd, M, out.data_ptr(), _dtype_code(out.dtype),
+                               workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream_ptr())
+    else:
+        st = lib.gwq_linear(P._h, x.data_ptr(), xd, M, out.data_ptr(), _dtype_code(out.dtype), _stream_ptr())
     _check(st, "gwq_linear")
     return out
 
@@ -320,6 +337,10 @@ def gwq_linear_multi(Ps, x: torch.Tensor, out_dtype: torch.dtype | None = None, 
         _require_cuda(o, "out")
     if len(outs) != n or any(o.dtype != outs[0].dtype for o in outs):
         raise ValueError("one output per layer, all of one dtype")
+    if M > 32:   # no shared launch up there: one call per layer, each with the scratch it needs
+        for P, o in zip(Ps, outs):
+            gwq_linear(P, x, out=o)
+        return outs
     handles = (C.POINTER(gwq_packed) * max(n, 1))(*[P._h for P in Ps])
     ys = (C.c_void_p * max(n, 1))(*[o.data_ptr() for o in outs])
     st = lib.gwq_linear_multi(handles, n, x.data_ptr(), _dtype_code(x.dtype), M, ys,
@@ -399,6 +420,11 @@ def gwq_device_status(P: Packed) -> int:
     """Status recorded by the kernels of earlier gwq_linear calls on P (0 = ok); synchronises."""
     with torch.cuda.device(P.device):
         return int(load_library().gwq_device_status(P._h, _stream_ptr()))
+
+
+def gwq_set_wait_limit(P: Packed, cycles: int) -> None:
+    """SM cycles a bounded device-side wait may spin before the kernel gives up (negative: the default)."""
+    _check(int(load_library().gwq_set_wait_limit(P._h, int(cycles))), "gwq_set_wait_limit")
 
 
 def gwq_free(obj) -> None:

@@ -17,15 +17,29 @@ static bool prefers_tensor_core(const gwq_packed* P, int M) {
   return M > 16 && M <= GWQ_DECODE_MAX_M && P->group == 128 && P->N >= 10240 && P->K % 64 == 0 && pv->cv && pv->sz_t;
 }
 
-extern "C" gwq_status gwq_linear(const gwq_packed* P, const void* x, gwq_dtype xd, int32_t M, void* y,
-                                 gwq_dtype yd, void* stream_) {
+extern "C" size_t gwq_linear_workspace_bytes(const gwq_packed* P, gwq_dtype xd, int32_t M) {
+  if (!P || P->tag != GWQ_TAG_PACKED || !P->priv || M <= 0) return 0;
+  if (M <= GWQ_DECODE_MAX_M && !prefers_tensor_core(P, M) && gwq_decode_takes(P, M)) return 0;
+  return gwq_prefill_workspace_bytes(P, xd, M);
+}
+
+extern "C" gwq_status gwq_linear_ws(const gwq_packed* P, const void* x, gwq_dtype xd, int32_t M, void* y,
+                                    gwq_dtype yd, void* ws, size_t ws_bytes, void* stream_) {
   if (!P || P->tag != GWQ_TAG_PACKED || !P->S || !P->priv || !x || !y || M <= 0) return GWQ_ERR_INVALID_ARG;
   if (xd != GWQ_F16 && xd != GWQ_BF16) return GWQ_ERR_UNSUPPORTED;
   if (yd != GWQ_F16 && yd != GWQ_BF16 && yd != GWQ_F32) return GWQ_ERR_INVALID_ARG;
   if (!gwq_aligned16(x) || !gwq_aligned16(y)) return GWQ_ERR_INVALID_ARG;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-  if (M <= GWQ_DECODE_MAX_M && !prefers_tensor_core(P, M)) return gwq_launch_decode(P, x, xd, M, y, yd, stream);
-  return gwq_launch_prefill(P, x, xd, M, y, yd, stream);
+  if (M <= GWQ_DECODE_MAX_M && !prefers_tensor_core(P, M)) {
+    const gwq_status st = gwq_launch_decode(P, x, xd, M, y, yd, stream);
+    if (st != GWQ_ERR_UNSUPPORTED) return st;   // shapes the streaming kernel does not take: the tensor-core kernel
+  }
+  return gwq_launch_prefill(P, x, xd, M, y, yd, ws, ws_bytes, stream);
+}
+
+extern "C" gwq_status gwq_linear(const gwq_packed* P, const void* x, gwq_dtype xd, int32_t M, void* y,
+                                 gwq_dtype yd, void* stream_) {
+  return gwq_linear_ws(P, x, xd, M, y, yd, nullptr, 0, stream_);
 }
 
 extern "C" gwq_status gwq_linear_multi(const gwq_packed* const* P, int32_t count, const void* x, gwq_dtype xd,
@@ -78,8 +92,19 @@ static gwq_status linear_host(gwq_packed* P, const void* x_host, gwq_dtype xd, i
     GWQ_CUDA_TRY(cudaMalloc(&pv->y_stage, yb));
     pv->y_stage_bytes = yb;
   }
+  {
+    const size_t wb = gwq_linear_workspace_bytes(P, xd, M);
+    if (pv->ws_stage_bytes < wb) {
+      GWQ_CUDA_TRY(cudaStreamSynchronize(stream));
+      if (pv->ws_stage) cudaFree(pv->ws_stage);
+      pv->ws_stage = nullptr;
+      pv->ws_stage_bytes = 0;
+      GWQ_CUDA_TRY(cudaMalloc(&pv->ws_stage, wb));
+      pv->ws_stage_bytes = wb;
+    }
+  }
   GWQ_CUDA_TRY(cudaMemcpyAsync(pv->x_stage, x_host, xb, cudaMemcpyHostToDevice, stream));
-  st = gwq_linear(P, pv->x_stage, xd, M, pv->y_stage, yd, stream);
+  st = gwq_linear_ws(P, pv->x_stage, xd, M, pv->y_stage, yd, pv->ws_stage, pv->ws_stage_bytes, stream);
   if (st != GWQ_OK) return st;
   GWQ_CUDA_TRY(cudaMemcpyAsync(y_host, pv->y_stage, yb, cudaMemcpyDeviceToHost, stream));
   if (synchronise) GWQ_CUDA_TRY(cudaStreamSynchronize(stream));
@@ -112,6 +137,12 @@ extern "C" gwq_status gwq_device_status(const gwq_packed* P, void* stream_) {
   return (gwq_status)h;
 }
 
+extern "C" gwq_status gwq_set_wait_limit(gwq_packed* P, int64_t cycles) {
+  if (!P || P->tag != GWQ_TAG_PACKED || !P->priv) return GWQ_ERR_INVALID_ARG;
+  static_cast<gwq_priv*>(P->priv)->wait_cycles = cycles < 0 ? GWQ_DEFAULT_WAIT_CYCLES : (long long)cycles;
+  return GWQ_OK;
+}
+
 static void free_outliers(gwq_outliers* S) {
   if (!S) return;
   if (S->row_ptr) cudaFree(S->row_ptr);
@@ -137,7 +168,7 @@ extern "C" void gwq_free(void* obj) {
       if (pv->cv) cudaFree(pv->cv);
       if (pv->x_stage) cudaFree(pv->x_stage);
       if (pv->y_stage) cudaFree(pv->y_stage);
-      if (pv->x16) cudaFree(pv->x16);
+      if (pv->ws_stage) cudaFree(pv->ws_stage);
       if (pv->xt) cudaFree(pv->xt);
       if (pv->sz_t) cudaFree(pv->sz_t);
       if (pv->dev_status) cudaFree(pv->dev_status);
@@ -157,6 +188,7 @@ extern "C" const char* gwq_status_string(gwq_status s) {
     case GWQ_ERR_NONFINITE: return "GWQ_ERR_NONFINITE";
     case GWQ_ERR_TIMEOUT: return "GWQ_ERR_TIMEOUT";
     case GWQ_ERR_CUDA: return "GWQ_ERR_CUDA";
+    case GWQ_ERR_WORKSPACE: return "GWQ_ERR_WORKSPACE";
   }
   return "GWQ_ERR_UNKNOWN";
 }

@@ -30,13 +30,16 @@ struct gwq_priv {
   size_t x_stage_bytes;
   size_t y_stage_bytes;
   uint32_t* sz_t;        // [K/group][N]: scale fp16 bits | zero-point << 16 (tensor-core path)
-  void* x16;             // fp16 copy of bf16 activations for the tensor-core path (+ per-token scales)
-  size_t x16_bytes;
-  void* xt;              // token-major copy [K][tokens] of the activations (decode path, outlier gathers)
-  size_t xt_bytes;
+  void* ws_stage;        // scratch for gwq_linear_host where the product needs some
+  size_t ws_stage_bytes;
+  void* xt;              // token-major copy [K][32] of the activations and their group sums (decode path with more
+  size_t xt_bytes;       // than 8 tokens); created by gwq_pack
   int32_t* dev_status;   // device status word written by bounded waits
   int sm_count;
+  long long wait_cycles; // SM cycles a bounded device-side wait may spin (gwq_set_wait_limit)
 };
+
+#define GWQ_DEFAULT_WAIT_CYCLES (1000LL * 1000LL * 1000LL)
 
 static inline bool gwq_aligned16(const void* p) {
   return (reinterpret_cast<uintptr_t>(p) & 15u) == 0;
@@ -50,4 +53,7 @@ gwq_status gwq_launch_decode(const gwq_packed* P, const void* x, gwq_dtype xd, i
 gwq_status gwq_launch_decode_multi(const gwq_packed* const* P, int count, const void* x, gwq_dtype xd, int M,
                                    void* const* y, gwq_dtype yd, cudaStream_t stream);
 gwq_status gwq_launch_prefill(const gwq_packed* P, const void* x, gwq_dtype xd, int M, void* y,
-                              gwq_dtype yd, cudaStream_t stream);
+                              gwq_dtype yd, void* ws, size_t ws_bytes, cudaStream_t stream);
+size_t gwq_prefill_workspace_bytes(const gwq_packed* P, gwq_dtype xd, int M);
+bool gwq_decode_takes(const gwq_packed* P, int M);   // the streaming kernel has a variant for (P, M)
+size_t gwq_decode_scratch_bytes(int K);              // bytes of gwq_priv::xt

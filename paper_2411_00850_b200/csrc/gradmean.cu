@@ -1,4 +1,4 @@
-// Mean of the gradients of several calibration samples (Section 4.5, "Effect on Number of
+// Mean of the gradients of several calibration samples (Section 4.3, "Effect on Number of
 // Calibration": the outliers are located on the gradient mean).  One pass over all samples; the
 // arithmetic is fixed so that the result is reproducible bit for bit: FP32 additions in sample order
 // (round to nearest), then one FP32 division by the count.

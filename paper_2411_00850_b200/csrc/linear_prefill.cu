@@ -34,7 +34,7 @@ constexpr int kDequantGroups = 3;  // groups; group g takes the k-blocks g, g + 
 constexpr int kEpilogueWarps = 4;  // one thread per tile row
 constexpr int kCtaThreads = 32 * (2 + kDequantWarps * kDequantGroups + kEpilogueWarps);
 constexpr int kMaxStages = 8;
-constexpr long long kSpinCycles = 1000LL * 1000LL * 1000LL;   // about half a second of SM clock
+constexpr long long kSpinCycles = GWQ_DEFAULT_WAIT_CYCLES;   // about half a second of SM clock
 
 __device__ __forceinline__ unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
 
@@ -47,19 +47,27 @@ __device__ __forceinline__ void mbar_arrive(unsigned bar) {
 __device__ __forceinline__ void mbar_expect_tx(unsigned bar, unsigned bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-// Bounded wait for the phase with the given parity: gives up (false) after kSpinCycles, or as
-// soon as another role of the CTA has given up.
-__device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity, volatile int* abort_flag) {
+// Bounded wait for the phase with the given parity: gives up (false) after `limit` cycles, or as
+// soon as another role of the CTA has given up.  A first, non-blocking test decides the common case and
+// makes a limit of zero mean exactly "give up unless the phase has completed already".
+__device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity, volatile int* abort_flag, long long limit) {
+  unsigned done;
+  asm volatile(
+      "{\n .reg .pred p;\n mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.b32 %0, 1, 0, p;\n}\n"
+      : "=r"(done)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  if (done) return true;
+  if (limit <= 0) return false;
   const long long t0 = clock64();
   for (unsigned it = 0;; ++it) {
-    unsigned done;
     asm volatile(
         "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.b32 %0, 1, 0, p;\n}\n"
         : "=r"(done)
         : "r"(bar), "r"(parity)
         : "memory");
     if (done) return true;
-    if ((it & 63u) == 63u && (*abort_flag || clock64() - t0 > kSpinCycles)) return false;
+    if ((it & 63u) == 63u && (*abort_flag || clock64() - t0 > limit)) return false;
   }
 }
 
@@ -118,6 +126,7 @@ struct PrefillArgs {
   int32_t* status;
   const float* tok_scale;   // per token 2^e, or null (activations were fp16 already)
   int N, K, M, group;
+  long long wait_cycles;    // limit of every hand-over wait (the waits of the give-up path keep the default)
 };
 
 // bf16 [M,K] -> fp16 [M,K] scaled per token row by a power of two that puts the row's largest
@@ -212,7 +221,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmx, const PrefillArgs p, con
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* tiles =
       reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
-  __shared__ __align__(8) unsigned long long bars[3 * kMaxStages + 4];
+  __shared__ __align__(8) unsigned long long bars[3 * kMaxStages + 5];
   __shared__ unsigned tmem_base_s;
   __shared__ int abort_s;
   volatile int* abort_flag = &abort_s;
@@ -225,6 +234,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmx, const PrefillArgs p, con
   auto empty = [&](int s) { return bar0 + 8u * (2 * kMaxStages + s); };
   auto acc_full = [&](int a) { return bar0 + 8u * (3 * kMaxStages + a); };
   auto acc_empty = [&](int a) { return bar0 + 8u * (3 * kMaxStages + 2 + a); };
+  const unsigned drain_bar = bar0 + 8u * (3 * kMaxStages + 4);   // give-up path: completion of the MMAs in flight
+  const long long lim = p.wait_cycles;
   auto a_tile = [&](int s) { return tiles + (size_t)s * (kABytes + kBBytes); };
   auto b_tile = [&](int s) { return tiles + (size_t)s * (kABytes + kBBytes) + kABytes; };
   // this CTA's tiles: blockIdx.x, blockIdx.x + gridDim.x, ...; the feature tile runs fastest, so the CTAs
@@ -242,6 +253,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmx, const PrefillArgs p, con
       mbar_init(acc_full(a), 1);
       mbar_init(acc_empty(a), kEpilogueWarps);
     }
+    mbar_init(drain_bar, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {   // tensor memory: two accumulators of kAccCols columns x 128 lanes
@@ -265,7 +277,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmx, const PrefillArgs p, con
         const int m0 = (tile / ntn) * TOK;
         for (int kb = 0; kb < nkb && ok; ++kb) {
           const int it = ti * nkb + kb, s = it % stages, round = it / stages;
-          if (round > 0) ok = mbar_wait(empty(s), (round - 1) & 1, abort_flag);
+          if (round > 0) ok = mbar_wait(empty(s), (round - 1) & 1, abort_flag, lim);
           if (!ok) break;
           mbar_expect_tx(full_b(s), kBBytes);
           tma_load_2d(smem_u32(b_tile(s)), &tmx, kb * kBlockK, m0, full_b(s));
@@ -281,13 +293,13 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmx, const PrefillArgs p, con
                              ((unsigned)(TOK >> 3) << 17) | ((unsigned)(kTileN >> 4) << 24);
       for (int ti = 0; ti < my_tiles && ok; ++ti) {
         const int a = ti & 1;
-        if (ti >= 2) ok = mbar_wait(acc_empty(a), ((ti >> 1) - 1) & 1, abort_flag);   // drained by the epilogue
+        if (ti >= 2) ok = mbar_wait(acc_empty(a), ((ti >> 1) - 1) & 1, abort_flag, lim);   // drained by the epilogue
         if (!ok) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const unsigned acc = tmem_acc + (unsigned)(a * kAccCols);
         for (int kb = 0; kb < nkb && ok; ++kb) {
           const int it = ti * nkb + kb, s = it % stages, round = it / stages;
-          ok = mbar_wait(full_a(s), round & 1, abort_flag) && mbar_wait(full_b(s), round & 1, abort_flag);
+          ok = mbar_wait(full_a(s), round & 1, abort_flag, lim) && mbar_wait(full_b(s), round & 1, abort_flag, lim);
           if (!ok) break;
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           const uint64_t da = umma_desc(smem_u32(a_tile(s))), db = umma_desc(smem_u32(b_tile(s)));
@@ -375,7 +387,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmx, const PrefillArgs p, con
             out[16 * run + 15] = mul_scale<BF16>(sub_magic<BF16>(last | MAGIC, zm), s_hi2, s_lo2);
           }
         }
-        if (round > 0) ok = mbar_wait(empty(s), (round - 1) & 1, abort_flag);
+        if (round > 0) ok = mbar_wait(empty(s), (round - 1) & 1, abort_flag, lim);
         if (!ok) break;
         unsigned char* arow = a_tile(s) + r * 128;
 #pragma unroll
@@ -411,7 +423,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmx, const PrefillArgs p, con
       const int row = (tile % ntn) * kTileN + r, m0 = (tile / ntn) * TOK;
       const bool live = row < p.N;
       const int a = ti & 1;
-      ok = mbar_wait(acc_full(a), (ti >> 1) & 1, abort_flag);
+      ok = mbar_wait(acc_full(a), (ti >> 1) & 1, abort_flag, lim);
       if (!ok) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll 1
@@ -454,9 +466,16 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmx, const PrefillArgs p, con
     for (int s = 0; s < stages; ++s) {
       if (issued > s) {
         const int last_it = ((issued - 1 - s) / stages) * stages + s;   // last copy issued on stage s
-        (void)mbar_wait(full_b(s), (last_it / stages) & 1, &zero);
+        (void)mbar_wait(full_b(s), (last_it / stages) & 1, &zero, kSpinCycles);
       }
     }
+  }
+  if (warp == 1 && lane == 0 && abort_s) {
+    // MMAs that were issued may still read the stages and write tensor memory: one more commit arrives when all
+    // of them have completed; wait (bounded) for it before the tensor memory is freed
+    int zero = 0;
+    umma_commit(drain_bar);
+    (void)mbar_wait(drain_bar, 0, &zero, kSpinCycles);
   }
   __syncthreads();
   if (warp == 1) {
@@ -507,6 +526,7 @@ gwq_status launch(const gwq_packed* P, const void* x, const float* tok_scale, in
   PrefillArgs a;
   a.codes = P->codes; a.scales = P->scales; a.zeros = P->zeros; a.row_ptr = P->S->row_ptr; a.cv = pv->cv; a.sz_t = pv->sz_t;
   a.y = y; a.yd = yd; a.status = pv->dev_status; a.tok_scale = tok_scale; a.N = P->N; a.K = P->K; a.M = M; a.group = P->group;
+  a.wait_cycles = pv->wait_cycles;
   const int ntn = (P->N + kTileN - 1) / kTileN, ntiles = ntn * ((M + TOK - 1) / TOK);
   const int grid = ntiles < pv->sm_count ? ntiles : pv->sm_count;   // persistent: at most one CTA per SM
   prefill_kernel<BITS, TOK, BF16><<<grid, kCtaThreads, smem, stream>>>(tmx, a, stages, ntn, ntiles);
@@ -524,32 +544,29 @@ gwq_status launch_tok(const gwq_packed* P, const void* x, const float* tok_scale
 
 }  // namespace
 
+// Scratch of the tensor-core path: bf16 activations need an fp16 copy of x and one scale per token.
+size_t gwq_prefill_workspace_bytes(const gwq_packed* P, gwq_dtype xd, int M) {
+  const gwq_priv* pv = static_cast<const gwq_priv*>(P->priv);
+  if (!pv->cv || !pv->sz_t || P->K % kBlockK != 0) return 0;   // the general kernel needs none
+  if (xd != GWQ_BF16) return 0;
+  return (((size_t)M * P->K * 2 + 255) & ~(size_t)255) + (((size_t)M * 4 + 255) & ~(size_t)255);
+}
+
 // Prefill launcher: K <= 65536 (16-bit outlier columns).  Other shapes go to the general kernel.
-// bf16 activations need a scratch copy of x in fp16 (M K 2 bytes + M 4 bytes), kept in the packed
-// object and grown on demand (a growing call synchronises the stream and allocates).
+// bf16 activations are first rewritten into the caller's workspace (fp16 copy of x and the token scales).
 gwq_status gwq_launch_prefill(const gwq_packed* P, const void* x, gwq_dtype xd, int M, void* y, gwq_dtype yd,
-                              cudaStream_t stream) {
-  gwq_priv* pv = static_cast<gwq_priv*>(P->priv);
+                              void* ws, size_t ws_bytes, cudaStream_t stream) {
+  const gwq_priv* pv = static_cast<const gwq_priv*>(P->priv);
   if (!pv->cv || !pv->sz_t || P->K % kBlockK != 0) return gwq_launch_simt(P, x, xd, M, y, yd, stream);
   const float* tok_scale = nullptr;
   if (xd == GWQ_BF16) {
-    const size_t need = (size_t)M * P->K * 2 + (size_t)M * 4 + 256;
-    if (pv->x16_bytes < need) {
-      if (cudaStreamSynchronize(stream) != cudaSuccess) return GWQ_ERR_CUDA;
-      if (pv->x16) cudaFree(pv->x16);
-      pv->x16 = nullptr;
-      pv->x16_bytes = 0;
-      if (cudaMalloc(&pv->x16, need) != cudaSuccess) {
-        (void)cudaGetLastError();
-        return GWQ_ERR_ALLOC;
-      }
-      pv->x16_bytes = need;
-    }
-    float* ts = reinterpret_cast<float*>(static_cast<char*>(pv->x16) + (((size_t)M * P->K * 2 + 255) & ~(size_t)255));
-    bf16_rows_to_scaled_f16<<<M, 256, 0, stream>>>(static_cast<const uint16_t*>(x), static_cast<uint16_t*>(pv->x16), ts,
-                                                   P->K);
+    const size_t need = gwq_prefill_workspace_bytes(P, xd, M);
+    if (!ws || ws_bytes < need || (reinterpret_cast<uintptr_t>(ws) & 255u) != 0) return GWQ_ERR_WORKSPACE;
+    uint16_t* x16 = static_cast<uint16_t*>(ws);
+    float* ts = reinterpret_cast<float*>(static_cast<char*>(ws) + (((size_t)M * P->K * 2 + 255) & ~(size_t)255));
+    bf16_rows_to_scaled_f16<<<M, 256, 0, stream>>>(static_cast<const uint16_t*>(x), x16, ts, P->K);
     if (cudaGetLastError() != cudaSuccess) return GWQ_ERR_CUDA;
-    x = pv->x16;
+    x = x16;
     tok_scale = ts;
   }
   if (P->bits == 4) return launch_tok<4>(P, x, tok_scale, M, y, yd, stream);

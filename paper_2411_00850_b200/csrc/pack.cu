@@ -205,6 +205,7 @@ extern "C" gwq_status gwq_pack(const uint16_t* W, gwq_outliers* S, int32_t N, in
     return GWQ_ERR_ALLOC;
   }
   *pv = gwq_priv{};
+  pv->wait_cycles = GWQ_DEFAULT_WAIT_CYCLES;
   P->tag = GWQ_TAG_PACKED;
   P->N = N; P->K = K; P->bits = bits; P->group = group;
   P->codes = nullptr; P->scales = nullptr; P->zeros = nullptr; P->S = nullptr; P->priv = pv;
@@ -236,6 +237,10 @@ extern "C" gwq_status gwq_pack(const uint16_t* W, gwq_outliers* S, int32_t N, in
       GWQ_CUDA_TRY(cudaGetLastError());
     }
   }
+  if (K <= 65536 && group >= 64 && K % 128 == 0) {   // scratch of the streaming path with more than 8 tokens
+    GWQ_CUDA_TRY(cudaMalloc(&pv->xt, gwq_decode_scratch_bytes(K)));
+    pv->xt_bytes = gwq_decode_scratch_bytes(K);
+  }
   if (group >= 64) {   // the tensor-core path (one scale per 64-column k-block) takes groups of 64 and 128 only
     GWQ_CUDA_TRY(cudaMalloc(&pv->sz_t, ngroups * sizeof(uint32_t) + 16));
     transpose_scale_zero_kernel<<<(unsigned)((ngroups + 255) / 256), 256, 0, stream>>>(P->scales, P->zeros, pv->sz_t,
@@ -258,6 +263,7 @@ fail:
   if (P->zeros) cudaFree(P->zeros);
   if (pv->cv) cudaFree(pv->cv);
   if (pv->sz_t) cudaFree(pv->sz_t);
+  if (pv->xt) cudaFree(pv->xt);
   if (pv->dev_status) cudaFree(pv->dev_status);
   delete pv;
   delete P;

@@ -25,6 +25,14 @@ struct SelState {
 
 __device__ __forceinline__ unsigned int abs_key(unsigned int bits) { return bits & 0x7FFFFFFFu; }
 
+// Start of a selection: clears the histogram and the state words and sets the count to take (a kernel
+// argument, so nothing is copied from host memory that the caller might reuse).
+__global__ void __launch_bounds__(kThreads) sel_init_kernel(unsigned int* __restrict__ scratch, unsigned int k_out) {
+  for (int i = threadIdx.x; i < kBins + 4; i += kThreads) scratch[i] = 0u;
+  __syncthreads();
+  if (threadIdx.x == 0) reinterpret_cast<SelState*>(scratch + kBins)->k_rem = k_out;
+}
+
 // Histogram of one radix digit over the keys that match the decided prefix.
 __global__ void __launch_bounds__(kThreads) sel_hist_kernel(const uint4* __restrict__ G4, long long n4,
                                                             const SelState* __restrict__ st,
@@ -261,11 +269,7 @@ cudaError_t gwq_select_run(const uint16_t* W, const float* G, int N, int K, unsi
   unsigned int* take = n_tie + N;
   const long long numel = (long long)N * K;
   const long long n4 = numel / 4;
-  cudaError_t e;
-  if ((e = cudaMemsetAsync(scratch, 0, (kBins + 4) * sizeof(unsigned int), stream)) != cudaSuccess) return e;
-  if ((e = cudaMemcpyAsync(&st->k_rem, &k_out, sizeof(unsigned int), cudaMemcpyHostToDevice, stream)) !=
-      cudaSuccess)
-    return e;
+  sel_init_kernel<<<1, kThreads, 0, stream>>>(scratch, k_out);
   long long want = (n4 + kThreads - 1) / kThreads;
   const int grid = (int)(want < (long long)sm_count * 8 ? (want > 0 ? want : 1) : (long long)sm_count * 8);
   const int shifts[3] = {20, 10, 0}, nbits[3] = {11, 10, 10};

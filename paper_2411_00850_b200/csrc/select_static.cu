@@ -5,6 +5,8 @@
 // coming from cudaMalloc, and the CSR arrays are supplied by the caller.
 #include <math.h>
 
+#include <mutex>
+
 #include "common.cuh"
 
 // Implemented next to the selection kernels.
@@ -16,31 +18,36 @@ cudaError_t gwq_select_run(const uint16_t* W, const float* G, int N, int K, unsi
 #define GWQ_STATIC_MAX_ROWS 32768
 #define GWQ_STATIC_SCRATCH_WORDS (2048 + 4 + 3 * GWQ_STATIC_MAX_ROWS)
 
-// ~386 KiB of device memory, held by every GPU that loads this library until the
-// process exits.  Shared by all calls: its contents are whatever the last call left.
+// 401 424 bytes (392 KiB) of device memory, held by every GPU that loads this library until
+// the process exits.  Shared by all calls: its contents are whatever the last call left.
 static __device__ __align__(256) unsigned int g_select_scratch[GWQ_STATIC_SCRATCH_WORDS];
 
 namespace {
 constexpr int kMaxDevices = 64;
 unsigned int* g_scratch_addr[kMaxDevices] = {nullptr};
 int g_sm_count[kMaxDevices] = {0};
+gwq_status g_lookup_status[kMaxDevices] = {GWQ_OK};
+std::once_flag g_lookup_once[kMaxDevices];
 
 // The symbol's name is only a host-side handle; the kernels need its device address,
-// which differs per GPU.  Looked up once per device, with that device current.
+// which differs per GPU.  Looked up once per device, with that device current; host
+// threads that make their first call at the same time wait for the one lookup.
 gwq_status scratch_for_current_device(unsigned int** ptr, int* sms) {
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return GWQ_ERR_CUDA;
-  if (!g_scratch_addr[dev]) {
+  std::call_once(g_lookup_once[dev], [dev]() {
     void* p = nullptr;
-    if (cudaGetSymbolAddress(&p, g_select_scratch) != cudaSuccess || !p) {
-      (void)cudaGetLastError();
-      return GWQ_ERR_CUDA;
-    }
     int n = 0;
-    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return GWQ_ERR_CUDA;
+    if (cudaGetSymbolAddress(&p, g_select_scratch) != cudaSuccess || !p ||
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+      (void)cudaGetLastError();
+      g_lookup_status[dev] = GWQ_ERR_CUDA;
+      return;
+    }
     g_sm_count[dev] = n;
     g_scratch_addr[dev] = static_cast<unsigned int*>(p);
-  }
+  });
+  if (g_lookup_status[dev] != GWQ_OK) return g_lookup_status[dev];
   *ptr = g_scratch_addr[dev];
   *sms = g_sm_count[dev];
   return GWQ_OK;
@@ -64,7 +71,10 @@ extern "C" gwq_status gwq_select_outliers_static(const uint16_t* W, const float*
   if (kd < 0) kd = 0;
   if (kd > (double)numel) kd = (double)numel;
   const long long k_out = (long long)kd;
-  if (capacity < k_out) return GWQ_ERR_INVALID_ARG;  // caller's col_idx / val are too short
+  if (capacity < k_out) {  // caller's col_idx / val are too short: report the size they need
+    *nnz_host = k_out;
+    return GWQ_ERR_INVALID_ARG;
+  }
 
   unsigned int* scratch = nullptr;
   int sms = 0;

@@ -84,3 +84,16 @@ def test_tall_layers_take_the_tensor_core_kernel_from_17_tokens():
     # and shorter layers stay on the streaming kernel; fused siblings follow the same rule
     _check(10368, 512, 0.01, 4, 128, 90, [(16, "f16"), (17, "f16"), (24, "bf16"), (32, "f16"), (32, "bf16")])
     _check(10240, 256, 0.01, 3, 128, 91, [(17, "bf16"), (32, "f16")])
+
+
+@pytest.mark.parametrize("bits", [4, 3])
+def test_two_tiles_per_cta(bits):
+    # 8192 rows: more 16-row blocks than one wave of CTAs, at most one wave of 32-row blocks, so up to 8 tokens the
+    # streaming kernel runs with two m16 tiles per CTA (staged activations here; a ragged last block: 8200 rows)
+    _check(8192, 256, 0.01, bits, 128, 92 + bits, [(1, "f16"), (1, "bf16"), (3, "f16"), (8, "f16"), (8, "bf16"), (16, "f16")])
+    _check(8200, 128, 0.02, bits, 128, 96 + bits, [(1, "f16"), (5, "bf16")])
+
+
+def test_two_tiles_per_cta_with_activation_ring():
+    # 8 tokens of 6144 activations do not fit up front: per-warp rings, two tiles per CTA (7168 rows)
+    _check(7168, 6144, 0.01, 4, 128, 99, [(8, "f16"), (7, "bf16"), (1, "f16")])

@@ -1,4 +1,4 @@
-"""GPU parity of gwq_gradient_mean (Section 4.5: outliers located on the mean of the calibration
+"""GPU parity of gwq_gradient_mean (Section 4.3: outliers located on the mean of the calibration
 samples' gradients) against the CPU checker: same FP32 additions in the same order, so bit for bit,
 and the outlier set selected on the mean."""
 import numpy as np

@@ -91,6 +91,43 @@ def test_tensor_core_path(layer, M, dtype):
     assert_linear_close(y16, y_ref, bound, extra_rel=2.0 ** -8 if dtype == "bf16" else 0.0)
 
 
+@pytest.mark.parametrize("bits,dtype", [(4, "f16"), (3, "bf16")])
+def test_persistent_ctas_with_several_tiles_each(bits, dtype):
+    # N = 4096, K = 256, M = 4096: 32 x 16 = 512 tiles of 128 rows x 256 tokens on at most 148 persistent CTAs, so
+    # every CTA computes three or four tiles: both accumulators are reused (the wait for the epilogue to drain
+    # them), the stage ring wraps across tiles, and every output is checked
+    N, K, M = 4096, 256, 4096
+    W, G = synth.make_weight_and_grad(N, K, 26)
+    L = orc.quantize_layer(W, G, 0.01, bits, 128)
+    P = quantize_on_gpu(W, G, 0.01, bits, 128)
+    assert_packed_equal(P, L)
+    w_hat = oracle_w_hat(L)
+    bits16, xv = synth.make_activations(M, K, seed=126, dtype=dtype, heavy_channels=8)
+    y_ref, bound = orc.linear(xv, w_hat)
+    y = gwq.gwq_linear(P, x_tensor(bits16, dtype), out_dtype=torch.float32)
+    assert gwq.gwq_device_status(P) == 0
+    assert_linear_close(y, y_ref, bound)
+    P.free()
+
+
+def test_single_layer_config_seed_0():
+    # the single-layer configuration as written: 4096 x 4096, seed 0, 4 bits, groups of 128, 1 % outliers, fp16
+    # activations, one token; encoding bit for bit and every output
+    N = K = 4096
+    W, G = synth.make_weight_and_grad(N, K, synth.layer_seed(0, 0))
+    L = orc.quantize_layer(W, G, 0.01, 4, 128)
+    assert int(L["row_ptr"][-1]) == 167773
+    P = quantize_on_gpu(W, G, 0.01, 4, 128)
+    assert_packed_equal(P, L)
+    w_hat = oracle_w_hat(L)
+    bits16, xv = synth.make_activations(1, K, seed=synth.layer_seed(0, 0), dtype="f16")
+    y_ref, bound = orc.linear(xv, w_hat)
+    for out_dtype in (torch.float32, torch.float16):
+        y = gwq.gwq_linear(P, x_tensor(bits16, "f16"), out_dtype=out_dtype)
+        assert_linear_close(y, y_ref, bound)
+    P.free()
+
+
 def test_tensor_core_path_reads_back_columns_exactly_in_fp16():
     # one-hot fp16 activations: y[m] is column c of the reconstructed weight, outliers included
     P, L, w_hat = _layer(*PREFILL_LAYERS[0])

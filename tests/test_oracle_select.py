@@ -123,7 +123,7 @@ def test_select_special_values_order():
     assert len(ci) == 26 and zero_cols_taken == [0, 1]
 
 
-# ---------------------------------------------------------------- gradient mean over calibration samples (Section 4.5)
+# ---------------------------------------------------------------- gradient mean over calibration samples (Section 4.3)
 def test_gradient_mean_pins():
     rng = np.random.default_rng(21)
     G = rng.normal(size=(6, 8, 32)).astype(np.float32)
