@@ -323,7 +323,8 @@ def gwq_linear(P: Packed, x: torch.Tensor, out_dtype: torch.dtype | None = None,
     return out
 
 
-def gwq_linear_multi(Ps, x: torch.Tensor, out_dtype: torch.dtype | None = None, outs=None):
+def gwq_linear_multi(Ps, x: torch.Tensor, out_dtype: torch.dtype | None = None, outs=None,
+                     workspace: torch.Tensor | None = None):
     """[x (deq(P) + S_P)^T for P in Ps] for layers that read the same x [M,K]: one call, and for M <= 32 one launch."""
     lib = load_library()
     _require_cuda(x, "x")
@@ -337,9 +338,13 @@ def gwq_linear_multi(Ps, x: torch.Tensor, out_dtype: torch.dtype | None = None, 
         _require_cuda(o, "out")
     if len(outs) != n or any(o.dtype != outs[0].dtype for o in outs):
         raise ValueError("one output per layer, all of one dtype")
-    if M > 32:   # no shared launch up there: one call per layer, each with the scratch it needs
+    xd = _dtype_code(x.dtype)
+    need = 0 if xd == GWQ_F32 else max(int(lib.gwq_linear_workspace_bytes(P._h, xd, M)) for P in Ps)
+    if need > 0:   # products that take scratch memory: one call per layer, all on the same workspace (stream order)
+        if workspace is None or workspace.numel() * workspace.element_size() < need:
+            workspace = torch.empty(need, dtype=torch.uint8, device=x.device)
         for P, o in zip(Ps, outs):
-            gwq_linear(P, x, out=o)
+            gwq_linear(P, x, out=o, workspace=workspace)
         return outs
     handles = (C.POINTER(gwq_packed) * max(n, 1))(*[P._h for P in Ps])
     ys = (C.c_void_p * max(n, 1))(*[o.data_ptr() for o in outs])

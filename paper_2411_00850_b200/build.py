@@ -14,7 +14,7 @@ CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libgwq.so")
 SOURCES = ("decode_w4_f16.cu", "decode_w4_bf16.cu", "decode_w3_f16.cu", "decode_w3_bf16.cu", "select.cu",
-           "select_static.cu", "pack.cu", "linear_simt.cu", "linear_decode.cu", "linear_prefill.cu", "probe.cu",
+           "select_static.cu", "pack.cu", "linear_simt.cu", "linear_decode.cu", "linear_skinny.cu", "linear_prefill.cu", "probe.cu",
            "quality.cu", "gradmean.cu", "api.cu")
 NVCC_FLAGS = (
     "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",

@@ -17,8 +17,17 @@ static bool prefers_tensor_core(const gwq_packed* P, int M) {
   return M > 16 && M <= GWQ_DECODE_MAX_M && P->group == 128 && P->N >= 10240 && P->K % 64 == 0 && pv->cv && pv->sz_t;
 }
 
+#ifndef GWQ_TUNE_SKINNY_MIN_M
+#define GWQ_TUNE_SKINNY_MIN_M 9   // fewest tokens that go to the tcgen05 streaming kernel when a workspace is given
+#endif
+
+static bool wants_skinny(const gwq_packed* P, gwq_dtype xd, int M) {
+  return M >= GWQ_TUNE_SKINNY_MIN_M && M <= GWQ_DECODE_MAX_M && gwq_skinny_takes(P, xd, M);
+}
+
 extern "C" size_t gwq_linear_workspace_bytes(const gwq_packed* P, gwq_dtype xd, int32_t M) {
   if (!P || P->tag != GWQ_TAG_PACKED || !P->priv || M <= 0) return 0;
+  if (wants_skinny(P, xd, M)) return gwq_skinny_workspace_bytes(P, M);
   if (M <= GWQ_DECODE_MAX_M && !prefers_tensor_core(P, M) && gwq_decode_takes(P, M)) return 0;
   return gwq_prefill_workspace_bytes(P, xd, M);
 }
@@ -30,6 +39,9 @@ extern "C" gwq_status gwq_linear_ws(const gwq_packed* P, const void* x, gwq_dtyp
   if (yd != GWQ_F16 && yd != GWQ_BF16 && yd != GWQ_F32) return GWQ_ERR_INVALID_ARG;
   if (!gwq_aligned16(x) || !gwq_aligned16(y)) return GWQ_ERR_INVALID_ARG;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  // with a workspace, 9 to 32 fp16 tokens take the tcgen05 streaming kernel; without one the older kernels serve them
+  if (wants_skinny(P, xd, M) && ws && ws_bytes >= gwq_skinny_workspace_bytes(P, M))
+    return gwq_launch_skinny(P, x, M, y, yd, ws, ws_bytes, stream);
   if (M <= GWQ_DECODE_MAX_M && !prefers_tensor_core(P, M)) {
     const gwq_status st = gwq_launch_decode(P, x, xd, M, y, yd, stream);
     if (st != GWQ_ERR_UNSUPPORTED) return st;   // shapes the streaming kernel does not take: the tensor-core kernel

@@ -55,5 +55,9 @@ gwq_status gwq_launch_decode_multi(const gwq_packed* const* P, int count, const 
 gwq_status gwq_launch_prefill(const gwq_packed* P, const void* x, gwq_dtype xd, int M, void* y,
                               gwq_dtype yd, void* ws, size_t ws_bytes, cudaStream_t stream);
 size_t gwq_prefill_workspace_bytes(const gwq_packed* P, gwq_dtype xd, int M);
+bool gwq_skinny_takes(const gwq_packed* P, gwq_dtype xd, int M);
+size_t gwq_skinny_workspace_bytes(const gwq_packed* P, int M);
+gwq_status gwq_launch_skinny(const gwq_packed* P, const void* x, int M, void* y, gwq_dtype yd, void* ws, size_t ws_bytes,
+                             cudaStream_t stream);
 bool gwq_decode_takes(const gwq_packed* P, int M);   // the streaming kernel has a variant for (P, M)
 size_t gwq_decode_scratch_bytes(int K);              // bytes of gwq_priv::xt

@@ -21,11 +21,10 @@
 // multiplies the token's column by 2^e again.  fp16 also keeps the FP16 outliers exact.
 // Stages are handed over with mbarriers; every wait is bounded and, when it runs out, the CTA
 // records GWQ_ERR_TIMEOUT, leaves its loops, frees its tensor memory and returns.
-#include <cuda.h>
-
-#include "common.cuh"
+#include "tc_common.cuh"
 
 namespace {
+using namespace gwq_tc;
 
 constexpr int kTileN = 128;      // weight rows per CTA (UMMA M)
 constexpr int kBlockK = 64;      // k-block: 128 bytes of 16-bit operands
@@ -34,85 +33,6 @@ constexpr int kDequantGroups = 3;  // groups; group g takes the k-blocks g, g + 
 constexpr int kEpilogueWarps = 4;  // one thread per tile row
 constexpr int kCtaThreads = 32 * (2 + kDequantWarps * kDequantGroups + kEpilogueWarps);
 constexpr int kMaxStages = 8;
-constexpr long long kSpinCycles = GWQ_DEFAULT_WAIT_CYCLES;   // about half a second of SM clock
-
-__device__ __forceinline__ unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(unsigned bar, unsigned count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_arrive(unsigned bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(unsigned bar, unsigned bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-// Bounded wait for the phase with the given parity: gives up (false) after `limit` cycles, or as
-// soon as another role of the CTA has given up.  A first, non-blocking test decides the common case and
-// makes a limit of zero mean exactly "give up unless the phase has completed already".
-__device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity, volatile int* abort_flag, long long limit) {
-  unsigned done;
-  asm volatile(
-      "{\n .reg .pred p;\n mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.b32 %0, 1, 0, p;\n}\n"
-      : "=r"(done)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  if (done) return true;
-  if (limit <= 0) return false;
-  const long long t0 = clock64();
-  for (unsigned it = 0;; ++it) {
-    asm volatile(
-        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.b32 %0, 1, 0, p;\n}\n"
-        : "=r"(done)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    if (done) return true;
-    if ((it & 63u) == 63u && (*abort_flag || clock64() - t0 > limit)) return false;
-  }
-}
-
-__device__ __forceinline__ void tma_load_2d(unsigned dst, const CUtensorMap* map, int c0, int c1, unsigned bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar)
-      : "memory");
-}
-
-// Shared-memory matrix descriptor, K-major, 128-byte swizzle: rows of 128 bytes, 8-row atoms
-// 1024 bytes apart (tile base 1024-byte aligned).
-__device__ __forceinline__ uint64_t umma_desc(unsigned smem_addr) {
-  uint64_t d = 0;
-  d |= (uint64_t)((smem_addr >> 4) & 0x3FFFu);   // start address, 16-byte units
-  d |= (uint64_t)1 << 16;                        // leading byte offset (not used by swizzled K-major)
-  d |= (uint64_t)(1024 >> 4) << 32;              // stride byte offset: next 8-row atom
-  d |= (uint64_t)1 << 46;                        // descriptor version of this architecture
-  d |= (uint64_t)2 << 61;                        // layout type: 128-byte swizzle
-  return d;
-}
-
-__device__ __forceinline__ void umma_f16(unsigned tmem_d, uint64_t da, uint64_t db, unsigned idesc, unsigned accumulate) {
-  asm volatile(
-      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
-      " tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
-      ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-__device__ __forceinline__ void umma_commit(unsigned bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-
-__device__ __forceinline__ void tmem_ld32(unsigned taddr, unsigned (&v)[32]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,"
-      "%29,%30,%31}, [%32];\n"
-      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
-        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
-        "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
-        "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-      : "r"(taddr)
-      : "memory");
-}
 
 struct PrefillArgs {
   const uint32_t* codes;
@@ -387,7 +307,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmx, const PrefillArgs p, con
             out[16 * run + 15] = mul_scale<BF16>(sub_magic<BF16>(last | MAGIC, zm), s_hi2, s_lo2);
           }
         }
-        if (round > 0) ok = mbar_wait(empty(s), (round - 1) & 1, abort_flag, lim);
+        if (round > 0) ok = mbar_wait_warp(empty(s), (round - 1) & 1, abort_flag, lim);
         if (!ok) break;
         unsigned char* arow = a_tile(s) + r * 128;
 #pragma unroll
@@ -423,7 +343,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmx, const PrefillArgs p, con
       const int row = (tile % ntn) * kTileN + r, m0 = (tile / ntn) * TOK;
       const bool live = row < p.N;
       const int a = ti & 1;
-      ok = mbar_wait(acc_full(a), (ti >> 1) & 1, abort_flag, lim);
+      ok = mbar_wait_warp(acc_full(a), (ti >> 1) & 1, abort_flag, lim);
       if (!ok) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll 1
@@ -482,22 +402,6 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmx, const PrefillArgs p, con
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(2 * kAccCols) : "memory");
   }
-}
-
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  if (!fn) {
-    void* ptr = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
-        qres == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(ptr);
-  }
-  return fn;
 }
 
 template <int BITS, int TOK>
