@@ -8,17 +8,23 @@
 
 static size_t dtype_bytes(gwq_dtype d) { return d == GWQ_F32 ? 4 : 2; }
 
-// With 17 to 32 tokens the streaming kernel needs four token blocks (one CTA of 8 warps per SM) and copies 8 KB of
-// activations per KB of codes; on tall layers the tensor-core kernel's 32-token tile is faster (measured, 4 bit,
-// M = 32: 44 against 52 us on 11008 x 4096, 161 against 215 us on 28672 x 8192), on layers with few 128-row tiles it
-// is not (84 against 70 us on 8192 x 8192, 287 against 213 us on 8192 x 28672).
+// 17 to 32 tokens that the tcgen05 streaming kernel does not take (bf16 activations, or no workspace): the mma.sync
+// kernel needs four token blocks there (one CTA of 8 warps per SM, 8 KB of activations copied per KB of codes), so
+// the tensor-core kernel's 32-token tile is faster as soon as its 128-row tiles keep at least half of the SMs busy
+// (measured, 4 bit, M = 32: 44 against 52 us on 11008 x 4096 and 161 against 215 us on 28672 x 8192; 84 against 70 us
+// on 8192 x 8192, whose 64 tiles leave most SMs idle).
 static bool prefers_tensor_core(const gwq_packed* P, int M) {
   const gwq_priv* pv = static_cast<const gwq_priv*>(P->priv);
-  return M > 16 && M <= GWQ_DECODE_MAX_M && P->group == 128 && P->N >= 10240 && P->K % 64 == 0 && pv->cv && pv->sz_t;
+  const int sms = pv->sm_count > 0 ? pv->sm_count : 148;
+  return M > 16 && M <= GWQ_DECODE_MAX_M && P->group == 128 && 2 * ((P->N + 127) / 128) >= sms && P->K % 64 == 0 &&
+         pv->cv && pv->sz_t;
 }
 
 #ifndef GWQ_TUNE_SKINNY_MIN_M
-#define GWQ_TUNE_SKINNY_MIN_M 9   // fewest tokens that go to the tcgen05 streaming kernel when a workspace is given
+// fewest tokens that go to the tcgen05 streaming kernel when a workspace is given: its cost per step hardly depends on
+// the token count, the mma.sync kernel's grows with it; measured cross-over between 16 and 17 tokens (4 bit, 16 tokens:
+// 40 against 35 us on 8192 x 8192, 31 against 27 us on 11008 x 4096; 32 tokens: 52 against 70 us, 39 against 44 us)
+#define GWQ_TUNE_SKINNY_MIN_M 17
 #endif
 
 static bool wants_skinny(const gwq_packed* P, gwq_dtype xd, int M) {
@@ -39,7 +45,7 @@ extern "C" gwq_status gwq_linear_ws(const gwq_packed* P, const void* x, gwq_dtyp
   if (yd != GWQ_F16 && yd != GWQ_BF16 && yd != GWQ_F32) return GWQ_ERR_INVALID_ARG;
   if (!gwq_aligned16(x) || !gwq_aligned16(y)) return GWQ_ERR_INVALID_ARG;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-  // with a workspace, 9 to 32 fp16 tokens take the tcgen05 streaming kernel; without one the older kernels serve them
+  // with a workspace, 17 to 32 fp16 tokens take the tcgen05 streaming kernel; without one the other kernels serve them
   if (wants_skinny(P, xd, M) && ws && ws_bytes >= gwq_skinny_workspace_bytes(P, M))
     return gwq_launch_skinny(P, x, M, y, yd, ws, ws_bytes, stream);
   if (M <= GWQ_DECODE_MAX_M && !prefers_tensor_core(P, M)) {
@@ -182,6 +188,8 @@ extern "C" void gwq_free(void* obj) {
       if (pv->y_stage) cudaFree(pv->y_stage);
       if (pv->ws_stage) cudaFree(pv->ws_stage);
       if (pv->xt) cudaFree(pv->xt);
+      if (pv->ob) cudaFree(pv->ob);
+      if (pv->ob_ptr) cudaFree(pv->ob_ptr);
       if (pv->sz_t) cudaFree(pv->sz_t);
       if (pv->dev_status) cudaFree(pv->dev_status);
       delete pv;

@@ -34,6 +34,9 @@ struct gwq_priv {
   size_t ws_stage_bytes;
   void* xt;              // token-major copy [K][32] of the activations and their group sums (decode path with more
   size_t xt_bytes;       // than 8 tokens); created by gwq_pack
+  uint32_t* ob;          // outliers ordered by block of 128 rows x 128 columns: row << 23 | column << 16 | fp16 value
+  int32_t* ob_ptr;       // [blocks + 1] extents of the blocks in ob (block = tile * (K / 128) + column block)
+  void* ob_scratch;      // counters while gwq_pack builds ob
   int32_t* dev_status;   // device status word written by bounded waits
   int sm_count;
   long long wait_cycles; // SM cycles a bounded device-side wait may spin (gwq_set_wait_limit)

@@ -8,8 +8,10 @@
 //                        activation tile (tokens x 128 columns, two 128-byte-swizzled k-blocks) into a stage;
 //   warps 2..9         : two sets of four warps that take alternate steps, one thread per row: the row's codes
 //                        from shared memory -> masked in place into fp16 subnormals q 2^-24 (no arithmetic on the
-//                        codes) -> tensor memory (tcgen05.st), the A operand of the step; the row's FP16
-//                        outliers inside the step are dropped into an otherwise all-zero shared-memory tile;
+//                        codes) -> tensor memory (tcgen05.st), the A operand of the step;
+//   warps 15, 16       : one per set: the FP16 outliers of the step's block (a block-ordered copy of the CSR entries,
+//                        made by gwq_pack) are dropped into an otherwise all-zero shared-memory tile and taken out
+//                        again once the MMAs have read it;
 //   warp 1, one thread : tcgen05.mma kind::f16, M = 128 rows, N = tokens: 8 MMAs (K = 16) with A from tensor
 //                        memory into the step's accumulator, 8 more with the outlier tile as A into an
 //                        accumulator that runs over the whole tile (the tensor cores do the sparse product);
@@ -31,14 +33,15 @@ constexpr int kStages = 4;        // ring of codes + activation tiles
 constexpr int kSets = 2;          // expansion warp sets, one tensor-memory A buffer and one outlier tile each
 constexpr int kXs = 8;            // ring of group-sum slots
 constexpr int kWarpProducer = 0, kWarpMma = 1, kWarpExpand0 = 2, kWarpEpi0 = 2 + 4 * kSets, kWarpSums = kWarpEpi0 + 4;
-constexpr int kThreads = 32 * (kWarpSums + 1);
+constexpr int kWarpOut0 = kWarpSums + 1;
+constexpr int kThreads = 32 * (kWarpOut0 + kSets);
 constexpr int kOutTileBytes = kRows * 128 * 2;   // outlier tile of a step: 128 rows x 128 columns fp16 (two k-blocks)
 constexpr int kTmemCols = 256;
 
 struct SkinnyArgs {
   const uint32_t* szt;      // [K / group][N]: scale fp16 bits | zero-point << 16
-  const int32_t* row_ptr;
-  const uint32_t* cv;       // per outlier: fp16 value << 16 | column
+  const uint32_t* ob;       // outliers by block: row-in-block << 23 | column-in-block << 16 | fp16 value
+  const int32_t* ob_ptr;    // extents of the blocks in ob; block = tile * G + step of the tile = index of the step
   void* y;
   float* partial;           // [2 * gridDim][TOK][128] partial sums of tiles shared with other CTAs
   int32_t* status;
@@ -83,7 +86,7 @@ __device__ __forceinline__ void mma16816_ones(float (&d)[4], unsigned b0, unsign
 // first step of CTA p of P over `total` steps
 __device__ __host__ __forceinline__ long long range_begin(long long total, int P, int p) { return total * p / P; }
 
-// BITS: 3 or 4.  TOK: 16 or 32 tokens (UMMA N).  G64: groups of 64 columns (two accumulators per step).
+// BITS: 3 or 4.  TOK: tokens of a tile (UMMA N; 32 is the one instantiated).  G64: groups of 64 columns (two accumulators per step).
 template <int BITS, int TOK, bool G64>
 __global__ void __launch_bounds__(kThreads, 1)
 skinny_kernel(const __grid_constant__ CUtensorMap tmc, const __grid_constant__ CUtensorMap tmx, const SkinnyArgs p) {
@@ -131,7 +134,7 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmc, const __grid_constant__ C
       mbar_init(empty(s), 6);   // the step's four expansion warps, the MMA commit, the sums warp
     }
     for (int b = 0; b < kSets; ++b) {
-      mbar_init(a_full(b), 4);
+      mbar_init(a_full(b), 5);   // four expansion warps and the set's outlier warp
       mbar_init(a_empty(b), 1);
     }
     for (int d = 0; d < 2; ++d) {
@@ -246,23 +249,8 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmc, const __grid_constant__ C
     const int set = (warp - kWarpExpand0) >> 2;
     const int quad = warp & 3;                 // tensor-memory lane quarter this warp may access
     const int r = quad * 32 + lane;            // row inside the tile
-    unsigned char* otile = out_tiles + set * kOutTileBytes;
-    int jp = 0, je = 0;                        // CSR entries of the current row still ahead
-    int cl0 = 0, cl1 = 0;                      // entries dropped into the tile two steps ago (to be cleared)
-    int cur_tile = -1;
     for (int j = set; j < nsteps && ok; j += kSets) {
-      const long long it = it0 + j;
-      const int tile = (int)(it / G), grp = (int)(it % G);
       const int s = j % kStages;
-      const int row = tile * kRows + r;
-      if (tile != cur_tile) {
-        cur_tile = tile;
-        jp = je = 0;
-        if (row < p.N) {
-          jp = __ldg(p.row_ptr + row);
-          je = __ldg(p.row_ptr + row + 1);
-        }
-      }
       ok = mbar_wait_warp(full(s), (j / kStages) & 1, abort_flag, lim);
       if (!ok) break;
       // the row's packed words of the step
@@ -306,30 +294,7 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmc, const __grid_constant__ C
 #pragma unroll
         for (int c = 0; c < 4; ++c) tmem_st16(ta + (unsigned)(16 * c), a + 16 * c);
       }
-      // outliers: clear what this thread dropped two steps ago, then drop the row's entries of this step
-      for (int e = cl0; e < cl1; ++e) {
-        const unsigned col = __ldg(p.cv + e) & 127u;   // (the tile may have been another one: its row was r as well)
-        *reinterpret_cast<unsigned short*>(otile + (col >> 6) * (kOutTileBytes / 2) + r * 128 +
-                                           ((((col & 63u) >> 3) ^ (unsigned)(r & 7)) << 4) + ((col & 7u) << 1)) = 0;
-      }
-      {
-        const unsigned c_begin = (unsigned)grp * 128u, c_end = c_begin + 128u;
-        while (jp < je && (__ldg(p.cv + jp) & 0xFFFFu) < c_begin) ++jp;   // entries of the steps the other set took
-        cl0 = jp;
-        while (jp < je) {
-          const unsigned e = __ldg(p.cv + jp);
-          const unsigned col = e & 0xFFFFu;
-          if (col >= c_end) break;
-          const unsigned c = col - c_begin;
-          *reinterpret_cast<unsigned short*>(otile + (c >> 6) * (kOutTileBytes / 2) + r * 128 +
-                                             ((((c & 63u) >> 3) ^ (unsigned)(r & 7)) << 4) + ((c & 7u) << 1)) =
-              (unsigned short)(e >> 16);
-          ++jp;
-        }
-        cl1 = jp;
-      }
       asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to the MMA
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncwarp();
       if (lane == 0) {
@@ -346,17 +311,29 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmc, const __grid_constant__ C
     for (int m = 0; m < TOK; ++m) yacc[m] = 0.f;
     int piece = 0;
     bool head = true;   // the current piece contains the first step of this CTA
+    unsigned sz_next[AS];
+    if (nsteps > 0) {
+      const int row0 = (int)(it0 / G) * kRows + r, grp0 = (int)(it0 % G);
+#pragma unroll
+      for (int h = 0; h < AS; ++h) sz_next[h] = __ldg(p.szt + (size_t)(grp0 * AS + h) * p.N + (row0 < p.N ? row0 : p.N - 1));
+    }
     asm volatile("griddepcontrol.wait;" ::: "memory");   // y and the workspace may still be in use by the previous kernel
     for (int j = 0; j < nsteps && ok; ++j) {
       const long long it = it0 + j;
       const int tile = (int)(it / G), grp = (int)(it % G);
       const int row = tile * kRows + r;
-      const int rowc = row < p.N ? row : p.N - 1;
       const bool last = j == nsteps - 1 || grp == G - 1;
       const int xq = j % kXs;
       unsigned sz[AS];
 #pragma unroll
-      for (int h = 0; h < AS; ++h) sz[h] = __ldg(p.szt + (size_t)(grp * AS + h) * p.N + rowc);
+      for (int h = 0; h < AS; ++h) sz[h] = sz_next[h];
+      if (j + 1 < nsteps) {   // scale and zero-point of the next step: requested a step ahead
+        const long long itn = it + 1;
+        const int rown = (int)(itn / G) * kRows + r, grpn = (int)(itn % G);
+#pragma unroll
+        for (int h = 0; h < AS; ++h)
+          sz_next[h] = __ldg(p.szt + (size_t)(grpn * AS + h) * p.N + (rown < p.N ? rown : p.N - 1));
+      }
       ok = mbar_wait_warp(xs_full(xq), (j / kXs) & 1, abort_flag, lim);
       if (!ok) break;
 #pragma unroll
@@ -426,7 +403,7 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmc, const __grid_constant__ C
         head = false;
       }
     }
-  } else {
+  } else if (warp == kWarpSums) {
     // ------------------------------------------------------------------ sums of x over the step's groups, per token
     const int gid = lane >> 2, t = lane & 3;
     for (int j = 0; j < nsteps && ok; ++j) {
@@ -469,6 +446,55 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmc, const __grid_constant__ C
         mbar_arrive(empty(s));
       }
     }
+  } else {
+    // ------------------------------------------------------------------ outliers of the step's block -> the set's tile
+    const int set = warp - kWarpOut0;
+    unsigned char* otile = out_tiles + set * kOutTileBytes;
+    constexpr int kHeld = 8;                   // entries per lane kept in registers (256 per block; the rest is re-read)
+    unsigned held[kHeld];                      // the block's first entries; after the step: what has to be taken out again
+    int e0 = 0, e1 = 0, c0 = 0, c1 = 0;        // entries of this step's block, and of the block this set dropped last
+    // byte offset of entry v inside an outlier tile: two k-blocks, rows of 128 bytes, 128-byte swizzle
+    auto out_off = [&](unsigned v) {
+      const unsigned r = (v >> 23) & 127u, c = (v >> 16) & 127u;
+      return (c >> 6) * (unsigned)(kOutTileBytes / 2) + r * 128u + ((((c & 63u) >> 3) ^ (r & 7u)) << 4) + ((c & 7u) << 1);
+    };
+    auto fetch = [&](int j) {   // extents and first entries of the block of step j (requested a step ahead)
+      if (j < nsteps) {
+        e0 = __ldg(p.ob_ptr + it0 + j);
+        e1 = __ldg(p.ob_ptr + it0 + j + 1);
+#pragma unroll
+        for (int i = 0; i < kHeld; ++i) held[i] = e0 + lane + 32 * i < e1 ? __ldg(p.ob + e0 + lane + 32 * i) : 0xFFFFFFFFu;
+      }
+    };
+    unsigned prev[kHeld];
+#pragma unroll
+    for (int i = 0; i < kHeld; ++i) prev[i] = 0xFFFFFFFFu;
+    fetch(set);
+    for (int j = set; j < nsteps && ok; j += kSets) {
+      if (j >= kSets) ok = mbar_wait_warp(a_empty(set), ((j / kSets) - 1) & 1, abort_flag, lim);   // MMAs of two steps ago done
+      if (!ok) break;
+      // take out what the last step of this set dropped in, then drop in this step's entries
+#pragma unroll
+      for (int i = 0; i < kHeld; ++i)
+        if (prev[i] != 0xFFFFFFFFu) *reinterpret_cast<unsigned short*>(otile + out_off(prev[i])) = 0;
+      for (int e = c0 + lane + 32 * kHeld; e < c1; e += 32)
+        *reinterpret_cast<unsigned short*>(otile + out_off(__ldg(p.ob + e))) = 0;
+#pragma unroll
+      for (int i = 0; i < kHeld; ++i) {
+        prev[i] = held[i];
+        if (held[i] != 0xFFFFFFFFu) *reinterpret_cast<unsigned short*>(otile + out_off(held[i])) = (unsigned short)held[i];
+      }
+      for (int e = e0 + lane + 32 * kHeld; e < e1; e += 32) {
+        const unsigned v = __ldg(p.ob + e);
+        *reinterpret_cast<unsigned short*>(otile + out_off(v)) = (unsigned short)v;
+      }
+      c0 = e0;
+      c1 = e1;
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to the MMA
+      __syncwarp();
+      if (lane == 0) mbar_arrive(a_full(set));
+      fetch(j + kSets);   // behind the proxy fence, which would have waited for these loads
+    }
   }
   if (!ok) {
     *abort_flag = 1;
@@ -499,30 +525,38 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmc, const __grid_constant__ C
   }
 }
 
-// Adds the partial sums of the tiles that several CTAs share, in CTA order, and stores the rows.  One CTA per tile.
+// Adds the partial sums of the tiles that several CTAs share, in CTA order, and stores the rows.  One CTA per tile
+// and block of 8 tokens, one thread per (row, token); the loads of a sum are requested four at a time.
 template <int TOK>
-__global__ void __launch_bounds__(kRows) skinny_fixup_kernel(const float* __restrict__ partial, void* y, gwq_dtype yd, int N,
-                                                            int M, int G, long long total, int P) {
+__global__ void __launch_bounds__(kRows * 8) skinny_fixup_kernel(const float* __restrict__ partial, void* y, gwq_dtype yd,
+                                                                int N, int M, int G, long long total, int P) {
   asm volatile("griddepcontrol.wait;" ::: "memory");
-  const int tile = blockIdx.x, r = threadIdx.x;
+  const int tile = blockIdx.x, r = threadIdx.x, m = blockIdx.y * 8 + threadIdx.y;
   const long long first = (long long)tile * G, last = first + G - 1;
   // owner of a step: the last CTA whose range begins at or before it
   const int p_first = (int)(((first + 1) * P + total - 1) / total) - 1, p_last = (int)(((last + 1) * P + total - 1) / total) - 1;
   if (p_first == p_last) return;   // one CTA had the whole tile and stored it
   const int row = tile * kRows + r;
-  if (row >= N) return;
-  for (int m = 0; m < M; ++m) {
-    float v = 0.f;
-    for (int q = p_first; q <= p_last; ++q) {
-      const long long b = range_begin(total, P, q);
-      const bool is_head = b >= first && b <= last;   // the tile holds the CTA's first step: its first piece
-      v += partial[((size_t)(2 * q + (is_head ? 0 : 1)) * TOK + m) * kRows + r];
+  if (row >= N || m >= M) return;
+  // CTA q's piece of this tile is its first piece (slot 2q) when its range begins inside the tile: every q but
+  // possibly the first one, whose range may have begun in the tile before (then this is its last piece, slot 2q + 1)
+  const int first_slot = 2 * p_first + (range_begin(total, P, p_first) < first ? 1 : 0);
+  float v = 0.f;
+  for (int q0 = p_first; q0 <= p_last; q0 += 4) {
+    float t[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int q = q0 + u;
+      const int slot = q == p_first ? first_slot : 2 * q;
+      t[u] = q <= p_last ? __ldg(partial + ((size_t)slot * TOK + m) * kRows + r) : 0.f;
     }
-    const size_t idx = (size_t)m * N + row;
-    if (yd == GWQ_F32) reinterpret_cast<float*>(y)[idx] = v;
-    else if (yd == GWQ_F16) reinterpret_cast<__half*>(y)[idx] = __float2half_rn(v);
-    else reinterpret_cast<__nv_bfloat16*>(y)[idx] = __float2bfloat16_rn(v);
+#pragma unroll
+    for (int u = 0; u < 4; ++u) v += t[u];   // CTA order: the same bits every time
   }
+  const size_t idx = (size_t)m * N + row;
+  if (yd == GWQ_F32) reinterpret_cast<float*>(y)[idx] = v;
+  else if (yd == GWQ_F16) reinterpret_cast<__half*>(y)[idx] = __float2half_rn(v);
+  else reinterpret_cast<__nv_bfloat16*>(y)[idx] = __float2bfloat16_rn(v);
 }
 
 template <int BITS, int TOK, bool G64>
@@ -552,7 +586,7 @@ gwq_status launch(const gwq_packed* P, const void* x, int M, void* y, gwq_dtype 
   }
   const int tiles = (P->N + kRows - 1) / kRows;
   SkinnyArgs a;
-  a.szt = pv->sz_t; a.row_ptr = P->S->row_ptr; a.cv = pv->cv; a.y = y; a.partial = static_cast<float*>(ws);
+  a.szt = pv->sz_t; a.ob = pv->ob; a.ob_ptr = pv->ob_ptr; a.y = y; a.partial = static_cast<float*>(ws);
   a.status = pv->dev_status; a.yd = yd; a.N = P->N; a.K = P->K; a.M = M; a.G = P->K / 128;
   a.total = (long long)tiles * a.G; a.wait_cycles = pv->wait_cycles;
   const int sms = pv->sm_count > 0 ? pv->sm_count : 148;
@@ -574,8 +608,8 @@ gwq_status launch(const gwq_packed* P, const void* x, int M, void* y, gwq_dtype 
     (void)cudaGetLastError();
     return GWQ_ERR_CUDA;
   }
-  cfg.gridDim = dim3((unsigned)tiles);
-  cfg.blockDim = dim3(kRows);
+  cfg.gridDim = dim3((unsigned)tiles, (unsigned)((M + 7) / 8));
+  cfg.blockDim = dim3(kRows, 8);
   cfg.dynamicSmemBytes = 0;
   if (cudaLaunchKernelEx(&cfg, skinny_fixup_kernel<TOK>, (const float*)a.partial, y, yd, P->N, M, a.G, a.total, grid) != cudaSuccess) {
     (void)cudaGetLastError();
@@ -590,15 +624,15 @@ gwq_status launch(const gwq_packed* P, const void* x, int M, void* y, gwq_dtype 
 bool gwq_skinny_takes(const gwq_packed* P, gwq_dtype xd, int M) {
   const gwq_priv* pv = static_cast<const gwq_priv*>(P->priv);
   return xd == GWQ_F16 && M >= 1 && M <= 32 && (P->group == 64 || P->group == 128) && P->K % 128 == 0 && P->K <= 65536 &&
-         pv->cv && pv->sz_t;
+         pv->ob && pv->ob_ptr && pv->sz_t;
 }
 
 // Workspace: two partial tiles per CTA.
 size_t gwq_skinny_workspace_bytes(const gwq_packed* P, int M) {
   const gwq_priv* pv = static_cast<const gwq_priv*>(P->priv);
   const int sms = pv->sm_count > 0 ? pv->sm_count : 148;
-  const int tok = M <= 16 ? 16 : 32;
-  return (size_t)2 * sms * tok * kRows * sizeof(float);
+  (void)M;
+  return (size_t)2 * sms * 32 * kRows * sizeof(float);   // token tiles of 32
 }
 
 gwq_status gwq_launch_skinny(const gwq_packed* P, const void* x, int M, void* y, gwq_dtype yd, void* ws, size_t ws_bytes,
@@ -606,13 +640,7 @@ gwq_status gwq_launch_skinny(const gwq_packed* P, const void* x, int M, void* y,
   if (!ws || ws_bytes < gwq_skinny_workspace_bytes(P, M) || (reinterpret_cast<uintptr_t>(ws) & 255u) != 0)
     return GWQ_ERR_WORKSPACE;
   const bool g64 = P->group == 64;
-#define GWQ_SK(B, T)                                                              \
-  return g64 ? launch<B, T, true>(P, x, M, y, yd, ws, stream) : launch<B, T, false>(P, x, M, y, yd, ws, stream)
-  if (P->bits == 4) {
-    if (M <= 16) GWQ_SK(4, 16);
-    GWQ_SK(4, 32);
-  }
-  if (M <= 16) GWQ_SK(3, 16);
-  GWQ_SK(3, 32);
-#undef GWQ_SK
+  if (P->bits == 4)
+    return g64 ? launch<4, 32, true>(P, x, M, y, yd, ws, stream) : launch<4, 32, false>(P, x, M, y, yd, ws, stream);
+  return g64 ? launch<3, 32, true>(P, x, M, y, yd, ws, stream) : launch<3, 32, false>(P, x, M, y, yd, ws, stream);
 }

@@ -168,6 +168,54 @@ __global__ void fuse_col_val_kernel(const int32_t* __restrict__ col, const uint1
   if (i < n) cv[i] = ((uint32_t)val[i] << 16) | ((uint32_t)col[i] & 0xFFFFu);
 }
 
+// Block-ordered copy of the outliers for the tcgen05 streaming kernel: the matrix is cut into blocks of 128 rows x
+// 128 columns, numbered tile * (K / 128) + column block; ob_ptr[b] .. ob_ptr[b + 1] are the entries of block b, each
+// packed as row-in-block << 23 | column-in-block << 16 | fp16 value.  Three passes: count, scan, fill (the order of
+// the entries inside a block is whatever the atomics give; every entry has its own position, so it does not matter).
+__global__ void ob_count_kernel(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ col, int N, int G,
+                                unsigned int* __restrict__ cnt) {
+  const int row = blockIdx.x * blockDim.x + threadIdx.x;
+  if (row >= N) return;
+  unsigned int* c = cnt + (size_t)(row >> 7) * G;
+  for (int j = row_ptr[row]; j < row_ptr[row + 1]; ++j) atomicAdd(c + (col[j] >> 7), 1u);
+}
+// exclusive scan of cnt[0..n) into ptr[0..n], one block; cnt is cleared for the fill pass
+__global__ void __launch_bounds__(1024) ob_scan_kernel(unsigned int* __restrict__ cnt, int32_t* __restrict__ ptr, int n) {
+  __shared__ unsigned int part[1024];
+  const int t = threadIdx.x;
+  const int per = (n + 1023) / 1024, lo = min(n, t * per), hi = min(n, lo + per);
+  unsigned int sum = 0;
+  for (int i = lo; i < hi; ++i) sum += cnt[i];
+  part[t] = sum;
+  __syncthreads();
+  for (int off = 1; off < 1024; off <<= 1) {
+    const unsigned int v = t >= off ? part[t - off] : 0u;
+    __syncthreads();
+    part[t] += v;
+    __syncthreads();
+  }
+  unsigned int run = part[t] - sum;
+  for (int i = lo; i < hi; ++i) {
+    ptr[i] = (int32_t)run;
+    run += cnt[i];
+    cnt[i] = 0u;
+  }
+  if (t == 1023) ptr[n] = (int32_t)part[1023];
+}
+__global__ void ob_fill_kernel(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ col,
+                               const uint16_t* __restrict__ val, int N, int G, const int32_t* __restrict__ ptr,
+                               unsigned int* __restrict__ cursor, uint32_t* __restrict__ ob) {
+  const int row = blockIdx.x * blockDim.x + threadIdx.x;
+  if (row >= N) return;
+  const size_t b0 = (size_t)(row >> 7) * G;
+  for (int j = row_ptr[row]; j < row_ptr[row + 1]; ++j) {
+    const int c = col[j];
+    const size_t b = b0 + (c >> 7);
+    const unsigned int pos = atomicAdd(cursor + b, 1u);
+    ob[(size_t)ptr[b] + pos] = ((uint32_t)(row & 127) << 23) | ((uint32_t)(c & 127) << 16) | (uint32_t)val[j];
+  }
+}
+
 // Tensor-core-side copy of the group tables, transposed to [group][row] so that the 128 rows of a
 // tile read 128 neighbouring words.
 __global__ void transpose_scale_zero_kernel(const uint16_t* __restrict__ scales, const uint8_t* __restrict__ zeros,
@@ -237,6 +285,21 @@ extern "C" gwq_status gwq_pack(const uint16_t* W, gwq_outliers* S, int32_t N, in
       GWQ_CUDA_TRY(cudaGetLastError());
     }
   }
+  if (K <= 65536 && group >= 64 && K % 128 == 0) {   // block-ordered outliers of the tcgen05 streaming kernel
+    const long long nnz = S->nnz;
+    const int G = K / 128;
+    const size_t nblocks = (size_t)((N + 127) / 128) * G;
+    unsigned int* cnt = nullptr;
+    GWQ_CUDA_TRY(cudaMalloc(&pv->ob, (size_t)(nnz > 0 ? nnz : 1) * sizeof(uint32_t) + 16));
+    GWQ_CUDA_TRY(cudaMalloc(&pv->ob_ptr, (nblocks + 1) * sizeof(int32_t)));
+    GWQ_CUDA_TRY(cudaMalloc(&cnt, nblocks * sizeof(unsigned int)));
+    pv->ob_scratch = cnt;   // released once the stream has been synchronised below
+    GWQ_CUDA_TRY(cudaMemsetAsync(cnt, 0, nblocks * sizeof(unsigned int), stream));
+    ob_count_kernel<<<(N + 255) / 256, 256, 0, stream>>>(S->row_ptr, S->col_idx, N, G, cnt);
+    ob_scan_kernel<<<1, 1024, 0, stream>>>(cnt, pv->ob_ptr, (int)nblocks);
+    ob_fill_kernel<<<(N + 255) / 256, 256, 0, stream>>>(S->row_ptr, S->col_idx, S->val, N, G, pv->ob_ptr, cnt, pv->ob);
+    GWQ_CUDA_TRY(cudaGetLastError());
+  }
   if (K <= 65536 && group >= 64 && K % 128 == 0) {   // scratch of the streaming path with more than 8 tokens
     GWQ_CUDA_TRY(cudaMalloc(&pv->xt, gwq_decode_scratch_bytes(K)));
     pv->xt_bytes = gwq_decode_scratch_bytes(K);
@@ -249,6 +312,10 @@ extern "C" gwq_status gwq_pack(const uint16_t* W, gwq_outliers* S, int32_t N, in
   }
   GWQ_CUDA_TRY(cudaMemcpyAsync(&host_status, pv->dev_status, sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
   GWQ_CUDA_TRY(cudaStreamSynchronize(stream));
+  if (pv->ob_scratch) {
+    cudaFree(pv->ob_scratch);
+    pv->ob_scratch = nullptr;
+  }
   if (host_status != 0) {
     st = (gwq_status)host_status;
     goto fail;
@@ -264,6 +331,9 @@ fail:
   if (pv->cv) cudaFree(pv->cv);
   if (pv->sz_t) cudaFree(pv->sz_t);
   if (pv->xt) cudaFree(pv->xt);
+  if (pv->ob) cudaFree(pv->ob);
+  if (pv->ob_ptr) cudaFree(pv->ob_ptr);
+  if (pv->ob_scratch) cudaFree(pv->ob_scratch);
   if (pv->dev_status) cudaFree(pv->dev_status);
   delete pv;
   delete P;

@@ -1,4 +1,4 @@
-"""GPU parity of the tcgen05 streaming kernel (fp16 activations, 9 to 32 tokens, reached through gwq_linear_ws)
+"""GPU parity of the tcgen05 streaming kernel (fp16 activations, 17 to 32 tokens, reached through gwq_linear_ws)
 against the CPU checker: every output, |y_gpu - y_ref| <= 1e-3 * sum_k |x_k w_hat_k| + 1e-5.  The layers are chosen
 so that the ranges of steps the CTAs take cut tiles in every way: tiles shared by several CTAs (partial sums added
 by the second kernel), CTAs that own whole tiles plus a head and a tail, a ragged last tile, one step per CTA."""
@@ -39,7 +39,7 @@ LAYERS = [
 
 
 @pytest.mark.parametrize("layer", LAYERS)
-@pytest.mark.parametrize("M", [9, 16, 17, 32])
+@pytest.mark.parametrize("M", [17, 24, 32])
 def test_streaming_tensor_core_kernel(layer, M):
     P, L, w_hat = _layer(*layer)
     bits16, xv = synth.make_activations(M, P.K, seed=200 + M, dtype="f16")
@@ -66,10 +66,10 @@ def test_one_hot_activations_read_back_weight_columns():
 
 def test_without_a_workspace_the_older_kernels_serve_the_call():
     P, L, w_hat = _layer(*LAYERS[0])
-    bits16, xv = synth.make_activations(16, P.K, seed=77, dtype="f16")
+    bits16, xv = synth.make_activations(20, P.K, seed=77, dtype="f16")
     x = x_tensor(bits16, "f16")
-    y = torch.empty((16, P.N), dtype=torch.float32, device=x.device)
-    st = gwq.load_library().gwq_linear(P._h, x.data_ptr(), gwq.GWQ_F16, 16, y.data_ptr(), gwq.GWQ_F32, None)
+    y = torch.empty((20, P.N), dtype=torch.float32, device=x.device)
+    st = gwq.load_library().gwq_linear(P._h, x.data_ptr(), gwq.GWQ_F16, 20, y.data_ptr(), gwq.GWQ_F32, None)
     torch.cuda.synchronize()
     assert st == 0
     y_ref, bound = orc.linear(xv, w_hat)
@@ -80,7 +80,7 @@ def test_give_up_path_of_the_streaming_kernel():
     # spin limit zero: the first wait that is not satisfied at once gives up; the kernel returns, reports it, and
     # the layer works again afterwards
     P, L, w_hat = _layer(*LAYERS[0])
-    bits16, xv = synth.make_activations(16, P.K, seed=78, dtype="f16")
+    bits16, xv = synth.make_activations(20, P.K, seed=78, dtype="f16")
     x = x_tensor(bits16, "f16")
     gwq.gwq_set_wait_limit(P, 0)
     gwq.gwq_linear(P, x, out_dtype=torch.float32)
