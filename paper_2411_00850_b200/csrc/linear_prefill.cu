@@ -131,10 +131,12 @@ __device__ __forceinline__ unsigned sub_magic(unsigned qm, unsigned zm) {
   }
 }
 
-template <int BITS, int TOK, bool BF16>
+// EXP: the weights have been expanded to fp16 [N, K] beforehand (expand_kernel): the producer loads the weight tile
+// by TMA as well and the dequantisation warps have nothing to do.
+template <int BITS, int TOK, bool BF16, bool EXP>
 __global__ void __launch_bounds__(kCtaThreads, 1)
-prefill_kernel(const __grid_constant__ CUtensorMap tmx, const PrefillArgs p, const int stages, const int ntn,
-               const int ntiles) {
+prefill_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUtensorMap tmw, const PrefillArgs p,
+               const int stages, const int ntn, const int ntiles) {
   constexpr int kABytes = kTileN * kBlockK * 2;   // 16 KB
   constexpr int kBBytes = TOK * kBlockK * 2;
   constexpr int kAccCols = TOK < 32 ? 32 : TOK;   // tensor-memory columns of one accumulator
@@ -199,8 +201,9 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmx, const PrefillArgs p, con
           const int it = ti * nkb + kb, s = it % stages, round = it / stages;
           if (round > 0) ok = mbar_wait(empty(s), (round - 1) & 1, abort_flag, lim);
           if (!ok) break;
-          mbar_expect_tx(full_b(s), kBBytes);
+          mbar_expect_tx(full_b(s), EXP ? kBBytes + kABytes : kBBytes);
           tma_load_2d(smem_u32(b_tile(s)), &tmx, kb * kBlockK, m0, full_b(s));
+          if (EXP) tma_load_2d(smem_u32(a_tile(s)), &tmw, kb * kBlockK, (tile % ntn) * kTileN, full_b(s));
           issued = it + 1;
         }
       }
@@ -219,7 +222,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmx, const PrefillArgs p, con
         const unsigned acc = tmem_acc + (unsigned)(a * kAccCols);
         for (int kb = 0; kb < nkb && ok; ++kb) {
           const int it = ti * nkb + kb, s = it % stages, round = it / stages;
-          ok = mbar_wait(full_a(s), round & 1, abort_flag, lim) && mbar_wait(full_b(s), round & 1, abort_flag, lim);
+          ok = (EXP || mbar_wait(full_a(s), round & 1, abort_flag, lim)) && mbar_wait(full_b(s), round & 1, abort_flag, lim);
           if (!ok) break;
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           const uint64_t da = umma_desc(smem_u32(a_tile(s))), db = umma_desc(smem_u32(b_tile(s)));
@@ -239,7 +242,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmx, const PrefillArgs p, con
     constexpr int WPB = kBlockK * BITS / 32;   // packed words per row per k-block (8 or 6)
     constexpr unsigned MAGIC = BF16 ? 0x43004300u : 0x64006400u;   // 128.0 / 1024.0: ulp = 1
     constexpr int kOutWin = 8;                 // outliers of the row kept this many entries ahead
-    for (int ti = 0; ti < my_tiles && ok; ++ti) {
+    for (int ti = 0; ti < (EXP ? 0 : my_tiles) && ok; ++ti) {
       const int tile = blockIdx.x + ti * gridDim.x;
       const int row = (tile % ntn) * kTileN + r;
       const bool live = row < p.N;
@@ -404,27 +407,93 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmx, const PrefillArgs p, con
   }
 }
 
-template <int BITS, int TOK>
-gwq_status launch(const gwq_packed* P, const void* x, const float* tok_scale, int M, void* y, gwq_dtype yd,
+// Two-phase path for many tokens: every token tile of the fused kernel expands the same weights again (M / 256
+// times), so beyond a few tiles the weights are expanded once, to fp16 [N, K] in the caller's workspace (the same
+// values the fused kernel writes into its tiles: exact q - z, one fp16 rounding of the product with the scale, the
+// FP16 outliers over their zero entries), and the contraction streams both operands by TMA.
+template <int BITS>
+__global__ void __launch_bounds__(256) expand_kernel(const uint32_t* __restrict__ codes, const uint32_t* __restrict__ sz_t,
+                                                     uint16_t* __restrict__ w16, int N, int K, int group) {
+  const int runs = K >> 5;                                   // runs of 32 columns per row
+  const long long i = (long long)blockIdx.x * 256 + threadIdx.x;
+  if (i >= (long long)N * runs) return;
+  const int row = (int)(i / runs), run = (int)(i % runs);
+  const uint32_t* src = codes + ((size_t)row * runs + run) * BITS;
+  unsigned w[BITS];
+  if (BITS == 4) {
+    const uint4 v = __ldg(reinterpret_cast<const uint4*>(src));
+    w[0] = v.x; w[1] = v.y; w[2] = v.z; w[BITS - 1] = v.w;
+  } else {
+#pragma unroll
+    for (int k = 0; k < BITS; ++k) w[k] = __ldg(src + k);
+  }
+  const unsigned sz = __ldg(sz_t + (size_t)((run * 32) / group) * N + row);
+  const unsigned s2 = (sz & 0xFFFFu) * 0x00010001u, zm = 0x64006400u | ((sz >> 16) * 0x00010001u);
+  unsigned out[16];
+  if (BITS == 4) {
+#pragma unroll
+    for (int t = 0; t < 4; ++t)
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        out[4 * t + j] = mul_scale<false>(sub_magic<false>(((w[t % BITS] >> (4 * j)) & 0x000F000Fu) | 0x64006400u, zm), s2, 0);
+  } else {
+#pragma unroll
+    for (int k = 0; k < 3; ++k)
+#pragma unroll
+      for (int pp = 0; pp < 5; ++pp)
+        out[5 * k + pp] = mul_scale<false>(sub_magic<false>(((w[k] >> (3 * pp)) & 0x00070007u) | 0x64006400u, zm), s2, 0);
+    const unsigned last = ((w[0] >> 15) & 0x00010001u) | ((w[1] >> 14) & 0x00020002u) | ((w[BITS - 1] >> 13) & 0x00040004u);
+    out[15] = mul_scale<false>(sub_magic<false>(last | 0x64006400u, zm), s2, 0);
+  }
+  uint4* dst = reinterpret_cast<uint4*>(w16 + (size_t)row * K + run * 32);
+#pragma unroll
+  for (int c = 0; c < 4; ++c) dst[c] = make_uint4(out[4 * c], out[4 * c + 1], out[4 * c + 2], out[4 * c + 3]);
+}
+// the FP16 outliers over their (exactly zero) expanded entries; one warp per row
+__global__ void __launch_bounds__(256) expand_outliers_kernel(const int32_t* __restrict__ row_ptr, const uint32_t* __restrict__ cv,
+                                                              uint16_t* __restrict__ w16, int N, int K) {
+  const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (row >= N) return;
+  uint16_t* dst = w16 + (size_t)row * K;
+  for (int j = row_ptr[row] + (threadIdx.x & 31); j < row_ptr[row + 1]; j += 32) {
+    const unsigned e = __ldg(cv + j);
+    dst[e & 0xFFFFu] = (uint16_t)(e >> 16);
+  }
+}
+
+template <int BITS, int TOK, bool EXP>
+gwq_status launch(const gwq_packed* P, const void* x, const float* tok_scale, const void* w16, int M, void* y, gwq_dtype yd,
                   cudaStream_t stream) {
   constexpr bool BF16 = false;   // operands are always fp16 here (see the file header)
   const gwq_priv* pv = static_cast<const gwq_priv*>(P->priv);
   EncodeTiledFn enc = encode_fn();
   if (!enc) return GWQ_ERR_CUDA;
-  CUtensorMap tmx;
-  const cuuint64_t dims[2] = {(cuuint64_t)P->K, (cuuint64_t)M};
-  const cuuint64_t strides[1] = {(cuuint64_t)P->K * 2};
-  const cuuint32_t box[2] = {(cuuint32_t)kBlockK, (cuuint32_t)TOK};
+  CUtensorMap tmx, tmw;
   const cuuint32_t estr[2] = {1, 1};
-  if (enc(&tmx, BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(x),
-          dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-    return GWQ_ERR_CUDA;
+  {
+    const cuuint64_t dims[2] = {(cuuint64_t)P->K, (cuuint64_t)M};
+    const cuuint64_t strides[1] = {(cuuint64_t)P->K * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kBlockK, (cuuint32_t)TOK};
+    if (enc(&tmx, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(x), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return GWQ_ERR_CUDA;
+  }
+  tmw = tmx;
+  if (EXP) {
+    const cuuint64_t dims[2] = {(cuuint64_t)P->K, (cuuint64_t)P->N};
+    const cuuint64_t strides[1] = {(cuuint64_t)P->K * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kBlockK, (cuuint32_t)kTileN};
+    if (enc(&tmw, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(w16), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return GWQ_ERR_CUDA;
+  }
   const int stage_bytes = kTileN * kBlockK * 2 + TOK * kBlockK * 2;
   int stages = (220 * 1024 - 1024) / stage_bytes;
   if (stages > kMaxStages) stages = kMaxStages;
   const size_t smem = (size_t)stages * stage_bytes + 1024;
-  if (cudaFuncSetAttribute(prefill_kernel<BITS, TOK, BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  if (cudaFuncSetAttribute(prefill_kernel<BITS, TOK, BF16, EXP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            (int)smem) != cudaSuccess)
     return GWQ_ERR_CUDA;
   PrefillArgs a;
@@ -433,39 +502,65 @@ gwq_status launch(const gwq_packed* P, const void* x, const float* tok_scale, in
   a.wait_cycles = pv->wait_cycles;
   const int ntn = (P->N + kTileN - 1) / kTileN, ntiles = ntn * ((M + TOK - 1) / TOK);
   const int grid = ntiles < pv->sm_count ? ntiles : pv->sm_count;   // persistent: at most one CTA per SM
-  prefill_kernel<BITS, TOK, BF16><<<grid, kCtaThreads, smem, stream>>>(tmx, a, stages, ntn, ntiles);
+  prefill_kernel<BITS, TOK, BF16, EXP><<<grid, kCtaThreads, smem, stream>>>(tmx, tmw, a, stages, ntn, ntiles);
   return cudaGetLastError() == cudaSuccess ? GWQ_OK : GWQ_ERR_CUDA;
 }
 
 template <int BITS>
 gwq_status launch_tok(const gwq_packed* P, const void* x, const float* tok_scale, int M, void* y, gwq_dtype yd,
                       cudaStream_t stream) {
-  if (M <= 32) return launch<BITS, 32>(P, x, tok_scale, M, y, yd, stream);
-  if (M <= 64) return launch<BITS, 64>(P, x, tok_scale, M, y, yd, stream);
-  if (M <= 128) return launch<BITS, 128>(P, x, tok_scale, M, y, yd, stream);
-  return launch<BITS, 256>(P, x, tok_scale, M, y, yd, stream);
+  if (M <= 32) return launch<BITS, 32, false>(P, x, tok_scale, nullptr, M, y, yd, stream);
+  if (M <= 64) return launch<BITS, 64, false>(P, x, tok_scale, nullptr, M, y, yd, stream);
+  if (M <= 128) return launch<BITS, 128, false>(P, x, tok_scale, nullptr, M, y, yd, stream);
+  return launch<BITS, 256, false>(P, x, tok_scale, nullptr, M, y, yd, stream);
+}
+
+// Tokens from which the weights are expanded once instead of once per token tile.  The expansion costs a pass of
+// 2.5 bytes per weight (about 40 us for 11008 x 4096) and the two-operand contraction is faster per tile than the
+// fused kernel only with 256-token tiles (128-token tiles ask L2 for 114 bytes per clock and SM); measured, bf16
+// activations, 4 bit: 835 against 731 TFLOP/s at 2048 tokens and 1044 against 895 at 8192 on 11008 x 4096, 796
+// against 693 and 1105 against 906 on 4096 x 11008; at 512 and 1024 tokens the fused kernel is level or ahead.
+constexpr int kExpandMinTokens = 2048;
+
+// Expanded weights: the expansion, the outliers over it, then the contraction with token tiles of 256.
+gwq_status launch_expanded(const gwq_packed* P, const void* x, const float* tok_scale, uint16_t* w16, int M, void* y,
+                           gwq_dtype yd, cudaStream_t stream) {
+  const gwq_priv* pv = static_cast<const gwq_priv*>(P->priv);
+  const long long runs = (long long)P->N * (P->K / 32);
+  if (P->bits == 4)
+    expand_kernel<4><<<(unsigned)((runs + 255) / 256), 256, 0, stream>>>(P->codes, pv->sz_t, w16, P->N, P->K, P->group);
+  else
+    expand_kernel<3><<<(unsigned)((runs + 255) / 256), 256, 0, stream>>>(P->codes, pv->sz_t, w16, P->N, P->K, P->group);
+  expand_outliers_kernel<<<(P->N + 7) / 8, 256, 0, stream>>>(P->S->row_ptr, pv->cv, w16, P->N, P->K);
+  if (cudaGetLastError() != cudaSuccess) return GWQ_ERR_CUDA;
+  return launch<4, 256, true>(P, x, tok_scale, w16, M, y, yd, stream);
 }
 
 }  // namespace
 
-// Scratch of the tensor-core path: bf16 activations need an fp16 copy of x and one scale per token.
-size_t gwq_prefill_workspace_bytes(const gwq_packed* P, gwq_dtype xd, int M) {
-  const gwq_priv* pv = static_cast<const gwq_priv*>(P->priv);
-  if (!pv->cv || !pv->sz_t || P->K % kBlockK != 0) return 0;   // the general kernel needs none
+// Scratch of the tensor-core path: bf16 activations need an fp16 copy of x and one scale per token; from
+// kExpandMinTokens tokens on, the fp16 expansion of the weights [N, K] follows.
+static size_t x16_bytes(const gwq_packed* P, gwq_dtype xd, int M) {
   if (xd != GWQ_BF16) return 0;
   return (((size_t)M * P->K * 2 + 255) & ~(size_t)255) + (((size_t)M * 4 + 255) & ~(size_t)255);
 }
+size_t gwq_prefill_workspace_bytes(const gwq_packed* P, gwq_dtype xd, int M) {
+  const gwq_priv* pv = static_cast<const gwq_priv*>(P->priv);
+  if (!pv->cv || !pv->sz_t || P->K % kBlockK != 0) return 0;   // the general kernel needs none
+  return x16_bytes(P, xd, M) + (M >= kExpandMinTokens ? (((size_t)P->N * P->K * 2 + 255) & ~(size_t)255) : 0);
+}
 
 // Prefill launcher: K <= 65536 (16-bit outlier columns).  Other shapes go to the general kernel.
-// bf16 activations are first rewritten into the caller's workspace (fp16 copy of x and the token scales).
+// bf16 activations are first rewritten into the caller's workspace (fp16 copy of x and the token scales); with room
+// for the expanded weights behind them, many tokens take the two-phase path, else the fused kernel.
 gwq_status gwq_launch_prefill(const gwq_packed* P, const void* x, gwq_dtype xd, int M, void* y, gwq_dtype yd,
                               void* ws, size_t ws_bytes, cudaStream_t stream) {
   const gwq_priv* pv = static_cast<const gwq_priv*>(P->priv);
   if (!pv->cv || !pv->sz_t || P->K % kBlockK != 0) return gwq_launch_simt(P, x, xd, M, y, yd, stream);
   const float* tok_scale = nullptr;
+  const size_t xb = x16_bytes(P, xd, M);
+  if ((xb > 0 && (!ws || ws_bytes < xb)) || (ws && (reinterpret_cast<uintptr_t>(ws) & 255u) != 0)) return GWQ_ERR_WORKSPACE;
   if (xd == GWQ_BF16) {
-    const size_t need = gwq_prefill_workspace_bytes(P, xd, M);
-    if (!ws || ws_bytes < need || (reinterpret_cast<uintptr_t>(ws) & 255u) != 0) return GWQ_ERR_WORKSPACE;
     uint16_t* x16 = static_cast<uint16_t*>(ws);
     float* ts = reinterpret_cast<float*>(static_cast<char*>(ws) + (((size_t)M * P->K * 2 + 255) & ~(size_t)255));
     bf16_rows_to_scaled_f16<<<M, 256, 0, stream>>>(static_cast<const uint16_t*>(x), x16, ts, P->K);
@@ -473,6 +568,8 @@ gwq_status gwq_launch_prefill(const gwq_packed* P, const void* x, gwq_dtype xd, 
     x = x16;
     tok_scale = ts;
   }
+  if (M >= kExpandMinTokens && ws && ws_bytes >= gwq_prefill_workspace_bytes(P, xd, M))
+    return launch_expanded(P, x, tok_scale, reinterpret_cast<uint16_t*>(static_cast<char*>(ws) + xb), M, y, yd, stream);
   if (P->bits == 4) return launch_tok<4>(P, x, tok_scale, M, y, yd, stream);
   return launch_tok<3>(P, x, tok_scale, M, y, yd, stream);
 }

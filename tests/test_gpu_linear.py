@@ -92,10 +92,13 @@ def test_tensor_core_path(layer, M, dtype):
 
 
 @pytest.mark.parametrize("bits,dtype", [(4, "f16"), (3, "bf16")])
-def test_persistent_ctas_with_several_tiles_each(bits, dtype):
+@pytest.mark.parametrize("expanded", [False, True])
+def test_persistent_ctas_with_several_tiles_each(bits, dtype, expanded):
     # N = 4096, K = 256, M = 4096: 32 x 16 = 512 tiles of 128 rows x 256 tokens on at most 148 persistent CTAs, so
     # every CTA computes three or four tiles: both accumulators are reused (the wait for the epilogue to drain
-    # them), the stage ring wraps across tiles, and every output is checked
+    # them), the stage ring wraps across tiles, and every output is checked.  Once with the weights expanded
+    # beforehand (workspace with room for them), once through the fused kernel (workspace for the fp16 copy of
+    # bf16 activations only, none for fp16 activations).
     N, K, M = 4096, 256, 4096
     W, G = synth.make_weight_and_grad(N, K, 26)
     L = orc.quantize_layer(W, G, 0.01, bits, 128)
@@ -104,7 +107,17 @@ def test_persistent_ctas_with_several_tiles_each(bits, dtype):
     w_hat = oracle_w_hat(L)
     bits16, xv = synth.make_activations(M, K, seed=126, dtype=dtype, heavy_channels=8)
     y_ref, bound = orc.linear(xv, w_hat)
-    y = gwq.gwq_linear(P, x_tensor(bits16, dtype), out_dtype=torch.float32)
+    x = x_tensor(bits16, dtype)
+    lib = gwq.load_library()
+    xd = gwq.GWQ_F16 if dtype == "f16" else gwq.GWQ_BF16
+    full = int(lib.gwq_linear_workspace_bytes(P._h, xd, M))
+    assert full >= N * K * 2                                     # 4096 tokens: the expansion is asked for
+    ws_bytes = full if expanded else full - N * K * 2            # without room for the weights: the fused kernel
+    ws = torch.empty(max(ws_bytes, 256), dtype=torch.uint8, device=x.device)
+    y = torch.zeros((M, N), dtype=torch.float32, device=x.device)
+    st = lib.gwq_linear_ws(P._h, x.data_ptr(), xd, M, y.data_ptr(), gwq.GWQ_F32, ws.data_ptr() if ws_bytes else None,
+                           ws_bytes, torch.cuda.current_stream().cuda_stream)
+    assert st == 0
     assert gwq.gwq_device_status(P) == 0
     assert_linear_close(y, y_ref, bound)
     P.free()
