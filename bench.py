@@ -79,7 +79,7 @@ def dominant_kernel_traffic():
     import hashlib
     try:
         rec = json.load(open(os.path.join(ROOT, "profiles", "decode_kernel_traffic.json")))
-        src = open(os.path.join(ROOT, "paper_2411_00850_b200", "csrc", "linear_decode.cu"), "rb").read()
+        src = open(os.path.join(ROOT, "paper_2411_00850_b200", "csrc", "decode_kernel.cuh"), "rb").read()
         if hashlib.sha1(src).hexdigest() != rec["kernel_source_sha1"]:
             return None
         return float(rec["dram_bytes_per_launch"]) / float(rec["algorithmic_bytes_per_launch"])
@@ -303,9 +303,11 @@ def run_cuda_arm(args):
     if rank == 0:
         sampler.start()
         time.sleep(0.3)
-    # the timed block of exactly `steps` steps is repeated `repeats` times (each block bracketed by a synchronisation on
-    # both sides); the headline is the median block, the fastest one is reported beside it
-    blocks_ms = [time_region(torch, lambda i: graphs[i % replicas](), args.steps) for _ in range(max(1, args.repeats))]
+    # the timed block of exactly `steps` steps is repeated at least `repeats` times and for at least `min_seconds` (each
+    # block bracketed by a synchronisation on both sides); the headline is the median block, the fastest one is beside it
+    blocks_ms, t_wall = [], time.perf_counter()
+    while len(blocks_ms) < max(1, args.repeats) or (time.perf_counter() - t_wall < args.min_seconds and len(blocks_ms) < 2000):
+        blocks_ms.append(time_region(torch, lambda i: graphs[i % replicas](), args.steps))
     ms_step, ms_step_min = float(np.median(blocks_ms)), float(min(blocks_ms))
     if world > 1:
         ms_step = max_over_ranks(ms_step, dev)
@@ -362,8 +364,9 @@ def run_cuda_arm(args):
         for L in layers:
             L["W"] = None
             L["G"] = None
+        out["config0_single_layer"] = bench_config0(torch, gwq, dev, detail_iters, hbm_peak)
         if not args.skip_70b:
-            out["decode_cases_70b"] = bench_decode_70b(torch, gwq, dev, max(3, detail_iters // 2), hbm_peak)
+            out["llama70b_cases"] = bench_config4(torch, gwq, dev, 3, hbm_peak, tf_burst, args.prefill_iters)
         out["prefill"] = bench_prefill(torch, gwq, dev, args, tf_burst, tf_sust)
         best = max(out["prefill"], key=lambda r: r["tflops"])
         out["prefill_roofline"] = {"bound": "tensor", "kernel": "gwq prefill linear (tcgen05)",
@@ -373,6 +376,21 @@ def run_cuda_arm(args):
                                    "frac_of_sustained": round(best["tflops"] / tf_sust, 4),
                                    "frac_of_nominal_2250": round(best["tflops"] / 2250.0, 4)}
         out["cpu_baseline"] = cpu_baseline(sample_seconds=args.cpu_seconds)
+        # compact copy of every per-case figure inside `roofline` ([N, K, bits, group, outlier %, M, us, fraction of the
+        # measured peak]: HBM for M <= 32, tensor burst for the rest), so that one record carries them all
+        cases = [[r["N"], r["K"], r["bits"], GROUP, 1.0, r["M"], r["us"], r["frac_measured_peak"]] for r in out["decode_cases"]]
+        c0 = out["config0_single_layer"]
+        cases.append([c0["N"], c0["K"], 4, GROUP, 1.0, 1, c0["us"], c0["frac_measured_peak"]])
+        for r in out.get("llama70b_cases", []):
+            cases.append([r["N"], r["K"], r["bits"], r["group"], round(100 * r["frac"], 1), r["M"], r["us"],
+                          r.get("frac_measured_peak", r.get("frac_measured_burst"))])
+        for r in out["prefill"]:
+            cases.append([r["N"], r["K"], 4, GROUP, 1.0, r["M"], r["us"], r["frac_measured_burst"]])
+        out["roofline"]["cases"] = cases
+        out["roofline"]["cases_columns"] = "N, K, bits, group, outlier %, M, us per call, fraction of measured peak (HBM copy rate for M <= 32, bf16 tensor burst above)"
+        out["roofline"]["decode_step_7b"] = [{"M": r["M"], "us": r["us_per_step"], "frac": r["frac_measured_peak"],
+                                               "x_library_fp16": r["speedup_over_library_fp16"]}
+                                              for r in out["decode_step_7b"]["cases"]]
     else:
         out["e2e"] = bench_e2e(torch, gwq, layers, cases, detail_iters, step_bytes, world)
     if world > 1:
@@ -431,10 +449,12 @@ def bench_decode_detail(torch, gwq, layers, xs, ys, iters, hbm_peak):
     return rows
 
 
-def bench_decode_70b(torch, gwq, dev, iters, hbm_peak, Ms=(1, 8, 32)):
-    """Llama-70B-shaped layers (8192 x 8192, 28672 x 8192, 8192 x 28672), 4 and 3 bits, group 128, 1 % outliers:
-    microseconds per launch with a cold L2, as in `bench_decode_detail`.  A layer is 31 to 137 MB of packed data,
-    so the fixed cost of a launch weighs little here and the figure shows what the kernel itself sustains."""
+def bench_config4(torch, gwq, dev, iters, hbm_peak, tf_burst, prefill_iters):
+    """Llama-70B-shaped layers (8192 x 8192, 28672 x 8192, 8192 x 28672) as the configuration states them: 4 and 3
+    bits, groups of 64 and 128, 0.5 / 1 / 2 % outliers, M = 1, 8, 32 (fp16 activations; microseconds per launch with
+    a cold L2, as in `bench_decode_detail`) and M = 2048 (bf16 activations with 8 heavy channels; TFLOP/s, the bf16
+    library product on the unquantised weights beside it).  A layer is 31 to 137 MB of packed data, so the fixed
+    cost of a launch weighs little here and the figures show what the kernels themselves sustain."""
     rows = []
     scrub = torch.zeros(64 * 1024 * 1024, dtype=torch.int32, device=dev)
     for si, (N, K) in enumerate(synth.LLAMA70B_SHAPES):
@@ -442,46 +462,86 @@ def bench_decode_70b(torch, gwq, dev, iters, hbm_peak, Ms=(1, 8, 32)):
         Wd, Gd = torch.from_numpy(W).to(dev), torch.from_numpy(G).to(dev)
         del W, G
         xs = {}
-        for M in Ms:
+        for M in (1, 8, 32):
             bits16, _ = synth.make_activations(M, K, seed=synth.layer_seed(4, si), dtype="f16")
             xs[M] = torch.from_numpy(bits16.view(np.int16).copy()).to(dev).view(torch.float16)
-        for bits in BIT_WIDTHS:
-            copies = 4 if N * K < 100_000_000 else 2     # more than the 126 MB L2 between reuses
-            packed = [gwq.gwq_pack(Wd, gwq.gwq_select_outliers(Wd, Gd, FRAC), bits, GROUP) for _ in range(copies)]
-            nnz = packed[0].nnz
+        bits16, _ = synth.make_activations(2048, K, seed=synth.layer_seed(4, si), dtype="bf16", heavy_channels=8)
+        xp = torch.from_numpy(bits16.view(np.int16).copy()).to(dev).view(torch.bfloat16)
+        Wb = Wd.to(torch.bfloat16)
+        for _ in range(2):
+            torch.matmul(xp, Wb.t())
+        lib_ms = time_region(torch, lambda i: torch.matmul(xp, Wb.t()), max(3, prefill_iters // 2))
+        del Wb
+        copies = 4 if N * K < 100_000_000 else 2     # more than the 126 MB L2 between reuses
+        for frac in (0.005, 0.01, 0.02):
+            S_list = [gwq.gwq_select_outliers(Wd, Gd, frac) for _ in range(copies * 4)]
+            for bits in BIT_WIDTHS:
+                for group in (64, 128):
+                    packed = [gwq.gwq_pack(Wd, S_list.pop(), bits, group) for _ in range(copies)]
+                    nnz = packed[0].nnz
+                    for M in (1, 8, 32):
+                        y = torch.empty((M, N), dtype=torch.float16, device=dev)
+                        need = max(int(gwq.load_library().gwq_linear_workspace_bytes(P._h, gwq.GWQ_F16, M)) for P in packed)
+                        ws = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
 
-            def probe():
-                for P in packed:
-                    gwq.gwq_read_probe(P)
-            replay_probe = capture(torch, probe)
-            floor_ms = None
-            for _ in range(iters):
-                int(scrub.sum().item())
-                ms = time_region(torch, lambda i: replay_probe(), 1)
-                floor_ms = ms if floor_ms is None else min(floor_ms, ms)
-            floor_us = floor_ms * 1e3 / copies
-            for M in Ms:
-                y = torch.empty((M, N), dtype=torch.float16, device=dev)
-
-                def run():
-                    for P in packed:
-                        gwq.gwq_linear(P, xs[M], out=y)
-                replay = capture(torch, run)
-                best = None
-                for _ in range(iters):
-                    int(scrub.sum().item())
-                    ms = time_region(torch, lambda i: replay(), 1)
-                    best = ms if best is None else min(best, ms)
-                us = best * 1e3 / copies
-                b = algorithmic_bytes(N, K, bits, GROUP, nnz, M)
-                rows.append({"N": N, "K": K, "bits": bits, "M": M, "us": round(us, 3), "bytes": b,
-                             "gbs": round(b / us / 1e3, 1), "frac_measured_peak": round(b / us / 1e3 / hbm_peak, 4),
-                             "frac_8TBs": round(b / us / 1e3 / 8000.0, 4), "launches_in_graph": copies,
-                             "read_only_launch_us": round(floor_us, 3), "x_read_only": round(us / floor_us, 2)})
-            del packed
-        del Wd, Gd
+                        def run():
+                            for P in packed:
+                                gwq.gwq_linear(P, xs[M], out=y, workspace=ws if need else None)
+                        replay = capture(torch, run)
+                        best = None
+                        for _ in range(iters):
+                            int(scrub.sum().item())
+                            ms = time_region(torch, lambda i: replay(), 1)
+                            best = ms if best is None else min(best, ms)
+                        us = best * 1e3 / copies
+                        b = algorithmic_bytes(N, K, bits, group, nnz, M)
+                        rows.append({"N": N, "K": K, "bits": bits, "group": group, "frac": frac, "M": M, "us": round(us, 2),
+                                     "gbs": round(b / us / 1e3, 1), "frac_measured_peak": round(b / us / 1e3 / hbm_peak, 4)})
+                    # M = 2048 on the tensor-core path (one packed copy; weights and activations exceed L2 together)
+                    P = packed[0]
+                    yp = torch.empty((2048, N), dtype=torch.bfloat16, device=dev)
+                    need = int(gwq.load_library().gwq_linear_workspace_bytes(P._h, gwq.GWQ_BF16, 2048))
+                    ws = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
+                    for _ in range(2):
+                        gwq.gwq_linear(P, xp, out=yp, workspace=ws)
+                    ms = time_region(torch, lambda i: gwq.gwq_linear(P, xp, out=yp, workspace=ws), max(3, prefill_iters // 2))
+                    tf = linear_flops(N, K, nnz, 2048) / (ms * 1e-3) / 1e12
+                    rows.append({"N": N, "K": K, "bits": bits, "group": group, "frac": frac, "M": 2048, "us": round(ms * 1e3, 1),
+                                 "tflops": round(tf, 1), "frac_measured_burst": round(tf / tf_burst, 4),
+                                 "library_bf16_us": round(lib_ms * 1e3, 1)})
+                    del packed, P, ws, yp
+            del S_list
+        del Wd, Gd, xp
+        torch.cuda.empty_cache()
     del scrub
     return rows
+
+
+def bench_config0(torch, gwq, dev, iters, hbm_peak):
+    """The single-layer configuration as written: 4096 x 4096, seed 0, 4 bits, groups of 128, 1 % outliers, fp16
+    activations, one token.  32 packed copies (300 MB) are cycled through in one CUDA graph, cold L2."""
+    N = K = 4096
+    W, G = synth.make_weight_and_grad(N, K, synth.layer_seed(0, 0))
+    Wd, Gd = torch.from_numpy(W).to(dev), torch.from_numpy(G).to(dev)
+    packed = [gwq.gwq_pack(Wd, gwq.gwq_select_outliers(Wd, Gd, FRAC), 4, GROUP) for _ in range(32)]
+    bits16, _ = synth.make_activations(1, K, seed=synth.layer_seed(0, 0), dtype="f16")
+    x = torch.from_numpy(bits16.view(np.int16).copy()).to(dev).view(torch.float16)
+    y = torch.empty((1, N), dtype=torch.float16, device=dev)
+
+    def run():
+        for P in packed:
+            gwq.gwq_linear(P, x, out=y)
+    replay = capture(torch, run)
+    scrub = torch.zeros(64 * 1024 * 1024, dtype=torch.int32, device=dev)
+    times = []
+    for _ in range(iters):
+        int(scrub.sum().item())
+        times.append(time_region(torch, lambda i: replay(), 1) * 1e3 / len(packed))
+    b = algorithmic_bytes(N, K, 4, GROUP, packed[0].nnz, 1)
+    us = min(times)
+    return {"N": N, "K": K, "bits": 4, "group": GROUP, "frac": FRAC, "M": 1, "seed": 0, "nnz": packed[0].nnz,
+            "us": round(us, 3), "us_median": round(float(np.median(times)), 3), "bytes": b, "gbs": round(b / us / 1e3, 1),
+            "frac_measured_peak": round(b / us / 1e3 / hbm_peak, 4), "launches_in_graph": len(packed)}
 
 
 def bench_dense_library(torch, layers, xs, iters, step_bytes, ms_step):
@@ -617,9 +677,11 @@ def bench_prefill(torch, gwq, dev, args, tf_burst, tf_sust):
             bits16, _ = synth.make_activations(M, K, seed=synth.layer_seed(2, si), dtype="bf16", heavy_channels=8)
             x = torch.from_numpy(bits16.view(np.int16).copy()).to(dev).view(torch.bfloat16)
             y = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
+            need = int(gwq.load_library().gwq_linear_workspace_bytes(P._h, gwq.GWQ_BF16, M))
+            ws = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)   # scratch of the call (caller-supplied)
             for _ in range(2):
-                gwq.gwq_linear(P, x, out=y)
-            ms = time_region(torch, lambda i: gwq.gwq_linear(P, x, out=y), args.prefill_iters)
+                gwq.gwq_linear(P, x, out=y, workspace=ws)
+            ms = time_region(torch, lambda i: gwq.gwq_linear(P, x, out=y, workspace=ws), args.prefill_iters)
             for _ in range(2):
                 torch.matmul(x, Wb.t())
             ms_lib = time_region(torch, lambda i: torch.matmul(x, Wb.t()), args.prefill_iters)
@@ -628,8 +690,9 @@ def bench_prefill(torch, gwq, dev, args, tf_burst, tf_sust):
             rows.append({"N": N, "K": K, "M": M, "us": round(ms * 1e3, 2), "tflops": round(tf, 2),
                          "frac_measured_burst": round(tf / tf_burst, 4), "frac_measured_sustained": round(tf / tf_sust, 4),
                          "frac_nominal_2250": round(tf / 2250.0, 4), "library_bf16_us": round(ms_lib * 1e3, 2),
-                         "library_bf16_tflops": round(2 * M * N * K / (ms_lib * 1e-3) / 1e12, 2)})
-            del x, y
+                         "library_bf16_tflops": round(2 * M * N * K / (ms_lib * 1e-3) / 1e12, 2),
+                         "workspace_bytes": need})
+            del x, y, ws
         P.free()
         del Wd, Wb
     return rows
@@ -755,7 +818,8 @@ def run_reference_arm(args):
     return {"impl": "reference", "metric": METRIC, "value": round(value, 4), "unit": "GB/s",
             "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": round(ms, 2), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "f64", "data": "synthetic", "config": {"workload": WORKLOAD, "sampled": vals[-1]["sample"]},
+            "dtype": "f64", "data": "synthetic",
+            "config": {"workload": WORKLOAD + " (sampled: q_proj 4096x4096 only)", "sampled": vals[-1]["sample"]},
             "cpu_baseline": {"value": round(value, 4), "unit": "GB/s", "cores": vals[-1]["cores"], "kind": "oracle",
                              "sample": vals[-1]["sample"]},
             "e2e": {"value": round(value, 4), "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -768,7 +832,9 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=("ours", "reference"))
-    ap.add_argument("--repeats", type=int, default=10, help="timed blocks of `steps` steps (median reported)")
+    ap.add_argument("--repeats", type=int, default=10, help="timed blocks of `steps` steps, at least (median reported)")
+    ap.add_argument("--min-seconds", type=float, default=2.0,
+                    help="keep timing blocks until this much time has passed, so that the clock sampler sees the load")
     ap.add_argument("--prefill-iters", type=int, default=20)
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--headline-only", action="store_true", help="skip the per-case detail sections")
