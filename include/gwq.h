@@ -115,6 +115,14 @@ gwq_status gwq_select_outliers_static(const uint16_t* W_f16, const float* G_f32,
                                       double frac, int32_t* row_ptr, int32_t* col_idx, uint16_t* val,
                                       int64_t capacity, int64_t* nnz_host, void* stream);
 
+/* Rows [row0, row1) of an outlier matrix as an object of its own (N = row1 - row0, same K, columns and values
+ * copied, row pointers re-based).  The outlier location of Eq. "o" ranks the whole matrix, so a layer whose
+ * rows are split over several GPUs is selected as a whole and then cut: every rank packs and multiplies its own
+ * rows, and one all-gather of y puts the product together (the paper runs on one GPU and has no counterpart).
+ *   *out: new library-owned object; S is unchanged.  Synchronises `stream`.
+ * Errors: INVALID_ARG (bad object, row range outside [0, N] or empty), ALLOC, CUDA.  On error *out is NULL. */
+gwq_status gwq_outliers_rows(const gwq_outliers* S, int32_t row0, int32_t row1, gwq_outliers** out, void* stream);
+
 /* Group-wise asymmetric quantization of the non-outliers (Section 3.2, Eqs. "s", "z",
  * "q") and bit-packing.  Per (row, group of `group` consecutive k), over non-outlier
  * entries only: lo = min(0, min w), hi = max(0, max w); s = (hi - lo) / (2^bits - 1)

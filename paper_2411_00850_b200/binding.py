@@ -23,7 +23,7 @@ STATUS_NAMES = {
     0: "GWQ_OK", 1: "GWQ_ERR_INVALID_ARG", 2: "GWQ_ERR_UNSUPPORTED", 3: "GWQ_ERR_ALLOC",
     4: "GWQ_ERR_NONFINITE", 5: "GWQ_ERR_TIMEOUT", 6: "GWQ_ERR_CUDA", 7: "GWQ_ERR_WORKSPACE",
 }
-EXPORTS = ("gwq_select_outliers", "gwq_select_outliers_static", "gwq_pack", "gwq_linear", "gwq_linear_ws",
+EXPORTS = ("gwq_select_outliers", "gwq_select_outliers_static", "gwq_outliers_rows", "gwq_pack", "gwq_linear", "gwq_linear_ws",
            "gwq_linear_workspace_bytes", "gwq_linear_multi",
            "gwq_gradient_mean", "gwq_quality", "gwq_read_probe", "gwq_linear_host", "gwq_linear_host_async", "gwq_device_status", "gwq_set_wait_limit", "gwq_free", "gwq_status_string")
 GWQ_MULTI_MAX = 4
@@ -65,6 +65,9 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     lib.gwq_select_outliers_static.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_double,
                                                C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64,
                                                C.POINTER(C.c_int64), C.c_void_p]
+    lib.gwq_outliers_rows.restype = C.c_int
+    lib.gwq_outliers_rows.argtypes = [C.POINTER(gwq_outliers), C.c_int32, C.c_int32, C.POINTER(C.POINTER(gwq_outliers)),
+                                      C.c_void_p]
     lib.gwq_pack.restype = C.c_int
     lib.gwq_pack.argtypes = [C.c_void_p, C.POINTER(gwq_outliers), C.c_int32, C.c_int32, C.c_int32, C.c_int32,
                              C.POINTER(C.POINTER(gwq_packed)), C.c_void_p]
@@ -279,6 +282,15 @@ def gwq_select_outliers_static(W: torch.Tensor, G: torch.Tensor, frac: float, ro
                                             col_idx.data_ptr(), val.data_ptr(), cap, C.byref(nnz), _stream_ptr())
     _check(st, "gwq_select_outliers_static")
     return int(nnz.value)
+
+
+def gwq_outliers_rows(S: Outliers, row0: int, row1: int) -> Outliers:
+    """Rows [row0, row1) of S as an outlier matrix of its own (for a layer whose rows are split over ranks)."""
+    out = C.POINTER(gwq_outliers)()
+    with torch.cuda.device(S.device):
+        st = load_library().gwq_outliers_rows(S._h, int(row0), int(row1), C.byref(out), _stream_ptr())
+    _check(st, "gwq_outliers_rows")
+    return Outliers(out, S.device)
 
 
 def gwq_pack(W: torch.Tensor, S: Outliers, bits: int, group: int) -> Packed:

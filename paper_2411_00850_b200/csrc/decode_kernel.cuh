@@ -60,6 +60,7 @@ struct Variant {
   int tp;      // tokens rounded up to 1, 4, 8, 16 or 32
   int nbuf;    // 0: all of x staged up front; 2, 3: per-warp ring of that many tiles
   int rt;      // m16 tiles per CTA (rows = 16 rt)
+  int deep;    // 1: eight groups of codes in flight per warp instead of four (one tile, up to 8 tokens; two CTAs per SM)
   bool g64;    // groups of 64 columns
 };
 
@@ -338,7 +339,14 @@ template <int NB> struct StepAcc<3, NB, false> { using type = AccRaw3<NB>; };
 template <int BITS, int NB> struct StepAcc<BITS, NB, true> { using type = AccSub<NB>; };
 
 // resident CTAs the register budget is cut for
-__host__ __device__ constexpr int min_blocks(int nb, int rt) { return rt == 1 ? (nb == 1 ? 3 : (nb == 2 ? 2 : 1)) : (nb == 1 ? 2 : 1); }
+__host__ __device__ constexpr int min_blocks(int nb, int rt, bool deep) {
+  return deep ? 2 : (rt == 1 ? (nb == 1 ? 3 : (nb == 2 ? 2 : 1)) : (nb == 1 ? 2 : 1));
+}
+
+template <class F, int... I>
+__device__ __forceinline__ void unroll_slots(F&& f, std::integer_sequence<int, I...>) {
+  (f(std::integral_constant<int, I>{}), ...);
+}
 
 // TP = tokens rounded up to 1, 4, 8, 16 or 32.
 // NBUF = 0: the activations of all chunks are staged up front by the whole CTA (small M K).
@@ -353,11 +361,13 @@ __host__ __device__ constexpr int min_blocks(int nb, int rt) { return rt == 1 ? 
 // of x come from the all-ones MMA (which sees the same zeros); a single token's are reduced over half a warp each.
 // TP <= 16 there.
 // RT: m16 tiles (16 rows each) of the CTA; every warp step loads the B fragments once and runs all RT tiles on them.
-template <int BITS, int TP, bool BF16, int NBUF, bool G64, int RT>
-__global__ void __launch_bounds__(kThreads, min_blocks(token_blocks(TP, G64), RT))
+// DEEP: eight groups of codes in flight per warp (grids that leave an SM at most two CTAs: fewer warps have to keep
+// as many bytes in flight).
+template <int BITS, int TP, bool BF16, int NBUF, bool G64, int RT, bool DEEP>
+__global__ void __launch_bounds__(kThreads, min_blocks(token_blocks(TP, G64), RT, DEEP))
 decode_kernel(const MultiArgs ma) {
   constexpr int R = 16 * RT;                       // rows of the CTA
-  constexpr int D = RT == 1 ? 4 : 2;               // groups of codes in flight per warp and tile
+  constexpr int D = DEEP ? 8 : (RT == 1 ? 4 : 2);  // groups of codes in flight per warp and tile
   constexpr int NB = token_blocks(TP, G64);        // token blocks of the MMA (8 tokens; 4 with groups of 64)
   constexpr int WPR = BITS;                        // words per run of 32 columns
   // raw path: sum_k x_k of a group from shared memory (one token), from the table that comes with the
@@ -733,16 +743,9 @@ decode_kernel(const MultiArgs ma) {
     }
     tp += (G64 ? 2 * kWarps : kWarps) * R;
   };
-  using std::integral_constant;
-  static_assert(D == 2 || D == 4, "the step loop is written out for two or four register slots");
-  for (int c0 = 0; c0 < nsteps; c0 += D) {
-    do_step(c0, integral_constant<int, 0>{});
-    if (c0 + 1 < nsteps) do_step(c0 + 1, integral_constant<int, 1>{});
-    if (D == 4) {
-      if (c0 + 2 < nsteps) do_step(c0 + 2, integral_constant<int, 2 % D>{});
-      if (c0 + 3 < nsteps) do_step(c0 + 3, integral_constant<int, 3 % D>{});
-    }
-  }
+  for (int c0 = 0; c0 < nsteps; c0 += D)   // the register slot of a step is a compile-time constant
+    unroll_slots([&](auto slot) { if (c0 + decltype(slot)::value < nsteps) do_step(c0 + decltype(slot)::value, slot); },
+                 std::make_integer_sequence<int, D>{});
 
   // partial sums of the 8 warps: sm_red[warp][tile][nb][row][token]
 #pragma unroll
@@ -774,11 +777,11 @@ decode_kernel(const MultiArgs ma) {
   }
 }
 
-template <int BITS, int TP, bool BF16, int NBUF, bool G64, int RT>
+template <int BITS, int TP, bool BF16, int NBUF, bool G64, int RT, bool DEEP = false>
 cudaError_t launch(const Variant& v, const MultiArgs& a, cudaStream_t stream) {
   const size_t smem = smem_bytes(v, a.K, a.M, a.cvcap);
   if (smem > 48 * 1024) {
-    cudaError_t e = cudaFuncSetAttribute(decode_kernel<BITS, TP, BF16, NBUF, G64, RT>,
+    cudaError_t e = cudaFuncSetAttribute(decode_kernel<BITS, TP, BF16, NBUF, G64, RT, DEEP>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
   }
@@ -792,7 +795,7 @@ cudaError_t launch(const Variant& v, const MultiArgs& a, cudaStream_t stream) {
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, decode_kernel<BITS, TP, BF16, NBUF, G64, RT>, a);
+  return cudaLaunchKernelEx(&cfg, decode_kernel<BITS, TP, BF16, NBUF, G64, RT, DEEP>, a);
 }
 
 // the variants that exist: x staged up front for up to 8 tokens, rings of two tiles up to 8 tokens and of three beyond
@@ -805,6 +808,9 @@ cudaError_t launch_tp(const Variant& v, const MultiArgs& a, cudaStream_t stream)
         if constexpr (!G64) return launch<BITS, TP, BF16, 0, G64, 2>(v, a, stream);
         return cudaErrorInvalidValue;
       }
+      if constexpr (!G64) {
+        if (v.deep) return launch<BITS, TP, BF16, 0, G64, 1, true>(v, a, stream);
+      }
       return launch<BITS, TP, BF16, 0, G64, 1>(v, a, stream);
     }
     return cudaErrorInvalidValue;
@@ -814,6 +820,9 @@ cudaError_t launch_tp(const Variant& v, const MultiArgs& a, cudaStream_t stream)
       if (v.nbuf == 2) return launch<BITS, TP, BF16, 2, G64, 2>(v, a, stream);
     }
     return cudaErrorInvalidValue;
+  }
+  if constexpr (!G64 && TP <= 8) {
+    if (v.deep && v.nbuf == 2) return launch<BITS, TP, BF16, 2, G64, 1, true>(v, a, stream);
   }
   if (v.nbuf == 2) return launch<BITS, TP, BF16, 2, G64, 1>(v, a, stream);
   if constexpr (TP >= 16) return launch<BITS, TP, BF16, 3, G64, 1>(v, a, stream);

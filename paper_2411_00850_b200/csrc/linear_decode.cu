@@ -109,6 +109,12 @@ bool plan(const gwq_packed* const* P, int count, int M, Variant* v, int* cvcap) 
   if (GWQ_TUNE_RT == 1 || (GWQ_TUNE_RT == 2 && !g64 && v->tp <= 8)) v->rt = GWQ_TUNE_RT;
   long long blocks = 0;
   for (int i = 0; i < count; ++i) blocks += (P[i]->N + 16 * v->rt - 1) / (16 * v->rt);
+  // a grid that leaves an SM two CTAs at most anyway: twice the codes in flight per warp (more registers, which then
+  // cost no occupancy)
+  v->deep = (v->rt == 1 && !g64 && v->tp <= 8 && blocks <= 2LL * sms) ? 1 : 0;
+#ifdef GWQ_TUNE_DEEP
+  v->deep = (v->rt == 1 && !g64 && v->tp <= 8) ? GWQ_TUNE_DEEP : 0;
+#endif
   const int nchunks = (K / 128 + kChunkGroups - 1) / kChunkGroups;
   const size_t lim = v->rt == 2 ? kStageAllLimitTwoTiles : (blocks <= 2LL * sms ? kStageAllLimitSmallGrid : kStageAllLimit);
   // outlier entries per row kept in shared memory: one and a half times the average row, in steps of 32

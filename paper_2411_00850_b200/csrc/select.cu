@@ -336,3 +336,51 @@ fail:
   delete S;
   return st;
 }
+
+
+namespace {
+__global__ void rebase_row_ptr_kernel(const int32_t* __restrict__ src, int32_t* __restrict__ dst, int n, int32_t base) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) dst[i] = src[i] - base;
+}
+}  // namespace
+
+extern "C" gwq_status gwq_outliers_rows(const gwq_outliers* S, int32_t row0, int32_t row1, gwq_outliers** out,
+                                        void* stream_) {
+  if (out) *out = nullptr;
+  if (!S || !out || S->tag != GWQ_TAG_OUTLIERS || row0 < 0 || row1 > S->N || row0 >= row1) return GWQ_ERR_INVALID_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  gwq_status st = GWQ_OK;
+  int32_t ends[2] = {0, 0};
+  gwq_outliers* R = new (std::nothrow) gwq_outliers();
+  if (!R) return GWQ_ERR_ALLOC;
+  R->tag = GWQ_TAG_OUTLIERS;
+  R->N = row1 - row0;
+  R->K = S->K;
+  R->nnz = 0;
+  R->row_ptr = nullptr;
+  R->col_idx = nullptr;
+  R->val = nullptr;
+  GWQ_CUDA_TRY(cudaMemcpyAsync(&ends[0], S->row_ptr + row0, sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
+  GWQ_CUDA_TRY(cudaMemcpyAsync(&ends[1], S->row_ptr + row1, sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
+  GWQ_CUDA_TRY(cudaStreamSynchronize(stream));
+  R->nnz = ends[1] - ends[0];
+  GWQ_CUDA_TRY(cudaMalloc(&R->row_ptr, ((size_t)R->N + 1) * sizeof(int32_t)));
+  GWQ_CUDA_TRY(cudaMalloc(&R->col_idx, (size_t)(R->nnz > 0 ? R->nnz : 1) * sizeof(int32_t)));
+  GWQ_CUDA_TRY(cudaMalloc(&R->val, (size_t)(R->nnz > 0 ? R->nnz : 1) * sizeof(uint16_t) + 16));
+  rebase_row_ptr_kernel<<<(R->N + 1 + 255) / 256, 256, 0, stream>>>(S->row_ptr + row0, R->row_ptr, R->N + 1, ends[0]);
+  GWQ_CUDA_TRY(cudaGetLastError());
+  if (R->nnz > 0) {
+    GWQ_CUDA_TRY(cudaMemcpyAsync(R->col_idx, S->col_idx + ends[0], (size_t)R->nnz * sizeof(int32_t), cudaMemcpyDeviceToDevice, stream));
+    GWQ_CUDA_TRY(cudaMemcpyAsync(R->val, S->val + ends[0], (size_t)R->nnz * sizeof(uint16_t), cudaMemcpyDeviceToDevice, stream));
+  }
+  GWQ_CUDA_TRY(cudaStreamSynchronize(stream));
+  *out = R;
+  return GWQ_OK;
+fail:
+  if (R->row_ptr) cudaFree(R->row_ptr);
+  if (R->col_idx) cudaFree(R->col_idx);
+  if (R->val) cudaFree(R->val);
+  delete R;
+  return st;
+}
