@@ -117,3 +117,26 @@ def test_nonfinite_weight_is_an_error_and_bad_arguments():
         assert e.value.status == want
     S.free()
     torch.cuda.synchronize()
+
+
+def test_rows_of_an_outlier_matrix_pack_like_the_rows_of_the_whole():
+    # the selection ranks the whole matrix; a rank that owns rows [128, 300) cuts them out and packs them alone
+    N, K, r0, r1 = 300, 512, 128, 300
+    W, G = synth.make_weight_and_grad(N, K, 55)
+    L = orc.quantize_layer(W, G, 0.02, 3, 64)
+    Wd, Gd = torch.from_numpy(W).to("cuda:0"), torch.from_numpy(G).to("cuda:0")
+    S = gwq.gwq_select_outliers(Wd, Gd, 0.02)
+    S_loc = gwq.gwq_outliers_rows(S, r0, r1)
+    rp, ci, va = (t.cpu().numpy() for t in S_loc.arrays())
+    lo, hi = int(L["row_ptr"][r0]), int(L["row_ptr"][r1])
+    assert np.array_equal(rp, L["row_ptr"][r0:r1 + 1] - lo)
+    assert np.array_equal(ci, L["col_idx"][lo:hi]) and np.array_equal(va.view(np.uint16), L["val"][lo:hi])
+    P = gwq.gwq_pack(Wd[r0:r1].contiguous(), S_loc, 3, 64)
+    a = {k: v.cpu().numpy() for k, v in P.arrays().items()}
+    assert np.array_equal(a["words"].view(np.uint32), L["words"][r0:r1])
+    assert np.array_equal(a["scales"].view(np.uint16), L["scales"].view(np.uint16)[r0:r1])
+    assert np.array_equal(a["zeros"], L["zeros"][r0:r1])
+    with pytest.raises(gwq.GwqError):
+        gwq.gwq_outliers_rows(S, 10, 10)
+    P.free()
+    S.free()
