@@ -133,7 +133,8 @@ __device__ __forceinline__ unsigned sub_magic(unsigned qm, unsigned zm) {
 
 // EXP: the weights have been expanded to fp16 [N, K] beforehand (expand_kernel): the producer loads the weight tile
 // by TMA as well and the dequantisation warps have nothing to do.
-template <int BITS, int TOK, bool BF16, bool EXP>
+// GPK: scale groups per 64-column k-block: 1 (groups of 64 and 128), 2 (groups of 32), 4 (groups of 16).
+template <int BITS, int TOK, bool BF16, bool EXP, int GPK>
 __global__ void __launch_bounds__(kCtaThreads, 1)
 prefill_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUtensorMap tmw, const PrefillArgs p,
                const int stages, const int ntn, const int ntiles) {
@@ -260,31 +261,38 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
       // first k-block of this tile that belongs to the group
       int kb = ((gq - ti * nkb) % G + G) % G;
       unsigned wq[WPB];
-      unsigned sz_nx = 0;   // scale (fp16 bits) | zero-point << 16 of the group of the next k-block
+      unsigned sz_nx[GPK];   // scale (fp16 bits) | zero-point << 16 of the groups of the next k-block
+#pragma unroll
+      for (int g = 0; g < GPK; ++g) sz_nx[g] = 0;
       if (kb < nkb) {
         load_words<WPB>(crow + (size_t)kb * WPB, wq);
-        sz_nx = __ldg(szcol + (size_t)((kb * kBlockK) / p.group) * p.N);
+#pragma unroll
+        for (int g = 0; g < GPK; ++g) sz_nx[g] = __ldg(szcol + (size_t)((kb * kBlockK) / p.group + g) * p.N);
       }
       for (; kb < nkb && ok; kb += G) {
         const int it = ti * nkb + kb, s = it % stages, round = it / stages;
-        const float sc = live ? __half2float(__ushort_as_half((unsigned short)(sz_nx & 0xFFFFu))) : 0.f;
-        const unsigned z = sz_nx >> 16;
-        unsigned s_hi2, s_lo2 = 0;
-        if (BF16) {
-          const __nv_bfloat16 hi = __float2bfloat16_rn(sc);
-          const __nv_bfloat16 lo = __float2bfloat16_rn(sc - __bfloat162float(hi));
-          s_hi2 = (unsigned)__bfloat16_as_ushort(hi) * 0x00010001u;
-          s_lo2 = (unsigned)__bfloat16_as_ushort(lo) * 0x00010001u;
-        } else {
-          s_hi2 = (unsigned)__half_as_ushort(__float2half_rn(sc)) * 0x00010001u;
+        unsigned s_hi2[GPK], s_lo2[GPK], zm[GPK];   // per group of the k-block; pair h belongs to group h GPK / 32
+#pragma unroll
+        for (int g = 0; g < GPK; ++g) {
+          const float sc = live ? __half2float(__ushort_as_half((unsigned short)(sz_nx[g] & 0xFFFFu))) : 0.f;
+          s_lo2[g] = 0;
+          if (BF16) {
+            const __nv_bfloat16 hi = __float2bfloat16_rn(sc);
+            const __nv_bfloat16 lo = __float2bfloat16_rn(sc - __bfloat162float(hi));
+            s_hi2[g] = (unsigned)__bfloat16_as_ushort(hi) * 0x00010001u;
+            s_lo2[g] = (unsigned)__bfloat16_as_ushort(lo) * 0x00010001u;
+          } else {
+            s_hi2[g] = (unsigned)__half_as_ushort(__float2half_rn(sc)) * 0x00010001u;
+          }
+          zm[g] = MAGIC | ((sz_nx[g] >> 16) * 0x00010001u);
         }
-        const unsigned zm = MAGIC | (z * 0x00010001u);
         unsigned cur[WPB];
 #pragma unroll
         for (int i = 0; i < WPB; ++i) cur[i] = wq[i];
         if (kb + G < nkb) {   // codes, scale and zero-point of this group's next k-block
           load_words<WPB>(crow + (size_t)(kb + G) * WPB, wq);
-          sz_nx = __ldg(szcol + (size_t)(((kb + G) * kBlockK) / p.group) * p.N);
+#pragma unroll
+          for (int g = 0; g < GPK; ++g) sz_nx[g] = __ldg(szcol + (size_t)(((kb + G) * kBlockK) / p.group + g) * p.N);
         }
         // 64 codes -> 32 pairs (columns 2h, 2h+1) -> 8 chunks of 16 bytes
         unsigned out[32];
@@ -294,7 +302,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
 #pragma unroll
             for (int q4 = 0; q4 < 4; ++q4)
               out[4 * i + q4] = mul_scale<BF16>(
-                  sub_magic<BF16>(((cur[i % WPB] >> (4 * q4)) & 0x000F000Fu) | MAGIC, zm), s_hi2, s_lo2);
+                  sub_magic<BF16>(((cur[i % WPB] >> (4 * q4)) & 0x000F000Fu) | MAGIC, zm[(4 * i + q4) * GPK / 32]),
+                  s_hi2[(4 * i + q4) * GPK / 32], s_lo2[(4 * i + q4) * GPK / 32]);
         } else {
 #pragma unroll
           for (int run = 0; run < 2; ++run) {
@@ -304,10 +313,13 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
 #pragma unroll
               for (int pp = 0; pp < 5; ++pp)
                 out[16 * run + 5 * i + pp] =
-                    mul_scale<BF16>(sub_magic<BF16>(((w3[i] >> (3 * pp)) & 0x00070007u) | MAGIC, zm), s_hi2, s_lo2);
+                    mul_scale<BF16>(sub_magic<BF16>(((w3[i] >> (3 * pp)) & 0x00070007u) | MAGIC,
+                                                    zm[(16 * run + 5 * i + pp) * GPK / 32]),
+                                    s_hi2[(16 * run + 5 * i + pp) * GPK / 32], s_lo2[(16 * run + 5 * i + pp) * GPK / 32]);
             const unsigned last =
                 ((w3[0] >> 15) & 0x00010001u) | ((w3[1] >> 14) & 0x00020002u) | ((w3[2] >> 13) & 0x00040004u);
-            out[16 * run + 15] = mul_scale<BF16>(sub_magic<BF16>(last | MAGIC, zm), s_hi2, s_lo2);
+            out[16 * run + 15] = mul_scale<BF16>(sub_magic<BF16>(last | MAGIC, zm[(16 * run + 15) * GPK / 32]),
+                                                 s_hi2[(16 * run + 15) * GPK / 32], s_lo2[(16 * run + 15) * GPK / 32]);
           }
         }
         if (round > 0) ok = mbar_wait_warp(empty(s), (round - 1) & 1, abort_flag, lim);
@@ -427,23 +439,31 @@ __global__ void __launch_bounds__(256) expand_kernel(const uint32_t* __restrict_
 #pragma unroll
     for (int k = 0; k < BITS; ++k) w[k] = __ldg(src + k);
   }
-  const unsigned sz = __ldg(sz_t + (size_t)((run * 32) / group) * N + row);
-  const unsigned s2 = (sz & 0xFFFFu) * 0x00010001u, zm = 0x64006400u | ((sz >> 16) * 0x00010001u);
-  unsigned out[16];
+  // scale and zero-point of the run's two halves of 16 columns (one group unless the groups are 16 wide)
+  unsigned s2[2], zm[2];
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    const unsigned sz = __ldg(sz_t + (size_t)((run * 32 + 16 * h) / group) * N + row);
+    s2[h] = (sz & 0xFFFFu) * 0x00010001u;
+    zm[h] = 0x64006400u | ((sz >> 16) * 0x00010001u);
+  }
+  unsigned out[16];   // pair p (columns 2p, 2p+1 of the run) belongs to half p / 8
   if (BITS == 4) {
 #pragma unroll
     for (int t = 0; t < 4; ++t)
 #pragma unroll
       for (int j = 0; j < 4; ++j)
-        out[4 * t + j] = mul_scale<false>(sub_magic<false>(((w[t % BITS] >> (4 * j)) & 0x000F000Fu) | 0x64006400u, zm), s2, 0);
+        out[4 * t + j] = mul_scale<false>(sub_magic<false>(((w[t % BITS] >> (4 * j)) & 0x000F000Fu) | 0x64006400u, zm[t / 2]),
+                                          s2[t / 2], 0);
   } else {
 #pragma unroll
     for (int k = 0; k < 3; ++k)
 #pragma unroll
       for (int pp = 0; pp < 5; ++pp)
-        out[5 * k + pp] = mul_scale<false>(sub_magic<false>(((w[k] >> (3 * pp)) & 0x00070007u) | 0x64006400u, zm), s2, 0);
+        out[5 * k + pp] = mul_scale<false>(sub_magic<false>(((w[k] >> (3 * pp)) & 0x00070007u) | 0x64006400u, zm[(5 * k + pp) / 8]),
+                                           s2[(5 * k + pp) / 8], 0);
     const unsigned last = ((w[0] >> 15) & 0x00010001u) | ((w[1] >> 14) & 0x00020002u) | ((w[BITS - 1] >> 13) & 0x00040004u);
-    out[15] = mul_scale<false>(sub_magic<false>(last | 0x64006400u, zm), s2, 0);
+    out[15] = mul_scale<false>(sub_magic<false>(last | 0x64006400u, zm[1]), s2[1], 0);
   }
   uint4* dst = reinterpret_cast<uint4*>(w16 + (size_t)row * K + run * 32);
 #pragma unroll
@@ -461,7 +481,7 @@ __global__ void __launch_bounds__(256) expand_outliers_kernel(const int32_t* __r
   }
 }
 
-template <int BITS, int TOK, bool EXP>
+template <int BITS, int TOK, bool EXP, int GPK = 1>
 gwq_status launch(const gwq_packed* P, const void* x, const float* tok_scale, const void* w16, int M, void* y, gwq_dtype yd,
                   cudaStream_t stream) {
   constexpr bool BF16 = false;   // operands are always fp16 here (see the file header)
@@ -493,7 +513,7 @@ gwq_status launch(const gwq_packed* P, const void* x, const float* tok_scale, co
   int stages = (220 * 1024 - 1024) / stage_bytes;
   if (stages > kMaxStages) stages = kMaxStages;
   const size_t smem = (size_t)stages * stage_bytes + 1024;
-  if (cudaFuncSetAttribute(prefill_kernel<BITS, TOK, BF16, EXP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  if (cudaFuncSetAttribute(prefill_kernel<BITS, TOK, BF16, EXP, GPK>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            (int)smem) != cudaSuccess)
     return GWQ_ERR_CUDA;
   PrefillArgs a;
@@ -502,13 +522,21 @@ gwq_status launch(const gwq_packed* P, const void* x, const float* tok_scale, co
   a.wait_cycles = pv->wait_cycles;
   const int ntn = (P->N + kTileN - 1) / kTileN, ntiles = ntn * ((M + TOK - 1) / TOK);
   const int grid = ntiles < pv->sm_count ? ntiles : pv->sm_count;   // persistent: at most one CTA per SM
-  prefill_kernel<BITS, TOK, BF16, EXP><<<grid, kCtaThreads, smem, stream>>>(tmx, tmw, a, stages, ntn, ntiles);
+  prefill_kernel<BITS, TOK, BF16, EXP, GPK><<<grid, kCtaThreads, smem, stream>>>(tmx, tmw, a, stages, ntn, ntiles);
   return cudaGetLastError() == cudaSuccess ? GWQ_OK : GWQ_ERR_CUDA;
 }
 
 template <int BITS>
 gwq_status launch_tok(const gwq_packed* P, const void* x, const float* tok_scale, int M, void* y, gwq_dtype yd,
                       cudaStream_t stream) {
+  if (P->group == 32) {   // small groups: the smallest and the largest token tile only
+    if (M <= 32) return launch<BITS, 32, false, 2>(P, x, tok_scale, nullptr, M, y, yd, stream);
+    return launch<BITS, 256, false, 2>(P, x, tok_scale, nullptr, M, y, yd, stream);
+  }
+  if (P->group == 16) {
+    if (M <= 32) return launch<BITS, 32, false, 4>(P, x, tok_scale, nullptr, M, y, yd, stream);
+    return launch<BITS, 256, false, 4>(P, x, tok_scale, nullptr, M, y, yd, stream);
+  }
   if (M <= 32) return launch<BITS, 32, false>(P, x, tok_scale, nullptr, M, y, yd, stream);
   if (M <= 64) return launch<BITS, 64, false>(P, x, tok_scale, nullptr, M, y, yd, stream);
   if (M <= 128) return launch<BITS, 128, false>(P, x, tok_scale, nullptr, M, y, yd, stream);

@@ -304,7 +304,7 @@ extern "C" gwq_status gwq_pack(const uint16_t* W, gwq_outliers* S, int32_t N, in
     GWQ_CUDA_TRY(cudaMalloc(&pv->xt, gwq_decode_scratch_bytes(K)));
     pv->xt_bytes = gwq_decode_scratch_bytes(K);
   }
-  if (group >= 64) {   // the tensor-core path (one scale per 64-column k-block) takes groups of 64 and 128 only
+  {   // group table of the tensor-core and streaming paths, transposed
     GWQ_CUDA_TRY(cudaMalloc(&pv->sz_t, ngroups * sizeof(uint32_t) + 16));
     transpose_scale_zero_kernel<<<(unsigned)((ngroups + 255) / 256), 256, 0, stream>>>(P->scales, P->zeros, pv->sz_t,
                                                                                        N, K / group);

@@ -163,6 +163,28 @@ def test_small_groups(layer, M, dtype):
     assert_linear_close(y, y_ref, bound)
 
 
+SMALL_GROUP_LAYERS = [
+    (520, 1024, 0.01, 4, 16, 33),      # the paper's own group size (Section 3.2), ragged last tile
+    (520, 1024, 0.02, 3, 16, 34),
+    (384, 2048, 0.01, 4, 32, 35),
+    (384, 2048, 0.005, 3, 32, 36),
+]
+
+
+@pytest.mark.parametrize("layer", SMALL_GROUP_LAYERS)
+@pytest.mark.parametrize("M,dtype", [(1, "f16"), (1, "bf16"), (2, "f16"), (4, "bf16"), (8, "f16"), (17, "f16"), (32, "bf16"),
+                                     (33, "f16"), (300, "bf16"), (2100, "f16")])
+def test_small_groups_on_the_fast_paths(layer, M, dtype):
+    # K a multiple of 128: groups of 16 and 32 run on the tensor cores (one scale per 16 or 32 columns inside the
+    # 64-column k-block; the weights expanded beforehand from 2048 tokens on) and, for one token, on the streaming kernel
+    P, L, w_hat = _layer(*layer)
+    bits16, xv = synth.make_activations(M, P.K, seed=160 + M, dtype=dtype, heavy_channels=8 if M > 32 else 0)
+    y_ref, bound = orc.linear(xv, w_hat)
+    y = gwq.gwq_linear(P, x_tensor(bits16, dtype), out_dtype=torch.float32)
+    assert gwq.gwq_device_status(P) == 0
+    assert_linear_close(y, y_ref, bound)
+
+
 @pytest.mark.parametrize("layer", [DECODE_LAYERS[0], DECODE_LAYERS[3]])
 @pytest.mark.parametrize("M", [1, 8, 16, 32, 200])
 def test_repeated_calls_give_the_same_bits(layer, M):
