@@ -61,7 +61,7 @@ struct Variant {
   int nbuf;    // 0: all of x staged up front; 2, 3: per-warp ring of that many tiles
   int rt;      // m16 tiles per CTA (rows = 16 rt)
   int deep;    // 1: eight groups of codes in flight per warp instead of four (one tile, up to 8 tokens; two CTAs per SM)
-  bool g64;    // groups of 64 columns
+  int gs;      // scale groups per 128-column step: 1 (groups of 128), 2 (64), 4 (32), 8 (16)
 };
 
 size_t smem_bytes(const Variant& v, int K, int M, int cvcap);
@@ -77,7 +77,8 @@ constexpr int kChunkPieces = kChunkGroups * 16;      // 16-byte pieces per token
 constexpr int kRowPitch = kChunkPieces + kChunkPieces / 8 + 4;   // pieces, with padding
 constexpr int kTilePitch = 16;   // pieces per token row of a warp tile: no padding, the pieces of a row are permuted
 
-__host__ __device__ constexpr int token_blocks(int tp, bool g64) { return g64 ? (tp <= 4 ? 1 : tp / 4) : (tp <= 8 ? 1 : tp / 8); }
+// token blocks of 8 / gs tokens (an MMA has 8 columns: tokens x groups of the step)
+__host__ __device__ constexpr int token_blocks(int tp, int gs) { return tp * gs <= 8 ? 1 : tp * gs / 8; }
 
 }  // namespace gwq_decode
 
@@ -212,9 +213,10 @@ __device__ __forceinline__ void step_ones(const unsigned (&xr)[NB][16], float (&
 
 // Subtract variant (bf16 activations): (bits | magic) - (z | magic) = q - z exactly in bf16; one
 // accumulator, no ones operand.  zma / zmb hold magic | z in both halves.
+// (zma[h], zmb[h]: for pairs 8 h .. 8 h + 7 of the run; the two differ only with groups of 16 columns)
 template <int BITS, int NB>
-__device__ __forceinline__ void step_sub(const unsigned (&qa)[BITS], const unsigned (&qb)[BITS], unsigned zma,
-                                         unsigned zmb, const unsigned (&xr)[NB][16], AccSub<NB>& acc) {
+__device__ __forceinline__ void step_sub(const unsigned (&qa)[BITS], const unsigned (&qb)[BITS], const unsigned (&zma)[2],
+                                         const unsigned (&zmb)[2], const unsigned (&xr)[NB][16], AccSub<NB>& acc) {
   constexpr unsigned MAGIC = 0x43004300u;  // bf16 128.0: ulp = 1
   unsigned a[16], b[16];
   if (BITS == 4) {
@@ -222,23 +224,23 @@ __device__ __forceinline__ void step_sub(const unsigned (&qa)[BITS], const unsig
     for (int i = 0; i < 4; ++i)
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        a[4 * i + j] = sub_zero_bf16(((qa[i % BITS] >> (4 * j)) & 0x000F000Fu) | MAGIC, zma);
-        b[4 * i + j] = sub_zero_bf16(((qb[i % BITS] >> (4 * j)) & 0x000F000Fu) | MAGIC, zmb);
+        a[4 * i + j] = sub_zero_bf16(((qa[i % BITS] >> (4 * j)) & 0x000F000Fu) | MAGIC, zma[i >> 1]);
+        b[4 * i + j] = sub_zero_bf16(((qb[i % BITS] >> (4 * j)) & 0x000F000Fu) | MAGIC, zmb[i >> 1]);
       }
   } else {
 #pragma unroll
     for (int i = 0; i < 3; ++i)
 #pragma unroll
       for (int p = 0; p < 5; ++p) {
-        a[5 * i + p] = sub_zero_bf16(((qa[i] >> (3 * p)) & 0x00070007u) | MAGIC, zma);
-        b[5 * i + p] = sub_zero_bf16(((qb[i] >> (3 * p)) & 0x00070007u) | MAGIC, zmb);
+        a[5 * i + p] = sub_zero_bf16(((qa[i] >> (3 * p)) & 0x00070007u) | MAGIC, zma[(5 * i + p) >> 3]);
+        b[5 * i + p] = sub_zero_bf16(((qb[i] >> (3 * p)) & 0x00070007u) | MAGIC, zmb[(5 * i + p) >> 3]);
       }
     const unsigned la = ((qa[0] >> 15) & 0x00010001u) | ((qa[1] >> 14) & 0x00020002u) |
                         ((qa[BITS - 1] >> 13) & 0x00040004u);
     const unsigned lb = ((qb[0] >> 15) & 0x00010001u) | ((qb[1] >> 14) & 0x00020002u) |
                         ((qb[BITS - 1] >> 13) & 0x00040004u);
-    a[15] = sub_zero_bf16(la | MAGIC, zma);
-    b[15] = sub_zero_bf16(lb | MAGIC, zmb);
+    a[15] = sub_zero_bf16(la | MAGIC, zma[1]);
+    b[15] = sub_zero_bf16(lb | MAGIC, zmb[1]);
   }
 #pragma unroll
   for (int nb = 0; nb < NB; ++nb) {
@@ -360,19 +362,27 @@ __device__ __forceinline__ void unroll_slots(F&& f, std::integer_sequence<int, I
 // scale and zero-point it applies; the two halves of a token meet in the final sum.  With more than one token the sums
 // of x come from the all-ones MMA (which sees the same zeros); a single token's are reduced over half a warp each.
 // TP <= 16 there.
+// GS = 4, 8 (groups of 32, 16 columns) continue the scheme: a block holds 8 / GS tokens, column n is token n % (8 / GS)
+// restricted to group n / (8 / GS) of the step.  A lane's run of 32 columns is one group of 32 (its accumulator columns
+// 2t, 2t+1 are two tokens of that group), or two groups of 16 (pairs 0..7 and 8..15 of the run: column 2t is the first,
+// 2t+1 the second, one token per block; the two halves of the B fragment come from different places and the lane
+// applies two scales).  The sums of x come from the all-ones MMA.  Activations staged up front only.
 // RT: m16 tiles (16 rows each) of the CTA; every warp step loads the B fragments once and runs all RT tiles on them.
 // DEEP: eight groups of codes in flight per warp (grids that leave an SM at most two CTAs: fewer warps have to keep
 // as many bytes in flight).
-template <int BITS, int TP, bool BF16, int NBUF, bool G64, int RT, bool DEEP>
-__global__ void __launch_bounds__(kThreads, min_blocks(token_blocks(TP, G64), RT, DEEP))
+template <int BITS, int TP, bool BF16, int NBUF, int GS, int RT, bool DEEP>
+__global__ void __launch_bounds__(kThreads, min_blocks(token_blocks(TP, GS), RT, DEEP))
 decode_kernel(const MultiArgs ma) {
   constexpr int R = 16 * RT;                       // rows of the CTA
   constexpr int D = DEEP ? 8 : (RT == 1 ? 4 : 2);  // groups of codes in flight per warp and tile
-  constexpr int NB = token_blocks(TP, G64);        // token blocks of the MMA (8 tokens; 4 with groups of 64)
+  constexpr bool G64 = GS == 2;
+  constexpr int TB = 8 / GS;                       // tokens of a block
+  constexpr int NB = token_blocks(TP, GS);         // token blocks of the MMA
+  static_assert(GS < 4 || (NBUF == 0 && RT == 1 && !DEEP), "small groups: staged activations, one tile");
   constexpr int WPR = BITS;                        // words per run of 32 columns
   // raw path: sum_k x_k of a group from shared memory (one token), from the table that comes with the
   // token-major copy (ring mode), else from a second MMA with an all-ones A operand
-  constexpr bool ONES = !BF16 && TP != 1 && (G64 || NBUF == 0);
+  constexpr bool ONES = !BF16 && ((TP != 1 && (GS > 1 || NBUF == 0)) || GS > 2);
   constexpr int OWN = 2 * RT;                      // rows whose outliers a warp adds
 
   // the layer this CTA works for and its row block inside that layer
@@ -397,7 +407,7 @@ decode_kernel(const MultiArgs ma) {
   const int K = ma.K, M = ma.M;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int ngroups = K >> 7;               // warp steps of 128 columns in a row
-  const int ntab = G64 ? 2 * ngroups : ngroups;   // scale / zero-point entries in a row
+  const int ntab = GS * ngroups;   // scale / zero-point entries in a row
   // shared: zero page 64 B | scale and zero-point table [ntab][R] u32 | red [kWarps][RT][NB][128] f32 |
   //         outl [R][TP] f32 | outlier entries [kWarps][OWN][cvcap] u32 (x staged up front only) | x buffers
   // (the table is group-major: the eight rows a load instruction asks for are eight neighbouring words, no bank
@@ -630,16 +640,20 @@ decode_kernel(const MultiArgs ma) {
   // lane constants inside a chunk buffer: this lane's 64-byte segment of group `warp` for token gid
   // of every token block (lanes without a token read the zero page), the scale tables, the x sums
   // (ring mode: the four pieces of the segment sit in one aligned block of the permuted row, in the order i ^ xcx)
-  int xoff[NB], xcx[NB];
+  int xoff[NB][2], xcx[NB];   // [0]: pairs 0..7 of the run, [1]: pairs 8..15 (they differ only with groups of 16)
 #pragma unroll
   for (int nb = 0; nb < NB; ++nb) {
-    const int m = G64 ? nb * 4 + (gid & 3) : nb * 8 + gid;
-    const bool live = m < M && (!G64 || (gid >> 2) == (t >> 1));   // groups of 64: the other group's columns read as zero
-    xoff[nb] = !live ? -1 : (NBUF == 0 ? xs_piece(warp * 16 + t * 4, m) : m * kTilePitch + ((t ^ ((m >> 1) & 1)) << 2));
-    xcx[nb] = (NBUF == 0 || !live) ? 0 : ((t >> 1) ^ ((m & 1) << 1));
+    const int m = nb * TB + (gid % TB);
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh) {
+      // the column's group must be the group of the lane's (half) run: the other groups' columns read as zero
+      const bool live = m < M && (GS == 8 ? gid == 2 * t + hh : (gid / TB) == (t * GS) / 4);
+      xoff[nb][hh] = !live ? -1 : (NBUF == 0 ? xs_piece(warp * 16 + t * 4, m) : m * kTilePitch + ((t ^ ((m >> 1) & 1)) << 2));
+    }
+    xcx[nb] = (NBUF == 0 || xoff[nb][0] < 0) ? 0 : ((t >> 1) ^ ((m & 1) << 1));
   }
-  // scale | zero-point << 16 of row gid of tile 0, group `warp` (groups of 64: the lane's own half of step `warp`)
-  const uint32_t* tp = sm_tab + (G64 ? 2 * warp + (t >> 1) : warp) * R + gid;
+  // scale | zero-point << 16 of row gid of tile 0, first group of the lane's run in step `warp`
+  const uint32_t* tp = sm_tab + (GS * warp + (GS == 8 ? 2 * t : (t * GS) / 4)) * R + gid;
   const int xsum_off = (NBUF == 0 ? xs_piece(warp * 16 + (lane >> 1), 0) : ((lane >> 1) ^ (lane >> 4))) * 2 + (lane & 1);   // 8-byte units, token 0
 
   float yacc[RT][NB][4];
@@ -664,10 +678,11 @@ decode_kernel(const MultiArgs ma) {
     unsigned xr[NB][16];
 #pragma unroll
     for (int nb = 0; nb < NB; ++nb) {
-      const uint4* seg = xoff[nb] >= 0 ? buf + xoff[nb] : reinterpret_cast<const uint4*>(smem_raw);
+      const uint4* seg0 = xoff[nb][0] >= 0 ? buf + xoff[nb][0] : reinterpret_cast<const uint4*>(smem_raw);
+      const uint4* seg1 = GS == 8 ? (xoff[nb][1] >= 0 ? buf + xoff[nb][1] : reinterpret_cast<const uint4*>(smem_raw)) : seg0;
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
-        const uint4 v = seg[i ^ xcx[nb]];
+        const uint4 v = (i < 2 ? seg0 : seg1)[i ^ xcx[nb]];
         xr[nb][4 * i] = v.x; xr[nb][4 * i + 1] = v.y; xr[nb][4 * i + 2] = v.z; xr[nb][4 * i + 3] = v.w;
       }
     }
@@ -681,7 +696,7 @@ decode_kernel(const MultiArgs ma) {
         const float2 g2 = __ldg(reinterpret_cast<const float2*>(ma.xg + (size_t)(warp + kWarps * c) * TP + nb * 8 + 2 * t));
         xs[nb][0] = g2.x; xs[nb][1] = g2.y;
       }
-    } else if (!BF16) {   // one token: lane L adds columns 4L..4L+3, then the lanes of the group are summed
+    } else if (!BF16 && GS <= 2) {   // one token: lane L adds columns 4L..4L+3, then the lanes of the group are summed
       const uint2 h4 = reinterpret_cast<const uint2*>(buf)[xsum_off];
       const float2 f0 = __half22float2(*reinterpret_cast<const __half2*>(&h4.x));
       const float2 f1 = __half22float2(*reinterpret_cast<const __half2*>(&h4.y));
@@ -696,23 +711,27 @@ decode_kernel(const MultiArgs ma) {
 #pragma unroll
     for (int rt = 0; rt < RT; ++rt) {
       // (s 2^24, s z) on the raw path, (s, magic | z) on the subtract path
-      float2 ta, tb;
-      {
-        const unsigned sza = tp[16 * rt], szb = tp[16 * rt + 8];
+      float2 ta[2], tb[2];   // per accumulator column parity (two groups of 16 per lane), else both the same
+#pragma unroll
+      for (int e = 0; e < (GS == 8 ? 2 : 1); ++e) {
+        const unsigned sza = tp[16 * rt + e * R], szb = tp[16 * rt + 8 + e * R];
         const float sa = __half2float(__ushort_as_half((unsigned short)sza));
         const float sb = __half2float(__ushort_as_half((unsigned short)szb));
         const unsigned za = sza >> 16, zb = szb >> 16;
         if (BF16) {
-          ta = make_float2(sa, __uint_as_float(0x43004300u | (za * 0x00010001u)));
-          tb = make_float2(sb, __uint_as_float(0x43004300u | (zb * 0x00010001u)));
+          ta[e] = make_float2(sa, __uint_as_float(0x43004300u | (za * 0x00010001u)));
+          tb[e] = make_float2(sb, __uint_as_float(0x43004300u | (zb * 0x00010001u)));
         } else {
-          ta = make_float2(sa * 16777216.f, sa * (float)za);
-          tb = make_float2(sb * 16777216.f, sb * (float)zb);
+          ta[e] = make_float2(sa * 16777216.f, sa * (float)za);
+          tb[e] = make_float2(sb * 16777216.f, sb * (float)zb);
         }
       }
+      if (GS != 8) { ta[1] = ta[0]; tb[1] = tb[0]; }
       typename StepAcc<BITS, NB, BF16>::type acc;
       if constexpr (BF16) {
-        step_sub<BITS, NB>(wa[rt][d], wb[rt][d], __float_as_uint(ta.y), __float_as_uint(tb.y), xr, acc);
+        const unsigned zma[2] = {__float_as_uint(ta[0].y), __float_as_uint(ta[1].y)};
+        const unsigned zmb[2] = {__float_as_uint(tb[0].y), __float_as_uint(tb[1].y)};
+        step_sub<BITS, NB>(wa[rt][d], wb[rt][d], zma, zmb, xr, acc);
       } else if constexpr (BITS == 4) {
         step_raw4<NB>(wa[rt][d], wb[rt][d], xr, acc);
       } else {
@@ -727,8 +746,8 @@ decode_kernel(const MultiArgs ma) {
       for (int nb = 0; nb < NB; ++nb) {
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-          if (TP == 1 && (i & 1)) continue;   // a single token lives in accumulator column 0
-          const float2 tt = i < 2 ? ta : tb;
+          if (TP == 1 && GS < 8 && (i & 1)) continue;   // a single token lives in the even accumulator columns
+          const float2 tt = i < 2 ? ta[i & 1] : tb[i & 1];
           if constexpr (BF16) {
             yacc[rt][nb][i] = fmaf(tt.x, acc.c[nb][i], yacc[rt][nb][i]);
           } else if constexpr (BITS == 4) {
@@ -741,7 +760,7 @@ decode_kernel(const MultiArgs ma) {
         }
       }
     }
-    tp += (G64 ? 2 * kWarps : kWarps) * R;
+    tp += GS * kWarps * R;
   };
   for (int c0 = 0; c0 < nsteps; c0 += D)   // the register slot of a step is a compile-time constant
     unroll_slots([&](auto slot) { if (c0 + decltype(slot)::value < nsteps) do_step(c0 + decltype(slot)::value, slot); },
@@ -764,24 +783,24 @@ decode_kernel(const MultiArgs ma) {
     const int row = r0 + lr;
     if (row < N) {
       const int rt = lr >> 4, l16 = lr & 15;
-      const int nb = G64 ? m >> 2 : m >> 3, tk = G64 ? m & 3 : m & 7;
+      const int nb = m / TB, tk = m % TB;
       float v = sm_out[lr * TP + m];
 #pragma unroll
       for (int w = 0; w < kWarps; ++w) {
         const float* r = sm_red + ((w * RT + rt) * NB + nb) * 128 + l16 * 8 + tk;
-        v += r[0];
-        if (G64) v += r[4];   // the token's second group of every step
+#pragma unroll
+        for (int g = 0; g < GS; ++g) v += r[TB * g];   // the token's column in every group of the step
       }
       store_y(yout, ma.yd, (long long)m * N + row, v);
     }
   }
 }
 
-template <int BITS, int TP, bool BF16, int NBUF, bool G64, int RT, bool DEEP = false>
+template <int BITS, int TP, bool BF16, int NBUF, int GS, int RT, bool DEEP = false>
 cudaError_t launch(const Variant& v, const MultiArgs& a, cudaStream_t stream) {
   const size_t smem = smem_bytes(v, a.K, a.M, a.cvcap);
   if (smem > 48 * 1024) {
-    cudaError_t e = cudaFuncSetAttribute(decode_kernel<BITS, TP, BF16, NBUF, G64, RT, DEEP>,
+    cudaError_t e = cudaFuncSetAttribute(decode_kernel<BITS, TP, BF16, NBUF, GS, RT, DEEP>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
   }
@@ -795,57 +814,69 @@ cudaError_t launch(const Variant& v, const MultiArgs& a, cudaStream_t stream) {
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, decode_kernel<BITS, TP, BF16, NBUF, G64, RT, DEEP>, a);
+  return cudaLaunchKernelEx(&cfg, decode_kernel<BITS, TP, BF16, NBUF, GS, RT, DEEP>, a);
 }
 
 // the variants that exist: x staged up front for up to 8 tokens, rings of two tiles up to 8 tokens and of three beyond
-// (two when shared memory is short); two m16 tiles per CTA up to 8 tokens with groups of 128; groups of 64 up to 16 tokens
-template <int BITS, bool BF16, int TP, bool G64>
+// (two when shared memory is short); two m16 tiles per CTA, or eight groups of codes in flight, up to 8 tokens with
+// groups of 128; groups of 64 up to 16 tokens; groups of 32 up to 4 tokens and of 16 for one token, staged only
+template <int BITS, bool BF16, int TP, int GS>
 cudaError_t launch_tp(const Variant& v, const MultiArgs& a, cudaStream_t stream) {
-  if (v.nbuf == 0) {
-    if constexpr (TP <= 8) {
-      if (v.rt == 2) {
-        if constexpr (!G64) return launch<BITS, TP, BF16, 0, G64, 2>(v, a, stream);
-        return cudaErrorInvalidValue;
+  if constexpr (GS >= 4) {
+    if (v.nbuf == 0 && v.rt == 1 && !v.deep) return launch<BITS, TP, BF16, 0, GS, 1>(v, a, stream);
+    return cudaErrorInvalidValue;
+  } else {
+    if (v.nbuf == 0) {
+      if constexpr (TP <= 8) {
+        if (v.rt == 2) {
+          if constexpr (GS == 1) return launch<BITS, TP, BF16, 0, GS, 2>(v, a, stream);
+          return cudaErrorInvalidValue;
+        }
+        if constexpr (GS == 1) {
+          if (v.deep) return launch<BITS, TP, BF16, 0, GS, 1, true>(v, a, stream);
+        }
+        return launch<BITS, TP, BF16, 0, GS, 1>(v, a, stream);
       }
-      if constexpr (!G64) {
-        if (v.deep) return launch<BITS, TP, BF16, 0, G64, 1, true>(v, a, stream);
-      }
-      return launch<BITS, TP, BF16, 0, G64, 1>(v, a, stream);
+      return cudaErrorInvalidValue;
     }
+    if (v.rt == 2) {
+      if constexpr (GS == 1 && TP <= 8) {
+        if (v.nbuf == 2) return launch<BITS, TP, BF16, 2, GS, 2>(v, a, stream);
+      }
+      return cudaErrorInvalidValue;
+    }
+    if constexpr (GS == 1 && TP <= 8) {
+      if (v.deep && v.nbuf == 2) return launch<BITS, TP, BF16, 2, GS, 1, true>(v, a, stream);
+    }
+    if (v.nbuf == 2) return launch<BITS, TP, BF16, 2, GS, 1>(v, a, stream);
+    if constexpr (TP >= 16) return launch<BITS, TP, BF16, 3, GS, 1>(v, a, stream);
     return cudaErrorInvalidValue;
   }
-  if (v.rt == 2) {
-    if constexpr (!G64 && TP <= 8) {
-      if (v.nbuf == 2) return launch<BITS, TP, BF16, 2, G64, 2>(v, a, stream);
-    }
-    return cudaErrorInvalidValue;
-  }
-  if constexpr (!G64 && TP <= 8) {
-    if (v.deep && v.nbuf == 2) return launch<BITS, TP, BF16, 2, G64, 1, true>(v, a, stream);
-  }
-  if (v.nbuf == 2) return launch<BITS, TP, BF16, 2, G64, 1>(v, a, stream);
-  if constexpr (TP >= 16) return launch<BITS, TP, BF16, 3, G64, 1>(v, a, stream);
-  return cudaErrorInvalidValue;
 }
 
 template <int BITS, bool BF16>
 cudaError_t launch_any(const Variant& v, const MultiArgs& a, cudaStream_t stream) {
-  if (v.g64) {
+  if (v.gs == 8) return v.tp == 1 ? launch_tp<BITS, BF16, 1, 8>(v, a, stream) : cudaErrorInvalidValue;
+  if (v.gs == 4) {
+    if (v.tp == 1) return launch_tp<BITS, BF16, 1, 4>(v, a, stream);
+    if (v.tp == 4) return launch_tp<BITS, BF16, 4, 4>(v, a, stream);
+    return cudaErrorInvalidValue;
+  }
+  if (v.gs == 2) {
     switch (v.tp) {
-      case 1: return launch_tp<BITS, BF16, 1, true>(v, a, stream);
-      case 4: return launch_tp<BITS, BF16, 4, true>(v, a, stream);
-      case 8: return launch_tp<BITS, BF16, 8, true>(v, a, stream);
-      case 16: return launch_tp<BITS, BF16, 16, true>(v, a, stream);
+      case 1: return launch_tp<BITS, BF16, 1, 2>(v, a, stream);
+      case 4: return launch_tp<BITS, BF16, 4, 2>(v, a, stream);
+      case 8: return launch_tp<BITS, BF16, 8, 2>(v, a, stream);
+      case 16: return launch_tp<BITS, BF16, 16, 2>(v, a, stream);
     }
     return cudaErrorInvalidValue;
   }
   switch (v.tp) {
-    case 1: return launch_tp<BITS, BF16, 1, false>(v, a, stream);
-    case 4: return launch_tp<BITS, BF16, 4, false>(v, a, stream);
-    case 8: return launch_tp<BITS, BF16, 8, false>(v, a, stream);
-    case 16: return launch_tp<BITS, BF16, 16, false>(v, a, stream);
-    case 32: return launch_tp<BITS, BF16, 32, false>(v, a, stream);
+    case 1: return launch_tp<BITS, BF16, 1, 1>(v, a, stream);
+    case 4: return launch_tp<BITS, BF16, 4, 1>(v, a, stream);
+    case 8: return launch_tp<BITS, BF16, 8, 1>(v, a, stream);
+    case 16: return launch_tp<BITS, BF16, 16, 1>(v, a, stream);
+    case 32: return launch_tp<BITS, BF16, 32, 1>(v, a, stream);
   }
   return cudaErrorInvalidValue;
 }

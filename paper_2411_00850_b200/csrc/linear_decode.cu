@@ -6,9 +6,9 @@
 namespace gwq_decode {
 
 size_t smem_bytes(const Variant& v, int K, int M, int cvcap) {
-  const int R = 16 * v.rt, NB = token_blocks(v.tp, v.g64);
+  const int R = 16 * v.rt, NB = token_blocks(v.tp, v.gs);
   const int ngroups = K / 128, nchunks = (ngroups + kChunkGroups - 1) / kChunkGroups;
-  const size_t fixed = 64 + (size_t)R * (v.g64 ? 2 * ngroups : ngroups) * 4 + (size_t)kWarps * v.rt * NB * 128 * 4 +
+  const size_t fixed = 64 + (size_t)R * (v.gs * ngroups) * 4 + (size_t)kWarps * v.rt * NB * 128 * 4 +
                        (size_t)R * v.tp * 4;
   if (v.nbuf != 0) return fixed + (size_t)kWarps * v.nbuf * M * kTilePitch * 16;
   return fixed + (size_t)kWarps * 2 * v.rt * cvcap * 4 + (size_t)nchunks * M * kRowPitch * 16;
@@ -80,14 +80,18 @@ constexpr size_t kStageAllLimitTwoTiles = 96 * 1024;
 // 128, same K, group size and bit width in every layer, shared memory for at least a ring of two tiles.
 bool plan(const gwq_packed* const* P, int count, int M, Variant* v, int* cvcap) {
   if (count < 1 || count > kMaxLayers || M < 1 || M > 32) return false;
-  const bool g64 = P[0]->group == 64;
+  const int group = P[0]->group;
+  if (group != 128 && group != 64 && group != 32 && group != 16) return false;
+  const bool g64 = group == 64;
+  const int gs = 128 / group;
+  if (gs >= 4 && M > (gs == 4 ? 4 : 1)) return false;   // small groups: the token blocks shrink with the group
   const int K = P[0]->K;
   if (K % 128 != 0) return false;   // a warp step is 128 columns
   if (g64 && M > kMaxTokens64) return false;
   long long rows = 0, nnz = 0;
   for (int i = 0; i < count; ++i) {
     const gwq_priv* pvi = static_cast<const gwq_priv*>(P[i]->priv);
-    if ((P[i]->group != 128 && P[i]->group != 64) || P[i]->group != P[0]->group || !pvi->cv || !pvi->sz_t ||
+    if (P[i]->group != group || !pvi->cv || !pvi->sz_t ||
         P[i]->K != K || P[i]->bits != P[0]->bits)
       return false;
     if (g64 && M > 8 && (long long)P[i]->N * K > kMaxWeights64Wide) return false;
@@ -96,7 +100,7 @@ bool plan(const gwq_packed* const* P, int count, int M, Variant* v, int* cvcap) 
   }
   const gwq_priv* pv = static_cast<const gwq_priv*>(P[0]->priv);
   const int sms = pv->sm_count > 0 ? pv->sm_count : 148;
-  v->g64 = g64;
+  v->gs = gs;
   v->tp = M == 1 ? 1 : (M <= 4 ? 4 : (M <= 8 ? 8 : (M <= 16 ? 16 : 32)));
   // Two tiles per CTA (up to 8 tokens, groups of 128) halve the per-row cost of everything a CTA does once, but an SM
   // holds two such CTAs instead of three: they are taken where they turn a grid of more than one wave into a single one
@@ -105,15 +109,15 @@ bool plan(const gwq_packed* const* P, int count, int M, Variant* v, int* cvcap) 
     blocks1 += (P[i]->N + 15) / 16;
     blocks2 += (P[i]->N + 31) / 32;
   }
-  v->rt = (!g64 && v->tp <= 8 && blocks1 > 3LL * sms && blocks2 <= 2LL * sms) ? 2 : 1;
-  if (GWQ_TUNE_RT == 1 || (GWQ_TUNE_RT == 2 && !g64 && v->tp <= 8)) v->rt = GWQ_TUNE_RT;
+  v->rt = (gs == 1 && v->tp <= 8 && blocks1 > 3LL * sms && blocks2 <= 2LL * sms) ? 2 : 1;
+  if (GWQ_TUNE_RT == 1 || (GWQ_TUNE_RT == 2 && gs == 1 && v->tp <= 8)) v->rt = GWQ_TUNE_RT;
   long long blocks = 0;
   for (int i = 0; i < count; ++i) blocks += (P[i]->N + 16 * v->rt - 1) / (16 * v->rt);
   // a grid that leaves an SM two CTAs at most anyway: twice the codes in flight per warp (more registers, which then
   // cost no occupancy)
-  v->deep = (v->rt == 1 && !g64 && v->tp <= 8 && blocks <= 2LL * sms) ? 1 : 0;
+  v->deep = (v->rt == 1 && gs == 1 && v->tp <= 8 && blocks <= 2LL * sms) ? 1 : 0;
 #ifdef GWQ_TUNE_DEEP
-  v->deep = (v->rt == 1 && !g64 && v->tp <= 8) ? GWQ_TUNE_DEEP : 0;
+  v->deep = (v->rt == 1 && gs == 1 && v->tp <= 8) ? GWQ_TUNE_DEEP : 0;
 #endif
   const int nchunks = (K / 128 + kChunkGroups - 1) / kChunkGroups;
   const size_t lim = v->rt == 2 ? kStageAllLimitTwoTiles : (blocks <= 2LL * sms ? kStageAllLimitSmallGrid : kStageAllLimit);
@@ -124,6 +128,7 @@ bool plan(const gwq_packed* const* P, int count, int M, Variant* v, int* cvcap) 
   if (v->tp <= 8 && (size_t)nchunks * M * kRowPitch * 16 <= lim &&
       smem_bytes(*v, K, M, *cvcap) <= kSmemPerCta)
     return true;
+  if (gs >= 4) return false;                // small groups: staged activations only
   if (v->tp > 1 && !pv->xt) return false;   // ring mode gathers the outliers' activations from a token-major copy
   v->nbuf = v->tp <= 8 ? 2 : 3;
   if (v->nbuf == 3 && smem_bytes(*v, K, M, *cvcap) > kSmemPerCta) v->nbuf = 2;
