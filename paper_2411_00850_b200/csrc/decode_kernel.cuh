@@ -472,8 +472,10 @@ decode_kernel(const MultiArgs ma) {
 
   // CSR extents of the owned rows: jr[i] .. jr[i + 1] are the entries of owned row i
   int jr[OWN + 1];
+  if (NBUF != 0) {
 #pragma unroll
-  for (int i = 0; i <= OWN; ++i) jr[i] = __shfl_sync(0xFFFFFFFFu, rp, i);
+    for (int i = 0; i <= OWN; ++i) jr[i] = __shfl_sync(0xFFFFFFFFu, rp, i);
+  }
   constexpr int VT = TP < 8 ? TP : 8, TS = TP / VT, EPB = 32 / TS;
   constexpr int kPre = TP <= 8 ? 2 : 3;   // batches of EPB entries per row: 64 entries up to 8 tokens, 48 / 24 beyond
   unsigned epre[2][kPre];
@@ -487,17 +489,6 @@ decode_kernel(const MultiArgs ma) {
         const int j = jr[rr] + u * EPB + lane / TS;
         epre[rr][u] = j < jr[rr + 1] ? __ldg(cvp + j) : 0u;   // value 0, column 0
       }
-    }
-  } else {
-    // everything staged: the outlier entries of the owned rows (up to cvcap each) are copied into shared memory now
-    // and meet the staged activations before the K loop
-    const unsigned dst0 = (unsigned)__cvta_generic_to_shared(sm_cv + warp * OWN * kCvCap);
-#pragma unroll
-    for (int rr = 0; rr < OWN; ++rr) {
-      const int n = min(jr[rr + 1] - jr[rr], kCvCap);
-      for (int e = lane; e < n; e += 32)
-        asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst0 + (unsigned)(rr * kCvCap + e) * 4u),
-                     "l"(cvp + jr[rr] + e));
     }
   }
   // ---- from here on x is read
@@ -542,7 +533,23 @@ decode_kernel(const MultiArgs ma) {
   } else {
     stage_tile(0);
   }
-  asm volatile("cp.async.commit_group;" ::: "memory");   // also carries the scale / zero-point tables and the outlier entries
+  asm volatile("cp.async.commit_group;" ::: "memory");   // also carries the scale / zero-point tables
+  if (NBUF == 0) {
+    // everything staged: the outlier entries of the owned rows (up to cvcap each) are copied into shared memory in a
+    // group of their own (their addresses need the row pointers, a second trip to memory that nothing else waits
+    // for); they meet the staged activations after the K loop
+#pragma unroll
+    for (int i = 0; i <= OWN; ++i) jr[i] = __shfl_sync(0xFFFFFFFFu, rp, i);
+    const unsigned dst0 = (unsigned)__cvta_generic_to_shared(sm_cv + warp * OWN * kCvCap);
+#pragma unroll
+    for (int rr = 0; rr < OWN; ++rr) {
+      const int n = min(jr[rr + 1] - jr[rr], kCvCap);
+      for (int e = lane; e < n; e += 32)
+        asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst0 + (unsigned)(rr * kCvCap + e) * 4u),
+                     "l"(cvp + jr[rr] + e));
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  }
   if (NBUF != 0) {   // the tiles of the following steps, one group each
 #pragma unroll
     for (int c = 1; c + 1 < kBufs; ++c) {
@@ -605,37 +612,8 @@ decode_kernel(const MultiArgs ma) {
       if ((lane % LPV) / TS == 0) sm_out[(OWN * warp + rr) * TP + tok] = v[0];
     }
   }
-  asm volatile("cp.async.wait_group %0;" ::"n"(NBUF == 0 ? 0 : NBUF - 2) : "memory");   // tables (and first tile) landed
+  asm volatile("cp.async.wait_group %0;" ::"n"(NBUF == 0 ? 1 : NBUF - 2) : "memory");   // tables and x (or first tile) landed
   __syncthreads();
-
-  if (NBUF == 0) {
-    // CSR outliers of the owned rows, while the codes are still on their way: lane = entry, every token per lane,
-    // one transposing reduction per row; the entries come from shared memory (those beyond cvcap, rare, from global
-    // memory), the activations from the staged copy
-    const uint16_t* xs16 = reinterpret_cast<const uint16_t*>(sm_x);
-    const uint32_t* mycv = sm_cv + warp * OWN * kCvCap;
-#pragma unroll
-    for (int rr = 0; rr < OWN; ++rr) {
-      const int jb = jr[rr], je = jr[rr + 1];
-      float v[TP];
-#pragma unroll
-      for (int m = 0; m < TP; ++m) v[m] = 0.f;
-      for (int e0 = lane; e0 < je - jb; e0 += 32) {
-        const unsigned e = e0 < kCvCap ? mycv[rr * kCvCap + e0] : __ldg(cvp + jb + e0);
-        const float wv = __half2float(__ushort_as_half((unsigned short)(e >> 16)));
-        const unsigned col = e & 0xFFFFu;
-        const int base = (int)(col >> 10) * buf_pieces;            // chunk = col / 1024
-        const int pc = (int)((col & 1023u) >> 3), sub = (int)(col & 7u);
-#pragma unroll
-        for (int m = 0; m < TP; ++m)
-          if (TP == 1 || m < M)
-            v[m] = fmaf(wv, act_to_float<BF16>(xs16[((base + xs_piece(pc, m)) << 3) + sub]), v[m]);
-      }
-      reduce_tokens<TP, 1>(v, lane);
-      constexpr int LPT = 32 / TP;   // lanes per token after the reduction
-      if ((lane & (LPT - 1)) == 0) sm_out[(OWN * warp + rr) * TP + lane / LPT] = v[0];
-    }
-  }
 
   // lane constants inside a chunk buffer: this lane's 64-byte segment of group `warp` for token gid
   // of every token block (lanes without a token read the zero page), the scale tables, the x sums
@@ -765,6 +743,37 @@ decode_kernel(const MultiArgs ma) {
   for (int c0 = 0; c0 < nsteps; c0 += D)   // the register slot of a step is a compile-time constant
     unroll_slots([&](auto slot) { if (c0 + decltype(slot)::value < nsteps) do_step(c0 + decltype(slot)::value, slot); },
                  std::make_integer_sequence<int, D>{});
+
+  if (NBUF == 0) {
+    asm volatile("cp.async.wait_group 0;" ::: "memory");   // this warp's outlier entries have landed
+    __syncwarp();
+    // CSR outliers of the owned rows: lane = entry, every token per lane,
+    // one transposing reduction per row; the entries come from shared memory (those beyond cvcap, rare, from global
+    // memory), the activations from the staged copy
+    const uint16_t* xs16 = reinterpret_cast<const uint16_t*>(sm_x);
+    const uint32_t* mycv = sm_cv + warp * OWN * kCvCap;
+#pragma unroll
+    for (int rr = 0; rr < OWN; ++rr) {
+      const int jb = jr[rr], je = jr[rr + 1];
+      float v[TP];
+#pragma unroll
+      for (int m = 0; m < TP; ++m) v[m] = 0.f;
+      for (int e0 = lane; e0 < je - jb; e0 += 32) {
+        const unsigned e = e0 < kCvCap ? mycv[rr * kCvCap + e0] : __ldg(cvp + jb + e0);
+        const float wv = __half2float(__ushort_as_half((unsigned short)(e >> 16)));
+        const unsigned col = e & 0xFFFFu;
+        const int base = (int)(col >> 10) * buf_pieces;            // chunk = col / 1024
+        const int pc = (int)((col & 1023u) >> 3), sub = (int)(col & 7u);
+#pragma unroll
+        for (int m = 0; m < TP; ++m)
+          if (TP == 1 || m < M)
+            v[m] = fmaf(wv, act_to_float<BF16>(xs16[((base + xs_piece(pc, m)) << 3) + sub]), v[m]);
+      }
+      reduce_tokens<TP, 1>(v, lane);
+      constexpr int LPT = 32 / TP;   // lanes per token after the reduction
+      if ((lane & (LPT - 1)) == 0) sm_out[(OWN * warp + rr) * TP + lane / LPT] = v[0];
+    }
+  }
 
   // partial sums of the 8 warps: sm_red[warp][tile][nb][row][token]
 #pragma unroll
