@@ -130,9 +130,10 @@ gwq_status gwq_outliers_rows(const gwq_outliers* S, int32_t row0, int32_t row1, 
  * z = clip(rint(-lo / s), 0, 2^bits - 1); q = clip(rint(w / s) + z, 0, 2^bits - 1),
  * round-half-to-even; outliers get q = z.  A group with hi == lo gets s = 1, z = 0.
  *   bits: 3 or 4.  group: 16 (the value Section 3.2 names), 32, 64 or 128; K a multiple of 32 and of
- *      group.  The streaming path of gwq_linear takes group 128 (up to 32 tokens) and group 64 (up to
- *      16 tokens, K a multiple of 128), the tensor-core path 64 and 128; the other groups are served by
- *      the general kernel.
+ *      group.  Which kernel of gwq_linear serves a layer depends on its shape: with K a multiple of 128 (up to
+ *      65536) the streaming kernels take groups of 128 up to 32 tokens, of 64 up to 16, of 32 up to 4 and of 16
+ *      for one token; with K a multiple of 64 the tensor-core kernel takes every group size and token count;
+ *      anything else is served by a general (slow) kernel.
  *   W_f16: device, caller-owned, read only.
  *   S: from gwq_select_outliers with the same N, K; on success its ownership moves into
  *      *out (do not free it separately); on failure it stays with the caller.
@@ -144,14 +145,17 @@ gwq_status gwq_pack(const uint16_t* W_f16, gwq_outliers* S, int32_t N, int32_t K
 
 /* Forward product y = x (s (q - z) + S)^T (Section 3.2, Eq. "w", outliers in FP16).
  *   x: device [M, K], fp16 or bf16 (x_dtype).  y: device [M, N], y_dtype one of
- *   F16 / BF16 / F32.  Accumulation is FP32.  M >= 1; M <= 32 takes the bandwidth-bound
- *   streaming path, larger M the tensor-core path.
+ *   F16 / BF16 / F32.  Accumulation is FP32.  M >= 1.  Up to 32 tokens take a bandwidth-bound streaming
+ *   kernel (mma.sync; with a workspace, 17 to 32 fp16 tokens take a tcgen05 one: see gwq_linear_ws), more tokens
+ *   the tensor-core kernel (TMA, tcgen05, tensor memory), which with a workspace expands the weights once
+ *   from 2048 tokens on instead of once per token tile.
  *   Asynchronous on `stream`: the call only enqueues kernels.  It never allocates and never
  *   synchronises, so it may be captured into a CUDA graph from its first use.  Calls that share P
  *   must be enqueued on one stream (or otherwise ordered): with 9 to 32 tokens they share a small
  *   scratch buffer that gwq_pack created inside P.
- *   A call that needs more scratch than P holds (bf16 activations on the tensor-core path: an fp16
- *   copy of x) returns GWQ_ERR_WORKSPACE and does nothing: make it through gwq_linear_ws.
+ *   A call that cannot do without scratch (bf16 activations on the tensor-core path need an fp16 copy of
+ *   x) returns GWQ_ERR_WORKSPACE and does nothing: make it through gwq_linear_ws.  Calls that merely run
+ *   faster with scratch take their slower kernel here.
  * Errors: INVALID_ARG, UNSUPPORTED (x_dtype F32), WORKSPACE, CUDA (launch failure).      */
 gwq_status gwq_linear(const gwq_packed* P, const void* x, gwq_dtype x_dtype, int32_t M, void* y,
                       gwq_dtype y_dtype, void* stream);

@@ -216,26 +216,31 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmc, const __grid_constant__ C
         if (!ok) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint64_t dx0 = umma_desc(smem_u32(x_tile(s, 0))), dx1 = umma_desc(smem_u32(x_tile(s, 1)));
+        const uint64_t do0 = umma_desc(smem_u32(out_tiles + b * kOutTileBytes)),
+                       do1 = umma_desc(smem_u32(out_tiles + b * kOutTileBytes + kOutTileBytes / 2));
+        // MMAs into one accumulator depend on one another (a chain of K = 16 slices), so the step's chains are issued
+        // interleaved: the step accumulator(s) and the outlier accumulator advance together
 #pragma unroll
         for (int h = 0; h < AS; ++h) {
           const int q = j * AS + h, d = q & 1;
           if (q >= 2) ok = mbar_wait(d_empty(d), ((q >> 1) - 1) & 1, abort_flag, lim);
           if (!ok) break;
-          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-#pragma unroll
-          for (int k = 0; k < 8 / AS; ++k) {
-            const int kk = h * (8 / AS) + k;   // K = 16 slice of the step
-            umma_ts(tm_d(d), tm_a(b) + (unsigned)(8 * kk), (kk < 4 ? dx0 : dx1) + (uint64_t)(2 * (kk & 3)), idesc, k != 0);
-          }
-          umma_commit(d_full(d));
         }
         if (!ok) break;
-        const uint64_t do0 = umma_desc(smem_u32(out_tiles + b * kOutTileBytes)),
-                       do1 = umma_desc(smem_u32(out_tiles + b * kOutTileBytes + kOutTileBytes / 2));
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll
-        for (int kk = 0; kk < 8; ++kk)
-          umma_f16(tm_o(o), (kk < 4 ? do0 : do1) + (uint64_t)(2 * (kk & 3)), (kk < 4 ? dx0 : dx1) + (uint64_t)(2 * (kk & 3)),
-                   idesc, !(first && kk == 0));
+        for (int k = 0; k < 8 / AS; ++k) {
+#pragma unroll
+          for (int h = 0; h < AS; ++h) {
+            const int kk = h * (8 / AS) + k;   // K = 16 slice of the step
+            umma_ts(tm_d((j * AS + h) & 1), tm_a(b) + (unsigned)(8 * kk), (kk < 4 ? dx0 : dx1) + (uint64_t)(2 * (kk & 3)), idesc,
+                    k != 0);
+            umma_f16(tm_o(o), (kk < 4 ? do0 : do1) + (uint64_t)(2 * (kk & 3)), (kk < 4 ? dx0 : dx1) + (uint64_t)(2 * (kk & 3)),
+                     idesc, !(first && k == 0 && h == 0));
+          }
+        }
+#pragma unroll
+        for (int h = 0; h < AS; ++h) umma_commit(d_full((j * AS + h) & 1));
         umma_commit(a_empty(b));
         umma_commit(empty(s));
         if (last) {
@@ -311,12 +316,19 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmc, const __grid_constant__ C
     for (int m = 0; m < TOK; ++m) yacc[m] = 0.f;
     int piece = 0;
     bool head = true;   // the current piece contains the first step of this CTA
-    unsigned sz_next[AS];
-    if (nsteps > 0) {
-      const int row0 = (int)(it0 / G) * kRows + r, grp0 = (int)(it0 % G);
+    // scale and zero-point words of the next three steps: requested that far ahead, so that no step waits for memory
+    constexpr int kAhead = 3;
+    unsigned sz_ring[kAhead][AS];
+    auto load_sz = [&](int j, unsigned (&dst)[AS]) {
+      if (j < nsteps) {
+        const long long itn = it0 + j;
+        const int rown = (int)(itn / G) * kRows + r, grpn = (int)(itn % G);
 #pragma unroll
-      for (int h = 0; h < AS; ++h) sz_next[h] = __ldg(p.szt + (size_t)(grp0 * AS + h) * p.N + (row0 < p.N ? row0 : p.N - 1));
-    }
+        for (int h = 0; h < AS; ++h) dst[h] = __ldg(p.szt + (size_t)(grpn * AS + h) * p.N + (rown < p.N ? rown : p.N - 1));
+      }
+    };
+#pragma unroll
+    for (int a = 0; a < kAhead; ++a) load_sz(a, sz_ring[a]);
     asm volatile("griddepcontrol.wait;" ::: "memory");   // y and the workspace may still be in use by the previous kernel
     for (int j = 0; j < nsteps && ok; ++j) {
       const long long it = it0 + j;
@@ -326,14 +338,12 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmc, const __grid_constant__ C
       const int xq = j % kXs;
       unsigned sz[AS];
 #pragma unroll
-      for (int h = 0; h < AS; ++h) sz[h] = sz_next[h];
-      if (j + 1 < nsteps) {   // scale and zero-point of the next step: requested a step ahead
-        const long long itn = it + 1;
-        const int rown = (int)(itn / G) * kRows + r, grpn = (int)(itn % G);
+      for (int h = 0; h < AS; ++h) sz[h] = sz_ring[0][h];
 #pragma unroll
-        for (int h = 0; h < AS; ++h)
-          sz_next[h] = __ldg(p.szt + (size_t)(grpn * AS + h) * p.N + (rown < p.N ? rown : p.N - 1));
-      }
+      for (int a = 0; a + 1 < kAhead; ++a)
+#pragma unroll
+        for (int h = 0; h < AS; ++h) sz_ring[a][h] = sz_ring[a + 1][h];
+      load_sz(j + kAhead, sz_ring[kAhead - 1]);
       ok = mbar_wait_warp(xs_full(xq), (j / kXs) & 1, abort_flag, lim);
       if (!ok) break;
 #pragma unroll
@@ -458,10 +468,18 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmc, const __grid_constant__ C
       const unsigned r = (v >> 23) & 127u, c = (v >> 16) & 127u;
       return (c >> 6) * (unsigned)(kOutTileBytes / 2) + r * 128u + ((((c & 63u) >> 3) ^ (r & 7u)) << 4) + ((c & 7u) << 1);
     };
-    auto fetch = [&](int j) {   // extents and first entries of the block of step j (requested a step ahead)
+    int n0 = 0, n1 = 0;                        // extents of the block after next of this set (requested two steps ahead)
+    auto fetch_extents = [&](int j) {
       if (j < nsteps) {
-        e0 = __ldg(p.ob_ptr + it0 + j);
-        e1 = __ldg(p.ob_ptr + it0 + j + 1);
+        n0 = __ldg(p.ob_ptr + it0 + j);
+        n1 = __ldg(p.ob_ptr + it0 + j + 1);
+      }
+    };
+    auto fetch = [&](int j) {   // first entries of the block of step j, whose extents are in (n0, n1) by now
+      e0 = e1 = 0;
+      if (j < nsteps) {
+        e0 = n0;
+        e1 = n1;
 #pragma unroll
         for (int i = 0; i < kHeld; ++i) held[i] = e0 + lane + 32 * i < e1 ? __ldg(p.ob + e0 + lane + 32 * i) : 0xFFFFFFFFu;
       }
@@ -469,7 +487,9 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmc, const __grid_constant__ C
     unsigned prev[kHeld];
 #pragma unroll
     for (int i = 0; i < kHeld; ++i) prev[i] = 0xFFFFFFFFu;
+    fetch_extents(set);
     fetch(set);
+    fetch_extents(set + kSets);
     for (int j = set; j < nsteps && ok; j += kSets) {
       if (j >= kSets) ok = mbar_wait_warp(a_empty(set), ((j / kSets) - 1) & 1, abort_flag, lim);   // MMAs of two steps ago done
       if (!ok) break;
@@ -494,6 +514,7 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmc, const __grid_constant__ C
       __syncwarp();
       if (lane == 0) mbar_arrive(a_full(set));
       fetch(j + kSets);   // behind the proxy fence, which would have waited for these loads
+      fetch_extents(j + 2 * kSets);
     }
   }
   if (!ok) {
