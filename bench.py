@@ -211,6 +211,43 @@ def time_region(torch, fn, iters: int) -> float:
     torch.cuda.synchronize()
     return e0.elapsed_time(e1) / iters
 
+class ReadProbe:
+    """The read-only launch that gives the per-layer floor: the benchmark's own small CUDA library
+    (paper_2411_00850_b200/bench_aid), loaded here and given the public arrays of a packed layer."""
+
+    def __init__(self, torch):
+        import ctypes
+        path = os.path.join(ROOT, "paper_2411_00850_b200", "bench_aid", "libbench_read_probe.so")
+        if not os.path.exists(path):
+            raise RuntimeError(f"{path} is missing: build it with `python -m paper_2411_00850_b200.build`")
+        self.C = ctypes
+        self.lib = ctypes.CDLL(path)
+        self.lib.bench_read_probe.restype = ctypes.c_longlong
+        self.lib.bench_read_probe.argtypes = [ctypes.POINTER(ctypes.c_void_p), ctypes.POINTER(ctypes.c_ulonglong),
+                                              ctypes.c_int, ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p]
+        self.torch = torch
+        self.sink = torch.zeros(4, dtype=torch.int32, device="cuda")
+        self.blocks = 4 * torch.cuda.get_device_properties(0).multi_processor_count
+
+    def arrays(self, P):
+        """(pointer, bytes) of what a one-token product reads of P: codes, scales, zero-points, row pointers and
+        4 bytes per outlier (the column indices stand for the 4-byte entries the kernels stream)."""
+        h = P._h.contents
+        S = h.S.contents
+        groups = h.N * (h.K // h.group)
+        return [(h.codes, h.N * (h.K // 32) * h.bits * 4), (h.scales, groups * 2), (h.zeros, groups),
+                (S.row_ptr, (h.N + 1) * 4), (S.col_idx, S.nnz * 4)]
+
+    def launch(self, P):
+        arr = [(p, b) for (p, b) in self.arrays(P) if p and b >= 16]
+        base = (self.C.c_void_p * len(arr))(*[p for p, _ in arr])
+        size = (self.C.c_ulonglong * len(arr))(*[b for _, b in arr])
+        n = self.lib.bench_read_probe(base, size, len(arr), self.sink.data_ptr(), self.blocks,
+                                      self.torch.cuda.current_stream().cuda_stream)
+        if n < 0:
+            raise RuntimeError("bench_read_probe failed")
+        return int(n)
+
 
 def capture(torch, fn):
     """Capture fn() into a CUDA graph (after one eager run) and return a replay callable."""
@@ -407,6 +444,7 @@ def bench_decode_detail(torch, gwq, layers, xs, ys, iters, hbm_peak):
     # L2 scrub: READ 256 MB, so that the cache is left full of clean lines (a written scrub would leave dirty
     # lines whose write-back competes with the timed reads)
     scrub = torch.zeros(64 * 1024 * 1024, dtype=torch.int32, device=xs[(0, 1)].device)
+    read_probe = ReadProbe(torch)
 
     def scrub_l2():
         return int(scrub.sum().item())
@@ -419,7 +457,7 @@ def bench_decode_detail(torch, gwq, layers, xs, ys, iters, hbm_peak):
 
             def probe():
                 for (li, r) in members:
-                    gwq.gwq_read_probe(layers[li]["packed"][bits][r])
+                    read_probe.launch(layers[li]["packed"][bits][r])
             replay_probe = capture(torch, probe)
             floor_ms = None
             for _ in range(iters):

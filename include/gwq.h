@@ -205,13 +205,6 @@ gwq_status gwq_gradient_mean(const float* const* G_list, int32_t count, int64_t 
 gwq_status gwq_quality(const uint16_t* W_f16, const float* G_f32, const gwq_packed* P, double* sq_err,
                        double* first_order, void* stream);
 
-/* Measurement aid, no counterpart in the paper: one launch that reads, and only reads, the arrays a
- * one-token gwq_linear reads of P (packed codes, scales, zero-points, CSR row pointers, outlier entries).
- * Its duration is the floor for any forward product that is one kernel launch per layer; the benchmark
- * prints it beside the decode timings.  *bytes_read (host, may be NULL) receives the bytes it reads.
- * Asynchronous on `stream`.  Errors: INVALID_ARG, UNSUPPORTED (K > 65536), CUDA.                       */
-gwq_status gwq_read_probe(const gwq_packed* P, int64_t* bytes_read, void* stream);
-
 /* Same product with HOST buffers: copies x_host [M,K] to a staging buffer kept inside P,
  * runs gwq_linear, copies y back into y_host [M,N] and synchronises `stream`.
  * For best copy speed the host buffers should be page-locked.  The staging buffers (and the scratch

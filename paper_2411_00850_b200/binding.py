@@ -25,7 +25,7 @@ STATUS_NAMES = {
 }
 EXPORTS = ("gwq_select_outliers", "gwq_select_outliers_static", "gwq_outliers_rows", "gwq_pack", "gwq_linear", "gwq_linear_ws",
            "gwq_linear_workspace_bytes", "gwq_linear_multi",
-           "gwq_gradient_mean", "gwq_quality", "gwq_read_probe", "gwq_linear_host", "gwq_linear_host_async", "gwq_device_status", "gwq_set_wait_limit", "gwq_free", "gwq_status_string")
+           "gwq_gradient_mean", "gwq_quality", "gwq_linear_host", "gwq_linear_host_async", "gwq_device_status", "gwq_set_wait_limit", "gwq_free", "gwq_status_string")
 GWQ_MULTI_MAX = 4
 
 
@@ -87,8 +87,6 @@ def load_library(path: str = LIB_PATH) -> C.CDLL:
     lib.gwq_quality.restype = C.c_int
     lib.gwq_quality.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(gwq_packed), C.POINTER(C.c_double),
                                 C.POINTER(C.c_double), C.c_void_p]
-    lib.gwq_read_probe.restype = C.c_int
-    lib.gwq_read_probe.argtypes = [C.POINTER(gwq_packed), C.POINTER(C.c_int64), C.c_void_p]
     lib.gwq_linear_host.restype = C.c_int
     lib.gwq_linear_host.argtypes = lib.gwq_linear.argtypes
     lib.gwq_linear_host_async.restype = C.c_int
@@ -396,15 +394,6 @@ def gwq_quality(W: torch.Tensor, G: torch.Tensor, P: Packed):
         st = load_library().gwq_quality(W.data_ptr(), G.data_ptr(), P._h, C.byref(a), C.byref(b), _stream_ptr())
     _check(st, "gwq_quality")
     return float(a.value), float(b.value)
-
-
-def gwq_read_probe(P: Packed) -> int:
-    """Launch the read-only probe on P (asynchronous on the current stream); returns the bytes it reads."""
-    n = C.c_int64(0)
-    with torch.cuda.device(P.device):
-        st = load_library().gwq_read_probe(P._h, C.byref(n), _stream_ptr())
-    _check(st, "gwq_read_probe")
-    return int(n.value)
 
 
 def gwq_linear_host(P: Packed, x_host: torch.Tensor, y_host: torch.Tensor) -> torch.Tensor:

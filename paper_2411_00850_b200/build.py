@@ -13,8 +13,10 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libgwq.so")
+AID_SRC = os.path.join(HERE, "bench_aid", "read_probe.cu")    # the benchmark's read-only launch, a library of its own
+AID_LIB = os.path.join(HERE, "bench_aid", "libbench_read_probe.so")
 SOURCES = ("decode_w4_f16.cu", "decode_w4_bf16.cu", "decode_w3_f16.cu", "decode_w3_bf16.cu", "select.cu",
-           "select_static.cu", "pack.cu", "linear_simt.cu", "linear_decode.cu", "linear_skinny.cu", "linear_prefill.cu", "probe.cu",
+           "select_static.cu", "pack.cu", "linear_simt.cu", "linear_decode.cu", "linear_skinny.cu", "linear_prefill.cu",
            "quality.cu", "gradmean.cu", "api.cu")
 NVCC_FLAGS = (
     "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
@@ -44,7 +46,16 @@ def _stale(target: str, deps) -> bool:
 
 def needs_build() -> bool:
     deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)] + _headers()
-    return _stale(LIB, deps)
+    return _stale(LIB, deps) or _stale(AID_LIB, [AID_SRC])
+
+
+def _build_aid(force: bool) -> None:
+    if not force and not _stale(AID_LIB, [AID_SRC]):
+        return
+    res = subprocess.run([_nvcc(), *NVCC_FLAGS, "-shared", AID_SRC, "-o", AID_LIB, "-lcudart"],
+                         capture_output=True, text=True)
+    if res.returncode != 0:
+        raise RuntimeError("nvcc failed on read_probe.cu:\n" + res.stdout + res.stderr)
 
 
 def _compile(src: str, force: bool, verbose: bool) -> str:
@@ -66,6 +77,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if not force and not needs_build():
         return LIB
     os.makedirs(OBJ, exist_ok=True)
+    _build_aid(force)
     with ThreadPoolExecutor(max_workers=min(len(SOURCES), os.cpu_count() or 4)) as pool:
         logs = list(pool.map(lambda s: _compile(s, force, verbose), SOURCES))
     if verbose:
