@@ -481,9 +481,376 @@ __global__ void __launch_bounds__(256) expand_outliers_kernel(const int32_t* __r
   }
 }
 
+// ---------------------------------------------------------------------------------------------------------------
+// Contraction of the two-phase path on pairs of CTAs (a cluster of two SMs, tcgen05 cta_group::2): one MMA spans
+// 256 weight rows x 256 tokens, each CTA of the pair holding its 128 weight rows (A) and its 128 of the 256 token
+// rows (B) of a k-block in its own shared memory: 32 KB per k-block and SM instead of the 48 KB of a 128 x 256 tile,
+// which is what the contraction is bound by (the operands come out of L2).  Each CTA keeps the accumulators of
+// its 128 rows in its own tensor memory (two of 256 columns, so the epilogue of a tile runs under the next tile).
+//   warp 0, one thread : TMA (no multicast) of the CTA's two half tiles per k-block; the bytes of both CTAs are
+//                        counted by the `full` barrier of the pair's first CTA, which arms it;
+//   warp 1, one thread : in the pair's first CTA only: tcgen05.mma cta_group::2, and tcgen05.commit to both CTAs'
+//                        `empty` / `acc_full` barriers; in both CTAs the warp owns the tensor-memory allocation;
+//   warps 2..5         : epilogue, one thread per weight row of the CTA: tcgen05.ld, token scale, conversion into a
+//                        shared-memory tile of 32 tokens x 128 features that one thread hands to a TMA store (whole
+//                        256-byte rows of y instead of 2 bytes per thread); both CTAs' epilogue warps tell the first
+//                        CTA when an accumulator is free again.
+// Every wait is bounded (see the fused kernel); the two CTAs leave together through a cluster barrier.
+constexpr int kPairThreads = 32 * 6;
+constexpr int kPairStages = 6;
+constexpr int kPairTok = 256;                 // tokens of a pair's tile (UMMA N), 128 loaded by each CTA
+constexpr int kPairStageBytes = 2 * kTileN * kBlockK * 2;   // A half and B half of a k-block: 32 KB
+constexpr int kOutStageBytes = 32 * kTileN * 4;             // 32 tokens x 128 features, up to 4 bytes each
+
+__device__ __forceinline__ unsigned cluster_ctarank() {
+  unsigned r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// shared::cluster address, in the pair's first CTA, of the object at this CTA's shared address `addr`
+__device__ __forceinline__ unsigned in_first_cta(unsigned addr) {
+  unsigned r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, 0;" : "=r"(r) : "r"(addr));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(unsigned cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// TMA tile load of a CTA pair: the data lands in this CTA's shared memory, the bytes are counted by `bar_cluster`
+__device__ __forceinline__ void tma_load_2d_pair(unsigned dst, const CUtensorMap* map, int c0, int c1, unsigned bar_cluster) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar_cluster)
+      : "memory");
+}
+__device__ __forceinline__ void umma_f16_pair(unsigned tmem_d, uint64_t da, uint64_t db, unsigned idesc, unsigned accumulate) {
+  asm volatile(
+      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+      " tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n}\n"
+      ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// arrives, when the MMAs issued so far have completed, on this CTA's barrier
+__device__ __forceinline__ void umma_commit_pair_local(unsigned bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// arrives, when the MMAs issued so far have completed, on the barrier at this shared address in both CTAs of the pair
+__device__ __forceinline__ void umma_commit_pair(unsigned bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"((unsigned short)3)
+               : "memory");
+}
+
+// Order of a pair's tiles: bands of kBandTiles weight tiles, inside a band the weight tile runs fastest and the
+// token tile slowest.  The pairs work on neighbouring tiles at the same time, so what they read together is one
+// band of the weights (which stays in L2 for the whole band) and a few token tiles, instead of all of the weights
+// for every group of token tiles.
+#ifndef GWQ_TUNE_BAND
+#define GWQ_TUNE_BAND 8
+#endif
+constexpr int kBandTiles = GWQ_TUNE_BAND;
+__device__ __forceinline__ void pair_tile(int t, int ntn, int ntm, int& tn, int& tm) {
+  const int per_band = kBandTiles * ntm;
+  const int band = t / per_band, i = t - band * per_band;
+  const int width = min(kBandTiles, ntn - band * kBandTiles);   // the last band may be narrower
+  tm = i / width;
+  tn = band * kBandTiles + (i - tm * width);
+}
+
+struct PairArgs {
+  void* y;
+  gwq_dtype yd;
+  int32_t* status;
+  const float* tok_scale;   // per token 2^e, or null
+  int N, K, M;
+  int tma_store;            // y is written through tmy (its rows start on 16-byte boundaries), else by plain stores
+  long long wait_cycles;
+};
+
+// tmx: x16 [M][K] with boxes of 64 columns x 128 rows; tmw: expanded weights [N][K], same boxes.
+// tmy: y [M][N] with boxes of 128 output features x 32 tokens.
+// ntn: tiles of 256 weight rows; ntiles: all tiles (order: pair_tile); pairs: clusters of the launch.
+__global__ void __launch_bounds__(kPairThreads, 1)
+pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUtensorMap tmw,
+            const __grid_constant__ CUtensorMap tmy, const PairArgs p, const int ntn, const int ntiles, const int pairs) {
+  constexpr int kHalfBytes = kTileN * kBlockK * 2;   // 16 KB: 128 rows x 128 bytes
+  extern __shared__ unsigned char smem_dyn[];
+  unsigned char* tiles =
+      reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
+  __shared__ __align__(8) unsigned long long bars[2 * kPairStages + 5];
+  __shared__ unsigned tmem_base_s;
+  __shared__ int abort_s;
+  volatile int* abort_flag = &abort_s;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const unsigned rank = cluster_ctarank();       // 0: the pair's first CTA, which issues the MMAs
+  const int pair = blockIdx.x >> 1;
+  const int nkb = p.K / kBlockK;
+  const unsigned bar0 = smem_u32(bars);
+  auto full = [&](int s) { return bar0 + 8u * s; };                       // first CTA's: bytes of both CTAs
+  auto empty = [&](int s) { return bar0 + 8u * (kPairStages + s); };      // each CTA's own
+  auto acc_full = [&](int a) { return bar0 + 8u * (2 * kPairStages + a); };      // each CTA's own
+  auto acc_empty = [&](int a) { return bar0 + 8u * (2 * kPairStages + 2 + a); }; // first CTA's: both epilogues
+  const unsigned drain_bar = bar0 + 8u * (2 * kPairStages + 4);
+  const long long lim = p.wait_cycles;
+  auto a_tile = [&](int s) { return tiles + (size_t)s * kPairStageBytes; };
+  auto b_tile = [&](int s) { return tiles + (size_t)s * kPairStageBytes + kHalfBytes; };
+  unsigned char* out_stage = tiles + (size_t)kPairStages * kPairStageBytes;   // two tiles of 32 tokens x 128 features
+  const int my_tiles = pair < ntiles ? (ntiles - 1 - pair) / pairs + 1 : 0;
+  const int ntm = ntiles / ntn;   // token tiles
+
+  if (tid == 0) {
+    abort_s = 0;
+    for (int s = 0; s < kPairStages; ++s) {
+      mbar_init(full(s), 1);
+      mbar_init(empty(s), 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(acc_full(a), 1);
+      mbar_init(acc_empty(a), 2 * kEpilogueWarps);
+    }
+    mbar_init(drain_bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {   // tensor memory of both CTAs: two accumulators of 256 columns x 128 lanes each
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(512)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  cluster_sync_all();   // both CTAs' barriers exist before either signals the other
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const unsigned tmem_acc = tmem_base_s;
+  bool ok = *reinterpret_cast<volatile int32_t*>(p.status) == 0;   // an earlier CTA gave up: do no work
+  int issued = 0;   // k-block copies started (producer thread only), counted over all tiles
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ this CTA's halves of the operand tiles by TMA
+    if (lane == 0) {
+      for (int ti = 0; ti < my_tiles && ok; ++ti) {
+        int tn, tm;
+        pair_tile(pair + ti * pairs, ntn, ntm, tn, tm);
+        const int n0 = tn * (2 * kTileN) + (int)rank * kTileN;
+        const int m0 = tm * kPairTok + (int)rank * (kPairTok / 2);
+        for (int kb = 0; kb < nkb && ok; ++kb) {
+          const int it = ti * nkb + kb, s = it % kPairStages, round = it / kPairStages;
+          if (round > 0) ok = mbar_wait(empty(s), (round - 1) & 1, abort_flag, lim);
+          if (!ok) break;
+          if (rank == 0) mbar_expect_tx(full(s), 2 * kPairStageBytes);
+          const unsigned fb = in_first_cta(full(s));
+          tma_load_2d_pair(smem_u32(a_tile(s)), &tmw, kb * kBlockK, n0, fb);
+          tma_load_2d_pair(smem_u32(b_tile(s)), &tmx, kb * kBlockK, m0, fb);
+          issued = it + 1;
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issue (first CTA of the pair)
+    if (lane == 0 && rank == 0) {
+      // instruction descriptor: FP32 accumulate, A and B fp16, K-major, N = 256, M = 256 (128 rows per CTA)
+      const unsigned idesc = (1u << 4) | ((unsigned)(kPairTok >> 3) << 17) | ((unsigned)((2 * kTileN) >> 4) << 24);
+      for (int ti = 0; ti < my_tiles && ok; ++ti) {
+        const int a = ti & 1;
+        if (ti >= 2) ok = mbar_wait(acc_empty(a), ((ti >> 1) - 1) & 1, abort_flag, lim);   // drained by both epilogues
+        if (!ok) break;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const unsigned acc = tmem_acc + (unsigned)(a * kPairTok);
+        for (int kb = 0; kb < nkb && ok; ++kb) {
+          const int it = ti * nkb + kb, s = it % kPairStages, round = it / kPairStages;
+          ok = mbar_wait(full(s), round & 1, abort_flag, lim);
+          if (!ok) break;
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          const uint64_t da = umma_desc(smem_u32(a_tile(s))), db = umma_desc(smem_u32(b_tile(s)));
+#pragma unroll
+          for (int k = 0; k < kBlockK / 16; ++k)   // 32 bytes further along K inside the swizzle atom
+            umma_f16_pair(acc, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (kb | k) != 0);
+          umma_commit_pair(empty(s));
+        }
+        if (ok) umma_commit_pair(acc_full(a));
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue: one thread per weight row of the CTA
+    const int quad = warp & 3;                 // tensor-memory lane quarter this warp may access
+    const int r = quad * 32 + lane;
+    int chunk = 0;                             // chunks handed to the TMA store so far
+    for (int ti = 0; ti < my_tiles && ok; ++ti) {
+      int tn, tm;
+      pair_tile(pair + ti * pairs, ntn, ntm, tn, tm);
+      const int row = tn * (2 * kTileN) + (int)rank * kTileN + r, m0 = tm * kPairTok;
+      const bool live = row < p.N;
+      const int a = ti & 1;
+      ok = mbar_wait_warp(acc_full(a), (ti >> 1) & 1, abort_flag, lim);
+      {   // one verdict for the four epilogue warps: they meet at barriers inside the tile
+        unsigned all;
+        asm volatile("{\n .reg .pred q, r;\n setp.ne.b32 q, %1, 0;\n bar.red.and.pred r, 1, 128, q;\n selp.b32 %0, 1, 0, r;\n}\n"
+                     : "=r"(all) : "r"((unsigned)ok) : "memory");
+        ok = all != 0;
+      }
+      if (!ok) break;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+#pragma unroll 1
+      for (int c0 = 0; c0 < kPairTok; c0 += 32) {
+        if (m0 + c0 >= p.M) break;             // warp-uniform
+        unsigned v[32];
+        tmem_ld32(tmem_acc + ((unsigned)(quad * 32) << 16) + (unsigned)(a * kPairTok + c0), v);
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        if (p.tma_store) {
+          // the chunk goes through a shared-memory tile [32 tokens][128 features] (two of them, used in turn)
+          unsigned char* st = out_stage + (chunk & 1) * kOutStageBytes;
+          if (chunk >= 2) {   // the store that read this tile two chunks ago has finished reading it
+            if (warp == 2 && lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+          }
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            float f = __uint_as_float(v[i]);
+            if (p.tok_scale) f *= __ldg(p.tok_scale + min(m0 + c0 + i, p.M - 1));
+            if (p.yd == GWQ_F32) reinterpret_cast<float*>(st)[i * kTileN + r] = f;
+            else if (p.yd == GWQ_F16) reinterpret_cast<__half*>(st)[i * kTileN + r] = __float2half_rn(f);
+            else reinterpret_cast<__nv_bfloat16*>(st)[i * kTileN + r] = __float2bfloat16_rn(f);
+          }
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to the TMA
+          asm volatile("bar.sync 1, 128;" ::: "memory");
+          if (warp == 2 && lane == 0) {   // rows past N and tokens past M are clipped by the copy
+            asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+                         ::"l"(&tmy), "r"(tn * (2 * kTileN) + (int)rank * kTileN), "r"(m0 + c0), "r"(smem_u32(st))
+                         : "memory");
+            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+          }
+          ++chunk;
+        } else if (live) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            const int m = m0 + c0 + i;
+            if (m < p.M) {
+              float f = __uint_as_float(v[i]);
+              if (p.tok_scale) f *= __ldg(p.tok_scale + m);
+              const size_t idx = (size_t)m * p.N + row;
+              if (p.yd == GWQ_F32) reinterpret_cast<float*>(p.y)[idx] = f;
+              else if (p.yd == GWQ_F16) reinterpret_cast<__half*>(p.y)[idx] = __float2half_rn(f);
+              else reinterpret_cast<__nv_bfloat16*>(p.y)[idx] = __float2bfloat16_rn(f);
+            }
+          }
+        }
+      }
+      // the accumulator may be overwritten by the tile after next: both CTAs tell the first one
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(in_first_cta(acc_empty(a)));
+    }
+    // the stores still in flight read this CTA's shared memory
+    if (warp == 2 && lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+  }
+  if (!ok) {
+    *abort_flag = 1;
+    atomicExch(p.status, (int32_t)GWQ_ERR_TIMEOUT);
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (abort_s) {
+    // give-up path.  Bulk copies that were issued must land before the shared memory is given back; their bytes are
+    // counted in the first CTA, so this CTA waits a fixed time that is long against a copy instead (bounded).
+    if (warp == 0 && lane == 0 && issued > 0) {
+      const long long t0 = clock64();
+      while (clock64() - t0 < 200000) {}
+    }
+    // MMAs that were issued may still read both CTAs' stages and write both tensor memories: one more commit arrives
+    // when all of them have completed; wait (bounded) for it before the pair leaves
+    if (warp == 1 && lane == 0 && rank == 0) {
+      int zero = 0;
+      umma_commit_pair_local(drain_bar);
+      (void)mbar_wait(drain_bar, 0, &zero, kSpinCycles);
+    }
+  }
+  __syncthreads();
+  cluster_sync_all();   // neither CTA frees its tensor memory, or exits, while the other may still signal or write it
+  if (warp == 1) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(512) : "memory");
+  }
+}
+
+// Launch of the pair kernel on the expanded weights w16 [N][K] and fp16 activations x [M][K].
+gwq_status launch_pairs(const gwq_packed* P, const void* x, const float* tok_scale, const void* w16, int M, void* y,
+                        gwq_dtype yd, cudaStream_t stream) {
+  const gwq_priv* pv = static_cast<const gwq_priv*>(P->priv);
+  EncodeTiledFn enc = encode_fn();
+  if (!enc) return GWQ_ERR_CUDA;
+  CUtensorMap tmx, tmw;
+  const cuuint32_t estr[2] = {1, 1};
+  const cuuint32_t box[2] = {(cuuint32_t)kBlockK, (cuuint32_t)kTileN};
+  {
+    const cuuint64_t dims[2] = {(cuuint64_t)P->K, (cuuint64_t)M};
+    const cuuint64_t strides[1] = {(cuuint64_t)P->K * 2};
+    if (enc(&tmx, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(x), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return GWQ_ERR_CUDA;
+  }
+  {
+    const cuuint64_t dims[2] = {(cuuint64_t)P->K, (cuuint64_t)P->N};
+    const cuuint64_t strides[1] = {(cuuint64_t)P->K * 2};
+    if (enc(&tmw, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(w16), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return GWQ_ERR_CUDA;
+  }
+  const size_t esz = yd == GWQ_F32 ? 4 : 2;
+  const int tma_store = ((size_t)P->N * esz) % 16 == 0 ? 1 : 0;   // y itself is 16-byte aligned (checked at the entry point)
+  CUtensorMap tmy = tmx;
+  if (tma_store) {
+    const cuuint64_t dims[2] = {(cuuint64_t)P->N, (cuuint64_t)M};
+    const cuuint64_t strides[1] = {(cuuint64_t)P->N * esz};
+    const cuuint32_t obox[2] = {(cuuint32_t)kTileN, 32};
+    const CUtensorMapDataType dt = yd == GWQ_F32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
+                                                 : (yd == GWQ_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16);
+    if (enc(&tmy, dt, 2, y, dims, strides, obox, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+            CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return GWQ_ERR_CUDA;
+  }
+  const size_t smem = (size_t)kPairStages * kPairStageBytes + 2 * kOutStageBytes + 1024;
+  if (cudaFuncSetAttribute(pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return GWQ_ERR_CUDA;
+  PairArgs a;
+  a.y = y; a.yd = yd; a.status = pv->dev_status; a.tok_scale = tok_scale; a.N = P->N; a.K = P->K; a.M = M;
+  a.tma_store = tma_store;
+  a.wait_cycles = pv->wait_cycles;
+  const int ntn = (P->N + 2 * kTileN - 1) / (2 * kTileN), ntiles = ntn * ((M + kPairTok - 1) / kPairTok);
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.blockDim = dim3(kPairThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  // persistent: as many pairs as the device holds at once (pairs sit inside one GPC, so this may be fewer than SMs / 2)
+  cfg.gridDim = dim3(2u * (unsigned)(pv->sm_count / 2));
+  int resident = 0;
+  if (cudaOccupancyMaxActiveClusters(&resident, pair_kernel, &cfg) != cudaSuccess || resident < 1) {
+    (void)cudaGetLastError();
+    return GWQ_ERR_UNSUPPORTED;
+  }
+  int pairs = resident < pv->sm_count / 2 ? resident : pv->sm_count / 2;
+  if (pairs > ntiles) pairs = ntiles;
+  cfg.gridDim = dim3(2u * (unsigned)pairs);
+  if (cudaLaunchKernelEx(&cfg, pair_kernel, tmx, tmw, tmy, a, ntn, ntiles, pairs) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return GWQ_ERR_CUDA;
+  }
+  return GWQ_OK;
+}
+
 template <int BITS, int TOK, bool EXP, int GPK = 1>
-gwq_status launch(const gwq_packed* P, const void* x, const float* tok_scale, const void* w16, int M, void* y, gwq_dtype yd,
-                  cudaStream_t stream) {
+gwq_status launch(const gwq_packed* P, const void* x, const float* tok_scale, const void* w16, int M, void* y,
+                  gwq_dtype yd, cudaStream_t stream) {
   constexpr bool BF16 = false;   // operands are always fp16 here (see the file header)
   const gwq_priv* pv = static_cast<const gwq_priv*>(P->priv);
   EncodeTiledFn enc = encode_fn();
@@ -543,12 +910,21 @@ gwq_status launch_tok(const gwq_packed* P, const void* x, const float* tok_scale
   return launch<BITS, 256, false>(P, x, tok_scale, nullptr, M, y, yd, stream);
 }
 
-// Tokens from which the weights are expanded once instead of once per token tile.  The expansion costs a pass of
-// 2.5 bytes per weight (about 40 us for 11008 x 4096) and the two-operand contraction is faster per tile than the
-// fused kernel only with 256-token tiles (128-token tiles ask L2 for 114 bytes per clock and SM); measured, bf16
-// activations, 4 bit: 835 against 731 TFLOP/s at 2048 tokens and 1044 against 895 at 8192 on 11008 x 4096, 796
-// against 693 and 1105 against 906 on 4096 x 11008; at 512 and 1024 tokens the fused kernel is level or ahead.
-constexpr int kExpandMinTokens = 2048;
+// When the weights are expanded once instead of once per token tile.  The expansion is a pass of 2.5 bytes per weight
+// (about 40 us for 45 M weights, 210 us for 235 M) and the contraction on CTA pairs then runs at 1000 to 1600 TFLOP/s
+// where the fused kernel, whose tiles each expand their weights again, reaches 250 to 770.  Measured, bf16 activations,
+// 4 bit, fused against two-phase: 1024 tokens: 156 / 131 us on 11008 x 4096, 145 / 122 on 4096 x 11008, 199 / 168 on
+// 8192 x 8192, 632 / 565 on 28672 x 8192; 512 tokens: 114 / 104, 144 / 115 and 73 / 62 (4096 x 4096), but 117 / 125 on
+// 8192 x 8192 and 374 / 408 on 28672 x 8192; 384 tokens: 101 / 101 and 144 / 115; 256 tokens: 74 / 81.
+constexpr int kExpandMinTokens = 1024;                       // every layer
+constexpr int kExpandMinTokensSmall = 384;                   // layers of up to kExpandSmallWeights weights
+constexpr long long kExpandSmallWeights = 48LL * 1000 * 1000;
+static bool wants_expansion(const gwq_packed* P, int M) {
+#ifdef GWQ_TUNE_EXPAND_MIN
+  return M >= GWQ_TUNE_EXPAND_MIN;
+#endif
+  return M >= kExpandMinTokens || (M >= kExpandMinTokensSmall && (long long)P->N * P->K <= kExpandSmallWeights);
+}
 
 // Expanded weights: the expansion, the outliers over it, then the contraction with token tiles of 256.
 gwq_status launch_expanded(const gwq_packed* P, const void* x, const float* tok_scale, uint16_t* w16, int M, void* y,
@@ -561,13 +937,15 @@ gwq_status launch_expanded(const gwq_packed* P, const void* x, const float* tok_
     expand_kernel<3><<<(unsigned)((runs + 255) / 256), 256, 0, stream>>>(P->codes, pv->sz_t, w16, P->N, P->K, P->group);
   expand_outliers_kernel<<<(P->N + 7) / 8, 256, 0, stream>>>(P->S->row_ptr, pv->cv, w16, P->N, P->K);
   if (cudaGetLastError() != cudaSuccess) return GWQ_ERR_CUDA;
+  const gwq_status st = launch_pairs(P, x, tok_scale, w16, M, y, yd, stream);
+  if (st != GWQ_ERR_UNSUPPORTED) return st;   // no room for a cluster of two: one CTA per tile
   return launch<4, 256, true>(P, x, tok_scale, w16, M, y, yd, stream);
 }
 
 }  // namespace
 
 // Scratch of the tensor-core path: bf16 activations need an fp16 copy of x and one scale per token; from
-// kExpandMinTokens tokens on, the fp16 expansion of the weights [N, K] follows.
+// the token count where the two-phase path takes over (wants_expansion), the fp16 expansion of the weights follows.
 static size_t x16_bytes(const gwq_packed* P, gwq_dtype xd, int M) {
   if (xd != GWQ_BF16) return 0;
   return (((size_t)M * P->K * 2 + 255) & ~(size_t)255) + (((size_t)M * 4 + 255) & ~(size_t)255);
@@ -575,7 +953,7 @@ static size_t x16_bytes(const gwq_packed* P, gwq_dtype xd, int M) {
 size_t gwq_prefill_workspace_bytes(const gwq_packed* P, gwq_dtype xd, int M) {
   const gwq_priv* pv = static_cast<const gwq_priv*>(P->priv);
   if (!pv->cv || !pv->sz_t || P->K % kBlockK != 0) return 0;   // the general kernel needs none
-  return x16_bytes(P, xd, M) + (M >= kExpandMinTokens ? (((size_t)P->N * P->K * 2 + 255) & ~(size_t)255) : 0);
+  return x16_bytes(P, xd, M) + (wants_expansion(P, M) ? (((size_t)P->N * P->K * 2 + 255) & ~(size_t)255) : 0);
 }
 
 // Prefill launcher: K <= 65536 (16-bit outlier columns).  Other shapes go to the general kernel.
@@ -596,7 +974,7 @@ gwq_status gwq_launch_prefill(const gwq_packed* P, const void* x, gwq_dtype xd, 
     x = x16;
     tok_scale = ts;
   }
-  if (M >= kExpandMinTokens && ws && ws_bytes >= gwq_prefill_workspace_bytes(P, xd, M))
+  if (wants_expansion(P, M) && ws && ws_bytes >= gwq_prefill_workspace_bytes(P, xd, M))
     return launch_expanded(P, x, tok_scale, reinterpret_cast<uint16_t*>(static_cast<char*>(ws) + xb), M, y, yd, stream);
   if (P->bits == 4) return launch_tok<4>(P, x, tok_scale, M, y, yd, stream);
   return launch_tok<3>(P, x, tok_scale, M, y, yd, stream);

@@ -123,6 +123,28 @@ def test_persistent_ctas_with_several_tiles_each(bits, dtype, expanded):
     P.free()
 
 
+@pytest.mark.parametrize("N,K,M,bits,dtype", [(600, 320, 2300, 4, "f16"), (2700, 192, 2100, 3, "bf16"), (96, 64, 2048, 4, "f16")])
+def test_two_phase_path_ragged_tiles_and_bands(N, K, M, bits, dtype):
+    # the contraction on CTA pairs (tiles of 256 rows x 256 tokens, reached with many tokens and room for the
+    # expanded weights): ragged last tiles in both directions, 11 weight tiles (a full band of 8 and a narrower one),
+    # a layer smaller than one tile; every output
+    W, G = synth.make_weight_and_grad(N, K, 27)
+    L = orc.quantize_layer(W, G, 0.01, bits, 64)
+    P = quantize_on_gpu(W, G, 0.01, bits, 64)
+    assert_packed_equal(P, L)
+    w_hat = oracle_w_hat(L)
+    bits16, xv = synth.make_activations(M, K, seed=127, dtype=dtype, heavy_channels=4)
+    y_ref, bound = orc.linear(xv, w_hat)
+    x = x_tensor(bits16, dtype)
+    lib = gwq.load_library()
+    xd = gwq.GWQ_F16 if dtype == "f16" else gwq.GWQ_BF16
+    assert int(lib.gwq_linear_workspace_bytes(P._h, xd, M)) >= N * K * 2
+    y = gwq.gwq_linear(P, x, out_dtype=torch.float32)          # the binding supplies the workspace
+    assert gwq.gwq_device_status(P) == 0
+    assert_linear_close(y, y_ref, bound)
+    P.free()
+
+
 def test_single_layer_config_seed_0():
     # the single-layer configuration as written: 4096 x 4096, seed 0, 4 bits, groups of 128, 1 % outliers, fp16
     # activations, one token; encoding bit for bit and every output
@@ -176,7 +198,7 @@ SMALL_GROUP_LAYERS = [
                                      (33, "f16"), (300, "bf16"), (2100, "f16")])
 def test_small_groups_on_the_fast_paths(layer, M, dtype):
     # K a multiple of 128: groups of 16 and 32 run on the tensor cores (one scale per 16 or 32 columns inside the
-    # 64-column k-block; the weights expanded beforehand from 2048 tokens on) and, for one token, on the streaming kernel
+    # 64-column k-block; the weights expanded beforehand for many tokens) and, for one token, on the streaming kernel
     P, L, w_hat = _layer(*layer)
     bits16, xv = synth.make_activations(M, P.K, seed=160 + M, dtype=dtype, heavy_channels=8 if M > 32 else 0)
     y_ref, bound = orc.linear(xv, w_hat)

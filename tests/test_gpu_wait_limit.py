@@ -13,7 +13,8 @@ from tests.gpu_util import assert_linear_close, oracle_w_hat, quantize_on_gpu, x
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("N,K,M", [(128, 256, 64), (384, 2048, 300)])
+# the last case takes the two-phase path (the contraction on CTA pairs)
+@pytest.mark.parametrize("N,K,M", [(128, 256, 64), (384, 2048, 300), (600, 512, 2200)])
 def test_zero_spin_limit_gives_up_cleanly_and_the_layer_stays_usable(N, K, M):
     W, G = synth.make_weight_and_grad(N, K, 95)
     L = orc.quantize_layer(W, G, 0.01, 4, 128)
