@@ -31,6 +31,10 @@ template <int TP, bool BF16>
 __global__ void __launch_bounds__(128) tokens_to_columns(const uint16_t* __restrict__ x, uint16_t* __restrict__ xt,
                                                          float* __restrict__ xg, int M, int K) {
   __shared__ float red[4][TP];
+  // launched with programmatic stream serialization: the product that follows may start fetching its weights now;
+  // x may still be being written by the kernel before this one
+  asm volatile("griddepcontrol.launch_dependents;");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const int col = blockIdx.x * 128 + threadIdx.x;
   uint16_t v[TP];
 #pragma unroll
@@ -179,14 +183,28 @@ gwq_status gwq_launch_decode_multi(const gwq_packed* const* P, int count, const 
     uint16_t* xt = static_cast<uint16_t*>(pv->xt);
     float* xg = reinterpret_cast<float*>(static_cast<char*>(pv->xt) + (size_t)K * 32 * 2);
     const bool bf = xd == GWQ_BF16;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(K / 128));
+    cfg.blockDim = dim3(128);
+    cfg.stream = stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t pe = cudaSuccess;
     switch (v.tp) {
-#define GWQ_T2C(TP)                                                                                                 \
-  case TP:                                                                                                          \
-    if (bf) tokens_to_columns<TP, true><<<K / 128, 128, 0, stream>>>(a.x, xt, xg, M, K);                          \
-    else tokens_to_columns<TP, false><<<K / 128, 128, 0, stream>>>(a.x, xt, xg, M, K);                            \
+#define GWQ_T2C(TP)                                                                                   \
+  case TP:                                                                                            \
+    pe = bf ? cudaLaunchKernelEx(&cfg, tokens_to_columns<TP, true>, a.x, xt, xg, M, K)               \
+            : cudaLaunchKernelEx(&cfg, tokens_to_columns<TP, false>, a.x, xt, xg, M, K);             \
     break;
       GWQ_T2C(4) GWQ_T2C(8) GWQ_T2C(16) GWQ_T2C(32)
 #undef GWQ_T2C
+    }
+    if (pe != cudaSuccess) {
+      (void)cudaGetLastError();
+      return GWQ_ERR_CUDA;
     }
     if (cudaGetLastError() != cudaSuccess) return GWQ_ERR_CUDA;
     a.xt = xt;
