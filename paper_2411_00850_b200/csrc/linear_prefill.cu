@@ -910,6 +910,76 @@ gwq_status launch_tok(const gwq_packed* P, const void* x, const float* tok_scale
   return launch<BITS, 256, false>(P, x, tok_scale, nullptr, M, y, yd, stream);
 }
 
+// The same expansion by blocks of 128 rows x 128 columns, for layers that carry the block-ordered outlier list
+// (groups of 64 or 128, K a multiple of 128): one CTA expands a block into shared memory, drops the block's FP16
+// outliers over their zero entries there and writes whole 256-byte row segments: one pass, no 2-byte stores to
+// global memory.
+template <int BITS>
+__global__ void __launch_bounds__(256) expand_block_kernel(const uint32_t* __restrict__ codes, const uint32_t* __restrict__ sz_t,
+                                                           const uint32_t* __restrict__ ob, const int32_t* __restrict__ ob_ptr,
+                                                           uint16_t* __restrict__ w16, int N, int K, int group) {
+  constexpr int kPitch = 128 + 8;                  // halves per row of the tile: 16 bytes of padding
+  __shared__ __align__(16) uint16_t tile[128 * kPitch];
+  const int G = K >> 7;
+  const int blk = blockIdx.x, row0 = (blk / G) * 128, g = blk % G;
+  const int e0 = __ldg(ob_ptr + blk), e1 = __ldg(ob_ptr + blk + 1);
+#pragma unroll
+  for (int u = 0; u < 2; ++u) {
+    const int idx = threadIdx.x + 256 * u, r = idx >> 2, q = idx & 3;   // row of the block, run of 32 columns
+    const int row = min(row0 + r, N - 1);
+    const uint32_t* src = codes + ((size_t)row * (K >> 5) + g * 4 + q) * BITS;
+    unsigned w[BITS];
+    if (BITS == 4) {
+      const uint4 v = __ldg(reinterpret_cast<const uint4*>(src));
+      w[0] = v.x; w[1] = v.y; w[2] = v.z; w[BITS - 1] = v.w;
+    } else {
+#pragma unroll
+      for (int k = 0; k < BITS; ++k) w[k] = __ldg(src + k);
+    }
+    unsigned s2[2], zm[2];   // scale and zero-point of the run's two halves of 16 columns
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const unsigned sz = __ldg(sz_t + (size_t)((g * 128 + q * 32 + 16 * h) / group) * N + row);
+      s2[h] = (sz & 0xFFFFu) * 0x00010001u;
+      zm[h] = 0x64006400u | ((sz >> 16) * 0x00010001u);
+    }
+    unsigned out[16];
+    if (BITS == 4) {
+#pragma unroll
+      for (int t = 0; t < 4; ++t)
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+          out[4 * t + j] = mul_scale<false>(sub_magic<false>(((w[t % BITS] >> (4 * j)) & 0x000F000Fu) | 0x64006400u, zm[t / 2]),
+                                            s2[t / 2], 0);
+    } else {
+#pragma unroll
+      for (int k = 0; k < 3; ++k)
+#pragma unroll
+        for (int pp = 0; pp < 5; ++pp)
+          out[5 * k + pp] = mul_scale<false>(sub_magic<false>(((w[k] >> (3 * pp)) & 0x00070007u) | 0x64006400u, zm[(5 * k + pp) / 8]),
+                                             s2[(5 * k + pp) / 8], 0);
+      const unsigned last = ((w[0] >> 15) & 0x00010001u) | ((w[1] >> 14) & 0x00020002u) | ((w[BITS - 1] >> 13) & 0x00040004u);
+      out[15] = mul_scale<false>(sub_magic<false>(last | 0x64006400u, zm[1]), s2[1], 0);
+    }
+    uint4* dst = reinterpret_cast<uint4*>(tile + r * kPitch + q * 32);
+#pragma unroll
+    for (int c = 0; c < 4; ++c) dst[c] = make_uint4(out[4 * c], out[4 * c + 1], out[4 * c + 2], out[4 * c + 3]);
+  }
+  __syncthreads();
+  for (int e = e0 + threadIdx.x; e < e1; e += 256) {
+    const unsigned v = __ldg(ob + e);
+    tile[((v >> 23) & 127u) * kPitch + ((v >> 16) & 127u)] = (uint16_t)v;
+  }
+  __syncthreads();
+#pragma unroll
+  for (int u = 0; u < 8; ++u) {
+    const int id = threadIdx.x + 256 * u, r = id >> 4, pc = id & 15;   // 16-byte piece pc of row r
+    if (row0 + r < N)
+      *reinterpret_cast<uint4*>(w16 + (size_t)(row0 + r) * K + g * 128 + pc * 8) =
+          *reinterpret_cast<const uint4*>(tile + r * kPitch + pc * 8);
+  }
+}
+
 // When the weights are expanded once instead of once per token tile.  The expansion is a pass of 2.5 bytes per weight
 // (about 40 us for 45 M weights, 210 us for 235 M) and the contraction on CTA pairs then runs at 1000 to 1600 TFLOP/s
 // where the fused kernel, whose tiles each expand their weights again, reaches 250 to 770.  Measured, bf16 activations,
@@ -930,12 +1000,20 @@ static bool wants_expansion(const gwq_packed* P, int M) {
 gwq_status launch_expanded(const gwq_packed* P, const void* x, const float* tok_scale, uint16_t* w16, int M, void* y,
                            gwq_dtype yd, cudaStream_t stream) {
   const gwq_priv* pv = static_cast<const gwq_priv*>(P->priv);
-  const long long runs = (long long)P->N * (P->K / 32);
-  if (P->bits == 4)
-    expand_kernel<4><<<(unsigned)((runs + 255) / 256), 256, 0, stream>>>(P->codes, pv->sz_t, w16, P->N, P->K, P->group);
-  else
-    expand_kernel<3><<<(unsigned)((runs + 255) / 256), 256, 0, stream>>>(P->codes, pv->sz_t, w16, P->N, P->K, P->group);
-  expand_outliers_kernel<<<(P->N + 7) / 8, 256, 0, stream>>>(P->S->row_ptr, pv->cv, w16, P->N, P->K);
+  if (pv->ob && pv->ob_ptr && P->K % 128 == 0) {
+    const unsigned blocks = (unsigned)((P->N + 127) / 128) * (unsigned)(P->K / 128);
+    if (P->bits == 4)
+      expand_block_kernel<4><<<blocks, 256, 0, stream>>>(P->codes, pv->sz_t, pv->ob, pv->ob_ptr, w16, P->N, P->K, P->group);
+    else
+      expand_block_kernel<3><<<blocks, 256, 0, stream>>>(P->codes, pv->sz_t, pv->ob, pv->ob_ptr, w16, P->N, P->K, P->group);
+  } else {
+    const long long runs = (long long)P->N * (P->K / 32);
+    if (P->bits == 4)
+      expand_kernel<4><<<(unsigned)((runs + 255) / 256), 256, 0, stream>>>(P->codes, pv->sz_t, w16, P->N, P->K, P->group);
+    else
+      expand_kernel<3><<<(unsigned)((runs + 255) / 256), 256, 0, stream>>>(P->codes, pv->sz_t, w16, P->N, P->K, P->group);
+    expand_outliers_kernel<<<(P->N + 7) / 8, 256, 0, stream>>>(P->S->row_ptr, pv->cv, w16, P->N, P->K);
+  }
   if (cudaGetLastError() != cudaSuccess) return GWQ_ERR_CUDA;
   const gwq_status st = launch_pairs(P, x, tok_scale, w16, M, y, yd, stream);
   if (st != GWQ_ERR_UNSUPPORTED) return st;   // no room for a cluster of two: one CTA per tile
