@@ -497,9 +497,11 @@ __global__ void __launch_bounds__(256) expand_outliers_kernel(const int32_t* __r
 //                        CTA when an accumulator is free again.
 // Every wait is bounded (see the fused kernel); the two CTAs leave together through a cluster barrier.
 constexpr int kPairThreads = 32 * 6;
-constexpr int kPairStages = 6;
-constexpr int kPairTok = 256;                 // tokens of a pair's tile (UMMA N), 128 loaded by each CTA
-constexpr int kPairStageBytes = 2 * kTileN * kBlockK * 2;   // A half and B half of a k-block: 32 KB
+// TOK tokens per tile of a pair (UMMA N; 256, or 128 where that fills the pairs better), half of them loaded by each CTA
+template <int TOK> struct PairCfg {
+  static constexpr int kStageBytes = kTileN * kBlockK * 2 + (TOK / 2) * kBlockK * 2;   // A half and B half of a k-block
+  static constexpr int kStages = TOK == 256 ? 6 : 8;                                   // 192 KB of stages
+};
 constexpr int kOutStageBytes = 32 * kTileN * 4;             // 32 tokens x 128 features, up to 4 bytes each
 
 __device__ __forceinline__ unsigned cluster_ctarank() {
@@ -573,14 +575,16 @@ struct PairArgs {
 // tmx: x16 [M][K] with boxes of 64 columns x 128 rows; tmw: expanded weights [N][K], same boxes.
 // tmy: y [M][N] with boxes of 128 output features x 32 tokens.
 // ntn: tiles of 256 weight rows; ntiles: all tiles (order: pair_tile); pairs: clusters of the launch.
+template <int TOK>
 __global__ void __launch_bounds__(kPairThreads, 1)
 pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUtensorMap tmw,
             const __grid_constant__ CUtensorMap tmy, const PairArgs p, const int ntn, const int ntiles, const int pairs) {
   constexpr int kHalfBytes = kTileN * kBlockK * 2;   // 16 KB: 128 rows x 128 bytes
+  constexpr int kPairStages = PairCfg<TOK>::kStages, kPairStageBytes = PairCfg<TOK>::kStageBytes, kPairTok = TOK;
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* tiles =
       reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
-  __shared__ __align__(8) unsigned long long bars[2 * kPairStages + 5];
+  __shared__ __align__(8) unsigned long long bars[2 * 8 + 5];
   __shared__ unsigned tmem_base_s;
   __shared__ int abort_s;
   volatile int* abort_flag = &abort_s;
@@ -615,8 +619,8 @@ pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUt
     mbar_init(drain_bar, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 1) {   // tensor memory of both CTAs: two accumulators of 256 columns x 128 lanes each
-    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(512)
+  if (warp == 1) {   // tensor memory of both CTAs: two accumulators of TOK columns x 128 lanes each
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(2 * TOK)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
   }
@@ -640,7 +644,7 @@ pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUt
           const int it = ti * nkb + kb, s = it % kPairStages, round = it / kPairStages;
           if (round > 0) ok = mbar_wait(empty(s), (round - 1) & 1, abort_flag, lim);
           if (!ok) break;
-          if (rank == 0) mbar_expect_tx(full(s), 2 * kPairStageBytes);
+          if (rank == 0) mbar_expect_tx(full(s), 2 * kPairStageBytes);   // both CTAs' halves
           const unsigned fb = in_first_cta(full(s));
           tma_load_2d_pair(smem_u32(a_tile(s)), &tmw, kb * kBlockK, n0, fb);
           tma_load_2d_pair(smem_u32(b_tile(s)), &tmx, kb * kBlockK, m0, fb);
@@ -771,12 +775,13 @@ pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUt
   cluster_sync_all();   // neither CTA frees its tensor memory, or exits, while the other may still signal or write it
   if (warp == 1) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(512) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(2 * TOK) : "memory");
   }
 }
 
 // Launch of the pair kernel on the expanded weights w16 [N][K] and fp16 activations x [M][K].
-gwq_status launch_pairs(const gwq_packed* P, const void* x, const float* tok_scale, const void* w16, int M, void* y,
+template <int TOK>
+gwq_status launch_pairs_tok(const gwq_packed* P, const void* x, const float* tok_scale, const void* w16, int M, void* y,
                         gwq_dtype yd, cudaStream_t stream) {
   const gwq_priv* pv = static_cast<const gwq_priv*>(P->priv);
   EncodeTiledFn enc = encode_fn();
@@ -785,9 +790,10 @@ gwq_status launch_pairs(const gwq_packed* P, const void* x, const float* tok_sca
   const cuuint32_t estr[2] = {1, 1};
   const cuuint32_t box[2] = {(cuuint32_t)kBlockK, (cuuint32_t)kTileN};
   {
+    const cuuint32_t xbox[2] = {(cuuint32_t)kBlockK, (cuuint32_t)(TOK / 2)};
     const cuuint64_t dims[2] = {(cuuint64_t)P->K, (cuuint64_t)M};
     const cuuint64_t strides[1] = {(cuuint64_t)P->K * 2};
-    if (enc(&tmx, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(x), dims, strides, box, estr,
+    if (enc(&tmx, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(x), dims, strides, xbox, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return GWQ_ERR_CUDA;
@@ -813,13 +819,13 @@ gwq_status launch_pairs(const gwq_packed* P, const void* x, const float* tok_sca
             CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return GWQ_ERR_CUDA;
   }
-  const size_t smem = (size_t)kPairStages * kPairStageBytes + 2 * kOutStageBytes + 1024;
-  if (cudaFuncSetAttribute(pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return GWQ_ERR_CUDA;
+  const size_t smem = (size_t)PairCfg<TOK>::kStages * PairCfg<TOK>::kStageBytes + 2 * kOutStageBytes + 1024;
+  if (cudaFuncSetAttribute(pair_kernel<TOK>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return GWQ_ERR_CUDA;
   PairArgs a;
   a.y = y; a.yd = yd; a.status = pv->dev_status; a.tok_scale = tok_scale; a.N = P->N; a.K = P->K; a.M = M;
   a.tma_store = tma_store;
   a.wait_cycles = pv->wait_cycles;
-  const int ntn = (P->N + 2 * kTileN - 1) / (2 * kTileN), ntiles = ntn * ((M + kPairTok - 1) / kPairTok);
+  const int ntn = (P->N + 2 * kTileN - 1) / (2 * kTileN), ntiles = ntn * ((M + TOK - 1) / TOK);
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 2;
@@ -834,18 +840,32 @@ gwq_status launch_pairs(const gwq_packed* P, const void* x, const float* tok_sca
   // persistent: as many pairs as the device holds at once (pairs sit inside one GPC, so this may be fewer than SMs / 2)
   cfg.gridDim = dim3(2u * (unsigned)(pv->sm_count / 2));
   int resident = 0;
-  if (cudaOccupancyMaxActiveClusters(&resident, pair_kernel, &cfg) != cudaSuccess || resident < 1) {
+  if (cudaOccupancyMaxActiveClusters(&resident, pair_kernel<TOK>, &cfg) != cudaSuccess || resident < 1) {
     (void)cudaGetLastError();
     return GWQ_ERR_UNSUPPORTED;
   }
   int pairs = resident < pv->sm_count / 2 ? resident : pv->sm_count / 2;
   if (pairs > ntiles) pairs = ntiles;
   cfg.gridDim = dim3(2u * (unsigned)pairs);
-  if (cudaLaunchKernelEx(&cfg, pair_kernel, tmx, tmw, tmy, a, ntn, ntiles, pairs) != cudaSuccess) {
+  if (cudaLaunchKernelEx(&cfg, pair_kernel<TOK>, tmx, tmw, tmy, a, ntn, ntiles, pairs) != cudaSuccess) {
     (void)cudaGetLastError();
     return GWQ_ERR_CUDA;
   }
   return GWQ_OK;
+}
+
+// Tokens per tile: the pairs work in rounds of one tile each.  A 128-token tile loads 24 KB per k-block for half the
+// multiplies of a 256-token tile's 32 KB, and the operands come out of L2, so it takes about 0.8 of the time, not half
+// (measured, 512 tokens: 66 against 76 us where both need one round, 4096 x 11008; 69 against 64 us with three
+// rounds against two, 11008 x 4096): it is taken only where it needs hardly more rounds than the larger tile.
+gwq_status launch_pairs(const gwq_packed* P, const void* x, const float* tok_scale, const void* w16, int M, void* y, gwq_dtype yd,
+                        cudaStream_t stream) {
+  const gwq_priv* pv = static_cast<const gwq_priv*>(P->priv);
+  const long long pairs = pv->sm_count / 2 > 0 ? pv->sm_count / 2 : 1;
+  const long long ntn = (P->N + 2 * kTileN - 1) / (2 * kTileN);
+  const long long r256 = (ntn * ((M + 255) / 256) + pairs - 1) / pairs, r128 = (ntn * ((M + 127) / 128) + pairs - 1) / pairs;
+  if (4 * r128 < 5 * r256) return launch_pairs_tok<128>(P, x, tok_scale, w16, M, y, yd, stream);
+  return launch_pairs_tok<256>(P, x, tok_scale, w16, M, y, yd, stream);
 }
 
 template <int BITS, int TOK, bool EXP, int GPK = 1>
