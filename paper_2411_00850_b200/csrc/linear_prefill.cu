@@ -721,9 +721,12 @@ pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUt
           asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to the TMA
           asm volatile("bar.sync 1, 128;" ::: "memory");
           if (warp == 2 && lane == 0) {   // rows past N and tokens past M are clipped by the copy
-            asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
-                         ::"l"(&tmy), "r"(tn * (2 * kTileN) + (int)rank * kTileN), "r"(m0 + c0), "r"(smem_u32(st))
-                         : "memory");
+            // y is written once and not read again here: its lines are the first to leave L2, not the operands'
+            asm volatile(
+                "{\n .reg .b64 pol;\n createpolicy.fractional.L2::evict_first.b64 pol, 1.0;\n"
+                " cp.async.bulk.tensor.2d.global.shared::cta.bulk_group.L2::cache_hint [%0, {%1, %2}], [%3], pol;\n}\n"
+                ::"l"(&tmy), "r"(tn * (2 * kTileN) + (int)rank * kTileN), "r"(m0 + c0), "r"(smem_u32(st))
+                : "memory");
             asm volatile("cp.async.bulk.commit_group;" ::: "memory");
           }
           ++chunk;
