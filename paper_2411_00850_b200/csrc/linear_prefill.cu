@@ -710,13 +710,46 @@ pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUt
             if (warp == 2 && lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
             asm volatile("bar.sync 1, 128;" ::: "memory");
           }
+          // token scales of the chunk (one vector load per four tokens while the chunk lies inside M)
+          float ts[32];
+          if (p.tok_scale) {
+            if (m0 + c0 + 32 <= p.M) {
 #pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            float f = __uint_as_float(v[i]);
-            if (p.tok_scale) f *= __ldg(p.tok_scale + min(m0 + c0 + i, p.M - 1));
-            if (p.yd == GWQ_F32) reinterpret_cast<float*>(st)[i * kTileN + r] = f;
-            else if (p.yd == GWQ_F16) reinterpret_cast<__half*>(st)[i * kTileN + r] = __float2half_rn(f);
-            else reinterpret_cast<__nv_bfloat16*>(st)[i * kTileN + r] = __float2bfloat16_rn(f);
+              for (int q = 0; q < 8; ++q) {
+                const float4 t4 = __ldg(reinterpret_cast<const float4*>(p.tok_scale + m0 + c0) + q);
+                ts[4 * q] = t4.x; ts[4 * q + 1] = t4.y; ts[4 * q + 2] = t4.z; ts[4 * q + 3] = t4.w;
+              }
+            } else {
+#pragma unroll
+              for (int i = 0; i < 32; ++i) ts[i] = __ldg(p.tok_scale + min(m0 + c0 + i, p.M - 1));
+            }
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) ts[i] = 1.f;
+          }
+          if (p.yd == GWQ_F32) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) reinterpret_cast<float*>(st)[i * kTileN + r] = __uint_as_float(v[i]) * ts[i];
+          } else {
+            // 2-byte outputs: neighbouring lanes (features r, r + 1) swap one of every two tokens, so that each lane
+            // converts and stores a pair of neighbouring features of one token as one word
+            const bool odd = (lane & 1) != 0;
+            unsigned* st32 = reinterpret_cast<unsigned*>(st);
+#pragma unroll
+            for (int i = 0; i < 32; i += 2) {
+              const float f0 = __uint_as_float(v[i]) * ts[i], f1 = __uint_as_float(v[i + 1]) * ts[i + 1];
+              const float got = __shfl_xor_sync(0xFFFFFFFFu, odd ? f0 : f1, 1);
+              const float lo = odd ? got : f0, hi = odd ? f1 : got;   // features (r & ~1), (r | 1) of token i + odd
+              unsigned w;
+              if (p.yd == GWQ_F16) {
+                const __half2 h = __floats2half2_rn(lo, hi);
+                w = *reinterpret_cast<const unsigned*>(&h);
+              } else {
+                const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+                w = *reinterpret_cast<const unsigned*>(&h);
+              }
+              st32[((i + (odd ? 1 : 0)) * kTileN + (r & ~1)) >> 1] = w;
+            }
           }
           asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to the TMA
           asm volatile("bar.sync 1, 128;" ::: "memory");
