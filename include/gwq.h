@@ -147,9 +147,9 @@ gwq_status gwq_pack(const uint16_t* W_f16, gwq_outliers* S, int32_t N, int32_t K
  *   x: device [M, K], fp16 or bf16 (x_dtype).  y: device [M, N], y_dtype one of
  *   F16 / BF16 / F32.  Accumulation is FP32.  M >= 1.  Up to 32 tokens take a bandwidth-bound streaming
  *   kernel (mma.sync; with a workspace, 17 to 32 fp16 tokens take a tcgen05 one: see gwq_linear_ws), more tokens
- *   the tensor-core kernel (TMA, tcgen05, tensor memory), which with a workspace and enough tokens (from 1024 on,
- *   from 384 on for layers of up to 48 M weights) expands the weights once instead of once per token tile and
- *   contracts on pairs of CTAs (tcgen05 cta_group::2, tiles of 256 features x 256 tokens).
+ *   the tensor-core kernel (TMA, tcgen05, tensor memory), which with a workspace and enough tokens (more than 256;
+ *   from 64 on for layers with fewer 128-row tiles than the device has SMs) expands the weights once instead of
+ *   once per token tile and contracts on pairs of CTAs (tcgen05 cta_group::2, tiles of 256 features x 256 tokens).
  *   Asynchronous on `stream`: the call only enqueues kernels.  It never allocates and never
  *   synchronises, so it may be captured into a CUDA graph from its first use.  Calls that share P
  *   must be enqueued on one stream (or otherwise ordered): with 9 to 32 tokens they share a small

@@ -1037,19 +1037,23 @@ __global__ void __launch_bounds__(256) expand_block_kernel(const uint32_t* __res
 }
 
 // When the weights are expanded once instead of once per token tile.  The expansion is a pass of 2.5 bytes per weight
-// (about 40 us for 45 M weights, 210 us for 235 M) and the contraction on CTA pairs then runs at 1000 to 1600 TFLOP/s
-// where the fused kernel, whose tiles each expand their weights again, reaches 250 to 770.  Measured, bf16 activations,
-// 4 bit, fused against two-phase: 1024 tokens: 156 / 131 us on 11008 x 4096, 145 / 122 on 4096 x 11008, 199 / 168 on
-// 8192 x 8192, 632 / 565 on 28672 x 8192; 512 tokens: 114 / 104, 144 / 115 and 73 / 62 (4096 x 4096), but 117 / 125 on
-// 8192 x 8192 and 374 / 408 on 28672 x 8192; 384 tokens: 101 / 101 and 144 / 115; 256 tokens: 74 / 81.
-constexpr int kExpandMinTokens = 1024;                       // every layer
-constexpr int kExpandMinTokensSmall = 384;                   // layers of up to kExpandSmallWeights weights
-constexpr long long kExpandSmallWeights = 48LL * 1000 * 1000;
+// (24 us for 45 M weights, 125 us for 235 M); the contraction on CTA pairs then runs at 1000 to 1500 TFLOP/s, where the
+// fused kernel is bound by its dequantisation warps (250 to 770), expands the weights again for every token tile of
+// 256 and leaves SMs idle when the layer has fewer 128-row tiles than the device has SMs.  So: more than 256 tokens
+// always; from 64 tokens on where the 128-row tiles do not fill the SMs.  Measured, bf16 activations, 4 bit, fused
+// against two-phase (us): 11008 x 4096: 52 / 52 at 64 tokens, 58 / 54 at 128, 75 / 59 at 256, 114 / 78 at 512;
+// 4096 x 11008: 123 / 83 at 64, 147 / 86 at 256, 144 / 89 at 512; 4096 x 4096: 53 / 35 at 64, 74 / 39 at 256;
+// 8192 x 8192: 99 / 82 at 128, 117 / 84 at 256, 116 / 92 at 512; 28672 x 8192 (224 tiles on 148 SMs): 180 / 228 at 128,
+// 207 / 239 at 256, 361 / 307 at 384, 374 / 312 at 512.
+constexpr int kExpandAlwaysTokens = 257;   // more than one token tile of the fused kernel
+constexpr int kExpandMinTokens = 64;       // ... where the fused kernel's tiles leave SMs idle
 static bool wants_expansion(const gwq_packed* P, int M) {
 #ifdef GWQ_TUNE_EXPAND_MIN
   return M >= GWQ_TUNE_EXPAND_MIN;
 #endif
-  return M >= kExpandMinTokens || (M >= kExpandMinTokensSmall && (long long)P->N * P->K <= kExpandSmallWeights);
+  const gwq_priv* pv = static_cast<const gwq_priv*>(P->priv);
+  const int sms = pv->sm_count > 0 ? pv->sm_count : 148;
+  return M >= kExpandAlwaysTokens || (M >= kExpandMinTokens && (P->N + kTileN - 1) / kTileN < sms);
 }
 
 // Expanded weights: the expansion, the outliers over it, then the contraction with token tiles of 256.
