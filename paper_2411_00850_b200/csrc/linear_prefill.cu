@@ -21,6 +21,8 @@
 // multiplies the token's column by 2^e again.  fp16 also keeps the FP16 outliers exact.
 // Stages are handed over with mbarriers; every wait is bounded and, when it runs out, the CTA
 // records GWQ_ERR_TIMEOUT, leaves its loops, frees its tensor memory and returns.
+#include <atomic>
+
 #include "tc_common.cuh"
 
 namespace {
@@ -875,11 +877,19 @@ gwq_status launch_pairs_tok(const gwq_packed* P, const void* x, const float* tok
   cfg.numAttrs = 1;
   // persistent: as many pairs as the device holds at once (pairs sit inside one GPC, so this may be fewer than SMs / 2)
   cfg.gridDim = dim3(2u * (unsigned)(pv->sm_count / 2));
-  int resident = 0;
-  if (cudaOccupancyMaxActiveClusters(&resident, pair_kernel<TOK>, &cfg) != cudaSuccess || resident < 1) {
-    (void)cudaGetLastError();
-    return GWQ_ERR_UNSUPPORTED;
+  // (asked once per device and token-tile size: the answer depends on nothing else)
+  static std::atomic<int> resident_on[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) dev = 63;
+  int resident = resident_on[dev].load(std::memory_order_relaxed);
+  if (resident == 0) {
+    if (cudaOccupancyMaxActiveClusters(&resident, pair_kernel<TOK>, &cfg) != cudaSuccess || resident < 1) {
+      (void)cudaGetLastError();
+      resident = -1;
+    }
+    resident_on[dev].store(resident, std::memory_order_relaxed);
   }
+  if (resident < 1) return GWQ_ERR_UNSUPPORTED;
   int pairs = resident < pv->sm_count / 2 ? resident : pv->sm_count / 2;
   if (pairs > ntiles) pairs = ntiles;
   cfg.gridDim = dim3(2u * (unsigned)pairs);
