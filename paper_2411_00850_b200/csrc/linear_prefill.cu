@@ -1,7 +1,9 @@
 // Prefill path (M > 32) of y = x (s (q - z) + S)^T (Section 3.2, Eq. "w"): a dense contraction
-// on the 5th-generation tensor cores.
+// on the 5th-generation tensor cores, in two forms: a fused kernel that dequantises into its weight tiles (few
+// tokens; described here) and, further down, a two-phase path that expands the weights once and contracts on pairs
+// of CTAs.
 //
-// One CTA computes a tile of 128 output features x TOK tokens.  The weight rows are the M side
+// Fused kernel: one CTA computes a tile of 128 output features x TOK tokens.  The weight rows are the M side
 // of the MMA (A operand), the tokens its N side (B operand); both are K-major in shared memory
 // in the 128-byte-swizzled layout, the FP32 accumulator lives in tensor memory.
 //   warp 0, one thread : TMA loads of the activation tile (TOK x 64) per k-block
@@ -34,7 +36,7 @@ constexpr int kDequantWarps = 4;   // warps of one dequantisation group (one thr
 constexpr int kDequantGroups = 3;  // groups; group g takes the k-blocks g, g + 3, ... (numbered over all tiles)
 constexpr int kEpilogueWarps = 4;  // one thread per tile row
 constexpr int kCtaThreads = 32 * (2 + kDequantWarps * kDequantGroups + kEpilogueWarps);
-constexpr int kMaxStages = 8;
+constexpr int kMaxStages = 8;   // of the fused kernel
 
 struct PrefillArgs {
   const uint32_t* codes;
@@ -133,12 +135,10 @@ __device__ __forceinline__ unsigned sub_magic(unsigned qm, unsigned zm) {
   }
 }
 
-// EXP: the weights have been expanded to fp16 [N, K] beforehand (expand_kernel): the producer loads the weight tile
-// by TMA as well and the dequantisation warps have nothing to do.
 // GPK: scale groups per 64-column k-block: 1 (groups of 64 and 128), 2 (groups of 32), 4 (groups of 16).
-template <int BITS, int TOK, bool BF16, bool EXP, int GPK>
+template <int BITS, int TOK, bool BF16, int GPK>
 __global__ void __launch_bounds__(kCtaThreads, 1)
-prefill_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUtensorMap tmw, const PrefillArgs p,
+prefill_kernel(const __grid_constant__ CUtensorMap tmx, const PrefillArgs p,
                const int stages, const int ntn, const int ntiles) {
   constexpr int kABytes = kTileN * kBlockK * 2;   // 16 KB
   constexpr int kBBytes = TOK * kBlockK * 2;
@@ -204,9 +204,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
           const int it = ti * nkb + kb, s = it % stages, round = it / stages;
           if (round > 0) ok = mbar_wait(empty(s), (round - 1) & 1, abort_flag, lim);
           if (!ok) break;
-          mbar_expect_tx(full_b(s), EXP ? kBBytes + kABytes : kBBytes);
+          mbar_expect_tx(full_b(s), kBBytes);
           tma_load_2d(smem_u32(b_tile(s)), &tmx, kb * kBlockK, m0, full_b(s));
-          if (EXP) tma_load_2d(smem_u32(a_tile(s)), &tmw, kb * kBlockK, (tile % ntn) * kTileN, full_b(s));
           issued = it + 1;
         }
       }
@@ -225,7 +224,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
         const unsigned acc = tmem_acc + (unsigned)(a * kAccCols);
         for (int kb = 0; kb < nkb && ok; ++kb) {
           const int it = ti * nkb + kb, s = it % stages, round = it / stages;
-          ok = (EXP || mbar_wait(full_a(s), round & 1, abort_flag, lim)) && mbar_wait(full_b(s), round & 1, abort_flag, lim);
+          ok = mbar_wait(full_a(s), round & 1, abort_flag, lim) && mbar_wait(full_b(s), round & 1, abort_flag, lim);
           if (!ok) break;
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           const uint64_t da = umma_desc(smem_u32(a_tile(s))), db = umma_desc(smem_u32(b_tile(s)));
@@ -245,7 +244,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
     constexpr int WPB = kBlockK * BITS / 32;   // packed words per row per k-block (8 or 6)
     constexpr unsigned MAGIC = BF16 ? 0x43004300u : 0x64006400u;   // 128.0 / 1024.0: ulp = 1
     constexpr int kOutWin = 8;                 // outliers of the row kept this many entries ahead
-    for (int ti = 0; ti < (EXP ? 0 : my_tiles) && ok; ++ti) {
+    for (int ti = 0; ti < my_tiles && ok; ++ti) {
       const int tile = blockIdx.x + ti * gridDim.x;
       const int row = (tile % ntn) * kTileN + r;
       const bool live = row < p.N;
@@ -424,7 +423,9 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
 // Two-phase path for many tokens: every token tile of the fused kernel expands the same weights again (M / 256
 // times), so beyond a few tiles the weights are expanded once, to fp16 [N, K] in the caller's workspace (the same
 // values the fused kernel writes into its tiles: exact q - z, one fp16 rounding of the product with the scale, the
-// FP16 outliers over their zero entries), and the contraction streams both operands by TMA.
+// FP16 outliers over their zero entries), and the contraction (pair_kernel) streams both operands by TMA.
+// expand_kernel + expand_outliers_kernel serve the layers without a block-ordered outlier list (groups of 16 or 32,
+// K not a multiple of 128); the others take expand_block_kernel.
 template <int BITS>
 __global__ void __launch_bounds__(256) expand_kernel(const uint32_t* __restrict__ codes, const uint32_t* __restrict__ sz_t,
                                                      uint16_t* __restrict__ w16, int N, int K, int group) {
@@ -914,14 +915,13 @@ gwq_status launch_pairs(const gwq_packed* P, const void* x, const float* tok_sca
   return launch_pairs_tok<256>(P, x, tok_scale, w16, M, y, yd, stream);
 }
 
-template <int BITS, int TOK, bool EXP, int GPK = 1>
-gwq_status launch(const gwq_packed* P, const void* x, const float* tok_scale, const void* w16, int M, void* y,
-                  gwq_dtype yd, cudaStream_t stream) {
+template <int BITS, int TOK, int GPK = 1>
+gwq_status launch(const gwq_packed* P, const void* x, const float* tok_scale, int M, void* y, gwq_dtype yd, cudaStream_t stream) {
   constexpr bool BF16 = false;   // operands are always fp16 here (see the file header)
   const gwq_priv* pv = static_cast<const gwq_priv*>(P->priv);
   EncodeTiledFn enc = encode_fn();
   if (!enc) return GWQ_ERR_CUDA;
-  CUtensorMap tmx, tmw;
+  CUtensorMap tmx;
   const cuuint32_t estr[2] = {1, 1};
   {
     const cuuint64_t dims[2] = {(cuuint64_t)P->K, (cuuint64_t)M};
@@ -932,21 +932,11 @@ gwq_status launch(const gwq_packed* P, const void* x, const float* tok_scale, co
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return GWQ_ERR_CUDA;
   }
-  tmw = tmx;
-  if (EXP) {
-    const cuuint64_t dims[2] = {(cuuint64_t)P->K, (cuuint64_t)P->N};
-    const cuuint64_t strides[1] = {(cuuint64_t)P->K * 2};
-    const cuuint32_t box[2] = {(cuuint32_t)kBlockK, (cuuint32_t)kTileN};
-    if (enc(&tmw, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(w16), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-      return GWQ_ERR_CUDA;
-  }
   const int stage_bytes = kTileN * kBlockK * 2 + TOK * kBlockK * 2;
   int stages = (220 * 1024 - 1024) / stage_bytes;
   if (stages > kMaxStages) stages = kMaxStages;
   const size_t smem = (size_t)stages * stage_bytes + 1024;
-  if (cudaFuncSetAttribute(prefill_kernel<BITS, TOK, BF16, EXP, GPK>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  if (cudaFuncSetAttribute(prefill_kernel<BITS, TOK, BF16, GPK>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            (int)smem) != cudaSuccess)
     return GWQ_ERR_CUDA;
   PrefillArgs a;
@@ -955,7 +945,7 @@ gwq_status launch(const gwq_packed* P, const void* x, const float* tok_scale, co
   a.wait_cycles = pv->wait_cycles;
   const int ntn = (P->N + kTileN - 1) / kTileN, ntiles = ntn * ((M + TOK - 1) / TOK);
   const int grid = ntiles < pv->sm_count ? ntiles : pv->sm_count;   // persistent: at most one CTA per SM
-  prefill_kernel<BITS, TOK, BF16, EXP, GPK><<<grid, kCtaThreads, smem, stream>>>(tmx, tmw, a, stages, ntn, ntiles);
+  prefill_kernel<BITS, TOK, BF16, GPK><<<grid, kCtaThreads, smem, stream>>>(tmx, a, stages, ntn, ntiles);
   return cudaGetLastError() == cudaSuccess ? GWQ_OK : GWQ_ERR_CUDA;
 }
 
@@ -963,17 +953,17 @@ template <int BITS>
 gwq_status launch_tok(const gwq_packed* P, const void* x, const float* tok_scale, int M, void* y, gwq_dtype yd,
                       cudaStream_t stream) {
   if (P->group == 32) {   // small groups: the smallest and the largest token tile only
-    if (M <= 32) return launch<BITS, 32, false, 2>(P, x, tok_scale, nullptr, M, y, yd, stream);
-    return launch<BITS, 256, false, 2>(P, x, tok_scale, nullptr, M, y, yd, stream);
+    if (M <= 32) return launch<BITS, 32, 2>(P, x, tok_scale, M, y, yd, stream);
+    return launch<BITS, 256, 2>(P, x, tok_scale, M, y, yd, stream);
   }
   if (P->group == 16) {
-    if (M <= 32) return launch<BITS, 32, false, 4>(P, x, tok_scale, nullptr, M, y, yd, stream);
-    return launch<BITS, 256, false, 4>(P, x, tok_scale, nullptr, M, y, yd, stream);
+    if (M <= 32) return launch<BITS, 32, 4>(P, x, tok_scale, M, y, yd, stream);
+    return launch<BITS, 256, 4>(P, x, tok_scale, M, y, yd, stream);
   }
-  if (M <= 32) return launch<BITS, 32, false>(P, x, tok_scale, nullptr, M, y, yd, stream);
-  if (M <= 64) return launch<BITS, 64, false>(P, x, tok_scale, nullptr, M, y, yd, stream);
-  if (M <= 128) return launch<BITS, 128, false>(P, x, tok_scale, nullptr, M, y, yd, stream);
-  return launch<BITS, 256, false>(P, x, tok_scale, nullptr, M, y, yd, stream);
+  if (M <= 32) return launch<BITS, 32>(P, x, tok_scale, M, y, yd, stream);
+  if (M <= 64) return launch<BITS, 64>(P, x, tok_scale, M, y, yd, stream);
+  if (M <= 128) return launch<BITS, 128>(P, x, tok_scale, M, y, yd, stream);
+  return launch<BITS, 256>(P, x, tok_scale, M, y, yd, stream);
 }
 
 // The same expansion by blocks of 128 rows x 128 columns, for layers that carry the block-ordered outlier list
@@ -1085,9 +1075,7 @@ gwq_status launch_expanded(const gwq_packed* P, const void* x, const float* tok_
     expand_outliers_kernel<<<(P->N + 7) / 8, 256, 0, stream>>>(P->S->row_ptr, pv->cv, w16, P->N, P->K);
   }
   if (cudaGetLastError() != cudaSuccess) return GWQ_ERR_CUDA;
-  const gwq_status st = launch_pairs(P, x, tok_scale, w16, M, y, yd, stream);
-  if (st != GWQ_ERR_UNSUPPORTED) return st;   // no room for a cluster of two: one CTA per tile
-  return launch<4, 256, true>(P, x, tok_scale, w16, M, y, yd, stream);
+  return launch_pairs(P, x, tok_scale, w16, M, y, yd, stream);
 }
 
 }  // namespace
@@ -1123,7 +1111,10 @@ gwq_status gwq_launch_prefill(const gwq_packed* P, const void* x, gwq_dtype xd, 
     tok_scale = ts;
   }
   if (wants_expansion(P, M) && ws && ws_bytes >= gwq_prefill_workspace_bytes(P, xd, M))
-    return launch_expanded(P, x, tok_scale, reinterpret_cast<uint16_t*>(static_cast<char*>(ws) + xb), M, y, yd, stream);
+  {
+    const gwq_status st = launch_expanded(P, x, tok_scale, reinterpret_cast<uint16_t*>(static_cast<char*>(ws) + xb), M, y, yd, stream);
+    if (st != GWQ_ERR_UNSUPPORTED) return st;   // a device that holds no cluster of two such CTAs: the fused kernel
+  }
   if (P->bits == 4) return launch_tok<4>(P, x, tok_scale, M, y, yd, stream);
   return launch_tok<3>(P, x, tok_scale, M, y, yd, stream);
 }
