@@ -148,7 +148,7 @@ gwq_status gwq_pack(const uint16_t* W_f16, gwq_outliers* S, int32_t N, int32_t K
  *   F16 / BF16 / F32.  Accumulation is FP32.  M >= 1.  Up to 32 tokens take a bandwidth-bound streaming
  *   kernel (mma.sync; with a workspace, 17 to 32 fp16 tokens take a tcgen05 one: see gwq_linear_ws), more tokens
  *   the tensor-core kernel (TMA, tcgen05, tensor memory), which with a workspace and enough tokens (more than 256;
- *   from 64 on for layers with fewer 128-row tiles than the device has SMs) expands the weights once instead of
+ *   always for layers with fewer 128-row tiles than the device has SMs) expands the weights once instead of
  *   once per token tile and contracts on pairs of CTAs (tcgen05 cta_group::2, tiles of 256 features x 256 tokens).
  *   Asynchronous on `stream`: the call only enqueues kernels.  It never allocates and never
  *   synchronises, so it may be captured into a CUDA graph from its first use.  Calls that share P

@@ -1040,13 +1040,13 @@ __global__ void __launch_bounds__(256) expand_block_kernel(const uint32_t* __res
 // (24 us for 45 M weights, 125 us for 235 M); the contraction on CTA pairs then runs at 1000 to 1500 TFLOP/s, where the
 // fused kernel is bound by its dequantisation warps (250 to 770), expands the weights again for every token tile of
 // 256 and leaves SMs idle when the layer has fewer 128-row tiles than the device has SMs.  So: more than 256 tokens
-// always; from 64 tokens on where the 128-row tiles do not fill the SMs.  Measured, bf16 activations, 4 bit, fused
-// against two-phase (us): 11008 x 4096: 52 / 52 at 64 tokens, 58 / 54 at 128, 75 / 59 at 256, 114 / 78 at 512;
-// 4096 x 11008: 123 / 83 at 64, 147 / 86 at 256, 144 / 89 at 512; 4096 x 4096: 53 / 35 at 64, 74 / 39 at 256;
+// always; any number of tokens of this path (33 on) where the 128-row tiles do not fill the SMs.  Measured, bf16 activations, 4 bit, fused
+// against two-phase (us): 11008 x 4096: 49 / 51 at 33 tokens, 52 / 52 at 64, 58 / 54 at 128, 75 / 59 at 256, 114 / 78 at 512;
+// 4096 x 11008: 122 / 82 at 33, 123 / 83 at 64, 147 / 86 at 256, 144 / 89 at 512; 4096 x 4096: 51 / 36 at 33, 53 / 35 at 64, 74 / 39 at 256;
 // 8192 x 8192: 99 / 82 at 128, 117 / 84 at 256, 116 / 92 at 512; 28672 x 8192 (224 tiles on 148 SMs): 180 / 228 at 128,
 // 207 / 239 at 256, 361 / 307 at 384, 374 / 312 at 512.
 constexpr int kExpandAlwaysTokens = 257;   // more than one token tile of the fused kernel
-constexpr int kExpandMinTokens = 64;       // ... where the fused kernel's tiles leave SMs idle
+constexpr int kExpandMinTokens = 33;       // ... every call of this path where the fused kernel's tiles leave SMs idle
 static bool wants_expansion(const gwq_packed* P, int M) {
 #ifdef GWQ_TUNE_EXPAND_MIN
   return M >= GWQ_TUNE_EXPAND_MIN;

@@ -85,14 +85,14 @@ def test_tensor_core_path(layer, M, dtype):
     bits16, xv = synth.make_activations(M, P.K, seed=100 + M, dtype=dtype, heavy_channels=8)
     y_ref, bound = orc.linear(xv, w_hat)
     x = x_tensor(bits16, dtype)
-    y = gwq.gwq_linear(P, x, out_dtype=torch.float32)     # the binding's workspace: two-phase from 64 tokens on
+    y = gwq.gwq_linear(P, x, out_dtype=torch.float32)     # the binding's workspace: the two-phase path
     assert gwq.gwq_device_status(P) == 0
     assert_linear_close(y, y_ref, bound)
     # the fused kernel: a workspace without room for the expanded weights (none at all for fp16 activations)
     lib = gwq.load_library()
     xd = gwq.GWQ_F16 if dtype == "f16" else gwq.GWQ_BF16
-    small = int(lib.gwq_linear_workspace_bytes(P._h, xd, 33))   # 33 tokens never expand: the fp16 copy of x only
-    ws_bytes = max(small, 0) * ((M + 32) // 33 + 1) if small else 0
+    # room for the fp16 copy of bf16 activations and the token scales, none for the weights
+    ws_bytes = ((M * P.K * 2 + 255) // 256 + (M * 4 + 255) // 256) * 256 if dtype == "bf16" else 0
     ws = torch.empty(max(ws_bytes, 256), dtype=torch.uint8, device=x.device)
     yf = torch.zeros((M, P.N), dtype=torch.float32, device=x.device)
     st = lib.gwq_linear_ws(P._h, x.data_ptr(), xd, M, yf.data_ptr(), gwq.GWQ_F32, ws.data_ptr() if ws_bytes else None,
