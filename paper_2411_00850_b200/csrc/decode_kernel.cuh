@@ -153,19 +153,21 @@ __device__ __forceinline__ void step_raw4(const unsigned (&qa)[4], const unsigne
                                           const unsigned (&xr)[NB][16], AccRaw4<NB>& acc) {
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
-    const unsigned ta = qa[i] >> 8, tb = qb[i] >> 8;
+    // pairs 4i, 4i+1 end at position 0 and pairs 4i+2, 4i+3 at position 4, so that the two k-halves of an MMA are
+    // neighbouring words of the activation segment (one 64-bit register pair of the 128-bit load)
+    const unsigned ta4 = qa[i] >> 4, tb4 = qb[i] >> 4, ta8 = qa[i] >> 8, tb8 = qb[i] >> 8;
     const unsigned a00 = qa[i] & 0x000F000Fu, b00 = qb[i] & 0x000F000Fu;  // pair 4i   (position 0)
-    const unsigned a01 = qa[i] & 0x00F000F0u, b01 = qb[i] & 0x00F000F0u;  // pair 4i+1 (position 4)
-    const unsigned a02 = ta & 0x000F000Fu, b02 = tb & 0x000F000Fu;        // pair 4i+2 (position 0)
-    const unsigned a03 = ta & 0x00F000F0u, b03 = tb & 0x00F000F0u;        // pair 4i+3 (position 4)
+    const unsigned a01 = ta4 & 0x000F000Fu, b01 = tb4 & 0x000F000Fu;      // pair 4i+1 (position 0)
+    const unsigned a02 = ta4 & 0x00F000F0u, b02 = tb4 & 0x00F000F0u;      // pair 4i+2 (position 4)
+    const unsigned a03 = ta8 & 0x00F000F0u, b03 = tb8 & 0x00F000F0u;      // pair 4i+3 (position 4)
 #pragma unroll
     for (int nb = 0; nb < NB; ++nb) {
       if (i == 0) {
-        mma16816<false, true>(acc.c0[nb], a00, b00, a02, b02, xr[nb][4 * i], xr[nb][4 * i + 2]);
-        mma16816<false, true>(acc.c4[nb], a01, b01, a03, b03, xr[nb][4 * i + 1], xr[nb][4 * i + 3]);
+        mma16816<false, true>(acc.c0[nb], a00, b00, a01, b01, xr[nb][4 * i], xr[nb][4 * i + 1]);
+        mma16816<false, true>(acc.c4[nb], a02, b02, a03, b03, xr[nb][4 * i + 2], xr[nb][4 * i + 3]);
       } else {
-        mma16816<false, false>(acc.c0[nb], a00, b00, a02, b02, xr[nb][4 * i], xr[nb][4 * i + 2]);
-        mma16816<false, false>(acc.c4[nb], a01, b01, a03, b03, xr[nb][4 * i + 1], xr[nb][4 * i + 3]);
+        mma16816<false, false>(acc.c0[nb], a00, b00, a01, b01, xr[nb][4 * i], xr[nb][4 * i + 1]);
+        mma16816<false, false>(acc.c4[nb], a02, b02, a03, b03, xr[nb][4 * i + 2], xr[nb][4 * i + 3]);
       }
     }
   }
