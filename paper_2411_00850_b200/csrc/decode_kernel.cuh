@@ -129,8 +129,8 @@ __device__ __forceinline__ unsigned sub_zero_bf16(unsigned qm, unsigned zm) {
 //
 // Raw variant (fp16 activations).  The masked code bits are used directly as fp16 subnormals:
 // a code at mantissa bit position p is the number q 2^(p-24).  Integer instructions are the
-// scarce resource of this kernel (half-rate pipe), so codes are masked where they sit and only
-// one shift per word moves the upper byte down; the positions that occur (0 and 4 for 4 bits,
+// scarce resource of this kernel (half-rate pipe), so codes are masked where a shift or two per
+// word has put them, not moved one by one; the positions that occur (0 and 4 for 4 bits,
 // 0, 3 and 6 for 3 bits) each get their own accumulator, merged with the right power of two in
 // the group epilogue.
 template <int NB>
