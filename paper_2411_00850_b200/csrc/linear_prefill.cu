@@ -554,10 +554,11 @@ __device__ __forceinline__ void umma_commit_pair(unsigned bar) {
 // band of the weights (which stays in L2 for the whole band) and a few token tiles, instead of all of the weights
 // for every group of token tiles.
 constexpr int kBandTiles = 8;   // (4 to 16 measure alike; one band of all the weight tiles is 7 % slower)
-__device__ __forceinline__ void pair_tile(int t, int ntn, int ntm, int& tn, int& tm) {
+__host__ __device__ __forceinline__ void pair_tile(int t, int ntn, int ntm, int& tn, int& tm) {
   const int per_band = kBandTiles * ntm;
   const int band = t / per_band, i = t - band * per_band;
-  const int width = min(kBandTiles, ntn - band * kBandTiles);   // the last band may be narrower
+  const int left = ntn - band * kBandTiles;
+  const int width = kBandTiles < left ? kBandTiles : left;   // the last band may be narrower
   tm = i / width;
   tn = band * kBandTiles + (i - tm * width);
 }
@@ -578,7 +579,8 @@ struct PairArgs {
 template <int TOK>
 __global__ void __launch_bounds__(kPairThreads, 1)
 pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUtensorMap tmw,
-            const __grid_constant__ CUtensorMap tmy, const PairArgs p, const int ntn, const int ntiles, const int pairs) {
+            const __grid_constant__ CUtensorMap tmy, const __grid_constant__ CUtensorMap tmp, const PairArgs p, const int ntn,
+            const int ntiles, const int pairs, const int split) {
   constexpr int kHalfBytes = kTileN * kBlockK * 2;   // 16 KB: 128 rows x 128 bytes
   constexpr int kPairStages = PairCfg<TOK>::kStages, kPairStageBytes = PairCfg<TOK>::kStageBytes, kPairTok = TOK;
   extern __shared__ unsigned char smem_dyn[];
@@ -603,8 +605,24 @@ pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUt
   auto a_tile = [&](int s) { return tiles + (size_t)s * kPairStageBytes; };
   auto b_tile = [&](int s) { return tiles + (size_t)s * kPairStageBytes + kHalfBytes; };
   unsigned char* out_stage = tiles + (size_t)kPairStages * kPairStageBytes;   // two tiles of 32 tokens x 128 features
-  const int my_tiles = pair < ntiles ? (ntiles - 1 - pair) / pairs + 1 : 0;
   const int ntm = ntiles / ntn;   // token tiles
+  // Work items of this pair: the tiles pair, pair + pairs, ... of the full rounds; then, when the tiles left over for
+  // the last round are at most half as many as the pairs (split > 1), one K-slice of a left-over tile (its partial sums
+  // go to the workspace as FP32 and a second kernel adds the slices), else that tile whole.
+  const int full_rounds = ntiles / pairs, rem = ntiles - full_rounds * pairs;
+  const bool sliced = split > 1 && pair < rem * split;
+  const int my_items = full_rounds + ((split > 1 ? sliced : pair < rem) ? 1 : 0);
+  auto item = [&](int w, int& tile, int& kb0, int& kb1) {   // returns true for a K-slice
+    if (w < full_rounds || split <= 1) {
+      tile = pair + w * pairs; kb0 = 0; kb1 = nkb;
+      return false;
+    }
+    const int sl = pair % split;
+    tile = full_rounds * pairs + pair / split;
+    kb0 = (int)((long long)nkb * sl / split);
+    kb1 = (int)((long long)nkb * (sl + 1) / split);
+    return true;
+  };
 
   if (tid == 0) {
     abort_s = 0;
@@ -635,13 +653,15 @@ pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUt
   if (warp == 0) {
     // ------------------------------------------------------------------ this CTA's halves of the operand tiles by TMA
     if (lane == 0) {
-      for (int ti = 0; ti < my_tiles && ok; ++ti) {
-        int tn, tm;
-        pair_tile(pair + ti * pairs, ntn, ntm, tn, tm);
+      int it = 0;
+      for (int w = 0; w < my_items && ok; ++w) {
+        int tile, kb0, kb1, tn, tm;
+        item(w, tile, kb0, kb1);
+        pair_tile(tile, ntn, ntm, tn, tm);
         const int n0 = tn * (2 * kTileN) + (int)rank * kTileN;
         const int m0 = tm * kPairTok + (int)rank * (kPairTok / 2);
-        for (int kb = 0; kb < nkb && ok; ++kb) {
-          const int it = ti * nkb + kb, s = it % kPairStages, round = it / kPairStages;
+        for (int kb = kb0; kb < kb1 && ok; ++kb, ++it) {
+          const int s = it % kPairStages, round = it / kPairStages;
           if (round > 0) ok = mbar_wait(empty(s), (round - 1) & 1, abort_flag, lim);
           if (!ok) break;
           if (rank == 0) mbar_expect_tx(full(s), 2 * kPairStageBytes);   // both CTAs' halves
@@ -657,21 +677,24 @@ pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUt
     if (lane == 0 && rank == 0) {
       // instruction descriptor: FP32 accumulate, A and B fp16, K-major, N = 256, M = 256 (128 rows per CTA)
       const unsigned idesc = (1u << 4) | ((unsigned)(kPairTok >> 3) << 17) | ((unsigned)((2 * kTileN) >> 4) << 24);
-      for (int ti = 0; ti < my_tiles && ok; ++ti) {
-        const int a = ti & 1;
-        if (ti >= 2) ok = mbar_wait(acc_empty(a), ((ti >> 1) - 1) & 1, abort_flag, lim);   // drained by both epilogues
+      int it = 0;
+      for (int w = 0; w < my_items && ok; ++w) {
+        int tile, kb0, kb1;
+        item(w, tile, kb0, kb1);
+        const int a = w & 1;
+        if (w >= 2) ok = mbar_wait(acc_empty(a), ((w >> 1) - 1) & 1, abort_flag, lim);   // drained by both epilogues
         if (!ok) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const unsigned acc = tmem_acc + (unsigned)(a * kPairTok);
-        for (int kb = 0; kb < nkb && ok; ++kb) {
-          const int it = ti * nkb + kb, s = it % kPairStages, round = it / kPairStages;
+        for (int kb = kb0; kb < kb1 && ok; ++kb, ++it) {
+          const int s = it % kPairStages, round = it / kPairStages;
           ok = mbar_wait(full(s), round & 1, abort_flag, lim);
           if (!ok) break;
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           const uint64_t da = umma_desc(smem_u32(a_tile(s))), db = umma_desc(smem_u32(b_tile(s)));
 #pragma unroll
           for (int k = 0; k < kBlockK / 16; ++k)   // 32 bytes further along K inside the swizzle atom
-            umma_f16_pair(acc, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (kb | k) != 0);
+            umma_f16_pair(acc, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (kb > kb0 || k != 0) ? 1u : 0u);
           umma_commit_pair(empty(s));
         }
         if (ok) umma_commit_pair(acc_full(a));
@@ -682,13 +705,14 @@ pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUt
     const int quad = warp & 3;                 // tensor-memory lane quarter this warp may access
     const int r = quad * 32 + lane;
     int chunk = 0;                             // chunks handed to the TMA store so far
-    for (int ti = 0; ti < my_tiles && ok; ++ti) {
-      int tn, tm;
-      pair_tile(pair + ti * pairs, ntn, ntm, tn, tm);
+    for (int w = 0; w < my_items && ok; ++w) {
+      int tile, kb0, kb1, tn, tm;
+      const bool slice = item(w, tile, kb0, kb1);
+      pair_tile(tile, ntn, ntm, tn, tm);
       const int row = tn * (2 * kTileN) + (int)rank * kTileN + r, m0 = tm * kPairTok;
       const bool live = row < p.N;
-      const int a = ti & 1;
-      ok = mbar_wait_warp(acc_full(a), (ti >> 1) & 1, abort_flag, lim);
+      const int a = w & 1;
+      ok = mbar_wait_warp(acc_full(a), (w >> 1) & 1, abort_flag, lim);
       {   // one verdict for the four epilogue warps: they meet at barriers inside the tile
         unsigned all;
         asm volatile("{\n .reg .pred q, r;\n setp.ne.b32 q, %1, 0;\n bar.red.and.pred r, 1, 128, q;\n selp.b32 %0, 1, 0, r;\n}\n"
@@ -703,7 +727,7 @@ pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUt
         unsigned v[32];
         tmem_ld32(tmem_acc + ((unsigned)(quad * 32) << 16) + (unsigned)(a * kPairTok + c0), v);
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-        if (p.tma_store) {
+        if (p.tma_store || slice) {
           // the chunk goes through a shared-memory tile [32 tokens][128 features] (two of them, used in turn)
           unsigned char* st = out_stage + (chunk & 1) * kOutStageBytes;
           if (chunk >= 2) {   // the store that read this tile two chunks ago has finished reading it
@@ -727,7 +751,10 @@ pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUt
 #pragma unroll
             for (int i = 0; i < 32; ++i) ts[i] = 1.f;
           }
-          if (p.yd == GWQ_F32) {
+          if (slice) {   // raw FP32 partial sums of this K-slice; scale and conversion follow in the second kernel
+#pragma unroll
+            for (int i = 0; i < 32; ++i) reinterpret_cast<unsigned*>(st)[i * kTileN + r] = v[i];
+          } else if (p.yd == GWQ_F32) {
 #pragma unroll
             for (int i = 0; i < 32; ++i) reinterpret_cast<float*>(st)[i * kTileN + r] = __uint_as_float(v[i]) * ts[i];
           } else {
@@ -753,7 +780,12 @@ pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUt
           }
           asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to the TMA
           asm volatile("bar.sync 1, 128;" ::: "memory");
-          if (warp == 2 && lane == 0) {   // rows past N and tokens past M are clipped by the copy
+          if (warp == 2 && lane == 0 && slice) {   // slot `pair` of the partial tiles: [TOK tokens][256 features] FP32
+            asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+                         ::"l"(&tmp), "r"((int)rank * kTileN), "r"(pair * kPairTok + c0), "r"(smem_u32(st))
+                         : "memory");
+            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+          } else if (warp == 2 && lane == 0) {   // rows past N and tokens past M are clipped by the copy
             // y is written once and not read again here: its lines are the first to leave L2, not the operands'
             asm volatile(
                 "{\n .reg .b64 pol;\n createpolicy.fractional.L2::evict_first.b64 pol, 1.0;\n"
@@ -815,10 +847,52 @@ pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUt
   }
 }
 
+// K-slices of a left-over tile: split = pairs / left-over tiles when these are at most half as many as the pairs
+// (at least 8 k-blocks per slice, at most 8 slices) and the slices save more than adding them up costs, else 1.
+static int pair_split(int ntiles, int pairs, int nkb) {
+  const int rem = ntiles % pairs;
+  if (rem == 0 || 2 * rem > pairs) return 1;
+  int split = pairs / rem;
+  if (split > 8) split = 8;
+  while (split > 1 && nkb / split < 8) --split;
+  // the second kernel and the partial tiles cost about as much as 43 k-blocks of a tile (measured: 4096 x 4096 at 512
+  // tokens, two slices of 32 k-blocks: 47 against 41 us; 11008 x 4096, six slices: 75 against 80 us; 4096 x 11008, two
+  // slices of 86: 83 against 93 us, 65 against 90 us at 256 tokens)
+  if ((long long)nkb * (split - 1) < 43LL * split) return 1;
+  return split;
+}
+// bytes of the FP32 partial tiles: one slot of TOK tokens x 256 features per pair
+static size_t pair_partial_bytes(int sms) { return (size_t)(sms / 2 > 0 ? sms / 2 : 1) * 256 * 256 * sizeof(float); }
+
+// Adds the K-slices of the left-over tiles (slots t split .. t split + split - 1 of left-over tile t, in slice order:
+// the same bits every time), applies the token scale and stores y.  One CTA per tile and 4 tokens, one thread per
+// (feature, token); the loads of a sum are requested together.
+template <int TOK>
+__global__ void __launch_bounds__(1024) pair_fixup_kernel(const float* __restrict__ partial, void* y, gwq_dtype yd,
+                                                          const float* __restrict__ tok_scale, int N, int M, int ntn, int ntm,
+                                                          int first_tile, int split) {
+  int tn, tm;
+  pair_tile(first_tile + blockIdx.x, ntn, ntm, tn, tm);
+  const int n = tn * 256 + threadIdx.x, ml = blockIdx.y * 4 + threadIdx.y, m = tm * TOK + ml;
+  if (n >= N || m >= M) return;
+  const float* src = partial + ((size_t)blockIdx.x * split * TOK + ml) * 256 + threadIdx.x;
+  float t[8];
+#pragma unroll
+  for (int sl = 0; sl < 8; ++sl) t[sl] = sl < split ? __ldg(src + (size_t)sl * TOK * 256) : 0.f;
+  float v = t[0];
+#pragma unroll
+  for (int sl = 1; sl < 8; ++sl) v += t[sl];   // slice order
+  if (tok_scale) v *= __ldg(tok_scale + m);
+  const size_t idx = (size_t)m * N + n;
+  if (yd == GWQ_F32) reinterpret_cast<float*>(y)[idx] = v;
+  else if (yd == GWQ_F16) reinterpret_cast<__half*>(y)[idx] = __float2half_rn(v);
+  else reinterpret_cast<__nv_bfloat16*>(y)[idx] = __float2bfloat16_rn(v);
+}
+
 // Launch of the pair kernel on the expanded weights w16 [N][K] and fp16 activations x [M][K].
 template <int TOK>
-gwq_status launch_pairs_tok(const gwq_packed* P, const void* x, const float* tok_scale, const void* w16, int M, void* y,
-                        gwq_dtype yd, cudaStream_t stream) {
+gwq_status launch_pairs_tok(const gwq_packed* P, const void* x, const float* tok_scale, const void* w16, float* partial, int M,
+                            void* y, gwq_dtype yd, cudaStream_t stream) {
   const gwq_priv* pv = static_cast<const gwq_priv*>(P->priv);
   EncodeTiledFn enc = encode_fn();
   if (!enc) return GWQ_ERR_CUDA;
@@ -855,6 +929,16 @@ gwq_status launch_pairs_tok(const gwq_packed* P, const void* x, const float* tok
             CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return GWQ_ERR_CUDA;
   }
+  CUtensorMap tmp = tmx;   // FP32 partial tiles: rows = slot * TOK + token, 256 features each
+  if (partial) {
+    const int slots = pv->sm_count / 2 > 0 ? pv->sm_count / 2 : 1;
+    const cuuint64_t dims[2] = {256, (cuuint64_t)slots * TOK};
+    const cuuint64_t strides[1] = {256 * sizeof(float)};
+    const cuuint32_t obox[2] = {(cuuint32_t)kTileN, 32};
+    if (enc(&tmp, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, partial, dims, strides, obox, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return GWQ_ERR_CUDA;
+  }
   const size_t smem = (size_t)PairCfg<TOK>::kStages * PairCfg<TOK>::kStageBytes + 2 * kOutStageBytes + 1024;
   if (cudaFuncSetAttribute(pair_kernel<TOK>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return GWQ_ERR_CUDA;
   PairArgs a;
@@ -889,27 +973,39 @@ gwq_status launch_pairs_tok(const gwq_packed* P, const void* x, const float* tok
   }
   if (resident < 1) return GWQ_ERR_UNSUPPORTED;
   int pairs = resident < pv->sm_count / 2 ? resident : pv->sm_count / 2;
-  if (pairs > ntiles) pairs = ntiles;
+  const int split = partial ? pair_split(ntiles, pairs, P->K / kBlockK) : 1;   // fewer tiles than pairs: all of them left over
+  if (split == 1 && pairs > ntiles) pairs = ntiles;
   cfg.gridDim = dim3(2u * (unsigned)pairs);
-  if (cudaLaunchKernelEx(&cfg, pair_kernel<TOK>, tmx, tmw, tmy, a, ntn, ntiles, pairs) != cudaSuccess) {
+  if (cudaLaunchKernelEx(&cfg, pair_kernel<TOK>, tmx, tmw, tmy, tmp, a, ntn, ntiles, pairs, split) != cudaSuccess) {
     (void)cudaGetLastError();
     return GWQ_ERR_CUDA;
+  }
+  if (split > 1) {
+    const int rem = ntiles % pairs;
+    pair_fixup_kernel<TOK><<<dim3((unsigned)rem, TOK / 4), dim3(256, 4), 0, stream>>>(partial, y, yd, tok_scale, P->N, M, ntn, ntiles / ntn,
+                                                                          ntiles - rem, split);
+    if (cudaGetLastError() != cudaSuccess) return GWQ_ERR_CUDA;
   }
   return GWQ_OK;
 }
 
-// Tokens per tile: the pairs work in rounds of one tile each.  A 128-token tile loads 24 KB per k-block for half the
-// multiplies of a 256-token tile's 32 KB, and the operands come out of L2, so it takes about 0.8 of the time, not half
-// (measured, 512 tokens: 66 against 76 us where both need one round, 4096 x 11008; 69 against 64 us with three
-// rounds against two, 11008 x 4096): it is taken only where it needs hardly more rounds than the larger tile.
-gwq_status launch_pairs(const gwq_packed* P, const void* x, const float* tok_scale, const void* w16, int M, void* y, gwq_dtype yd,
-                        cudaStream_t stream) {
+// Tokens per tile: the pairs work in rounds of one tile each (the last round in K-slices when few tiles are left over).
+// A 128-token tile loads 24 KB per k-block for half the multiplies of a 256-token tile's 32 KB, and the operands come
+// out of L2, so it takes about 0.8 of the time, not half (measured, 512 tokens: 66 against 76 us where both need one
+// round, 4096 x 11008; 69 against 64 us with three rounds against two, 11008 x 4096): it is taken only where it needs
+// hardly more rounds than the larger tile.
+gwq_status launch_pairs(const gwq_packed* P, const void* x, const float* tok_scale, const void* w16, float* partial, int M, void* y,
+                        gwq_dtype yd, cudaStream_t stream) {
   const gwq_priv* pv = static_cast<const gwq_priv*>(P->priv);
-  const long long pairs = pv->sm_count / 2 > 0 ? pv->sm_count / 2 : 1;
-  const long long ntn = (P->N + 2 * kTileN - 1) / (2 * kTileN);
-  const long long r256 = (ntn * ((M + 255) / 256) + pairs - 1) / pairs, r128 = (ntn * ((M + 127) / 128) + pairs - 1) / pairs;
-  if (4 * r128 < 5 * r256) return launch_pairs_tok<128>(P, x, tok_scale, w16, M, y, yd, stream);
-  return launch_pairs_tok<256>(P, x, tok_scale, w16, M, y, yd, stream);
+  const int pairs = pv->sm_count / 2 > 0 ? pv->sm_count / 2 : 1;
+  const int ntn = (P->N + 2 * kTileN - 1) / (2 * kTileN), nkb = P->K / kBlockK;
+  auto rounds = [&](int tok) {   // in units of one tile's time
+    const int ntiles = ntn * ((M + tok - 1) / tok);
+    const int split = partial ? pair_split(ntiles, pairs, nkb) : 1;
+    return (double)(ntiles / pairs) + (ntiles % pairs ? 1.0 / split : 0.0);
+  };
+  if (0.8 * rounds(128) < rounds(256)) return launch_pairs_tok<128>(P, x, tok_scale, w16, partial, M, y, yd, stream);
+  return launch_pairs_tok<256>(P, x, tok_scale, w16, partial, M, y, yd, stream);
 }
 
 template <int BITS, int TOK, int GPK = 1>
@@ -1054,8 +1150,8 @@ static bool wants_expansion(const gwq_packed* P, int M) {
 }
 
 // Expanded weights: the expansion, the outliers over it, then the contraction with token tiles of 256.
-gwq_status launch_expanded(const gwq_packed* P, const void* x, const float* tok_scale, uint16_t* w16, int M, void* y,
-                           gwq_dtype yd, cudaStream_t stream) {
+gwq_status launch_expanded(const gwq_packed* P, const void* x, const float* tok_scale, uint16_t* w16, float* partial, int M,
+                           void* y, gwq_dtype yd, cudaStream_t stream) {
   const gwq_priv* pv = static_cast<const gwq_priv*>(P->priv);
   if (pv->ob && pv->ob_ptr && P->K % 128 == 0) {
     const unsigned blocks = (unsigned)((P->N + 127) / 128) * (unsigned)(P->K / 128);
@@ -1072,7 +1168,7 @@ gwq_status launch_expanded(const gwq_packed* P, const void* x, const float* tok_
     expand_outliers_kernel<<<(P->N + 7) / 8, 256, 0, stream>>>(P->S->row_ptr, pv->cv, w16, P->N, P->K);
   }
   if (cudaGetLastError() != cudaSuccess) return GWQ_ERR_CUDA;
-  return launch_pairs(P, x, tok_scale, w16, M, y, yd, stream);
+  return launch_pairs(P, x, tok_scale, w16, partial, M, y, yd, stream);
 }
 
 }  // namespace
@@ -1086,7 +1182,9 @@ static size_t x16_bytes(const gwq_packed* P, gwq_dtype xd, int M) {
 size_t gwq_prefill_workspace_bytes(const gwq_packed* P, gwq_dtype xd, int M) {
   const gwq_priv* pv = static_cast<const gwq_priv*>(P->priv);
   if (!pv->cv || !pv->sz_t || P->K % kBlockK != 0) return 0;   // the general kernel needs none
-  return x16_bytes(P, xd, M) + (wants_expansion(P, M) ? (((size_t)P->N * P->K * 2 + 255) & ~(size_t)255) : 0);
+  // (the expanded weights are followed by the FP32 partial tiles of the K-slices)
+  return x16_bytes(P, xd, M) +
+         (wants_expansion(P, M) ? (((size_t)P->N * P->K * 2 + 255) & ~(size_t)255) + pair_partial_bytes(pv->sm_count) : 0);
 }
 
 // Prefill launcher: K <= 65536 (16-bit outlier columns).  Other shapes go to the general kernel.
@@ -1109,7 +1207,9 @@ gwq_status gwq_launch_prefill(const gwq_packed* P, const void* x, gwq_dtype xd, 
   }
   if (wants_expansion(P, M) && ws && ws_bytes >= gwq_prefill_workspace_bytes(P, xd, M))
   {
-    const gwq_status st = launch_expanded(P, x, tok_scale, reinterpret_cast<uint16_t*>(static_cast<char*>(ws) + xb), M, y, yd, stream);
+    char* w16 = static_cast<char*>(ws) + xb;
+    float* partial = reinterpret_cast<float*>(w16 + (((size_t)P->N * P->K * 2 + 255) & ~(size_t)255));
+    const gwq_status st = launch_expanded(P, x, tok_scale, reinterpret_cast<uint16_t*>(w16), partial, M, y, yd, stream);
     if (st != GWQ_ERR_UNSUPPORTED) return st;   // a device that holds no cluster of two such CTAs: the fused kernel
   }
   if (P->bits == 4) return launch_tok<4>(P, x, tok_scale, M, y, yd, stream);

@@ -137,12 +137,14 @@ def test_persistent_ctas_with_several_tiles_each(bits, dtype, expanded):
 
 
 @pytest.mark.parametrize("N,K,M,bits,dtype", [(600, 320, 2300, 4, "f16"), (2700, 192, 2100, 3, "bf16"), (96, 64, 2048, 4, "f16"),
-                                                   (600, 384, 2300, 4, "bf16"), (300, 256, 2100, 3, "f16"), (9472, 128, 512, 4, "f16")])
+                                                   (600, 384, 2300, 4, "bf16"), (300, 256, 2100, 3, "f16"), (9472, 128, 512, 4, "f16"),
+                                                   (1500, 4096, 700, 4, "bf16"), (2560, 6144, 520, 3, "f16"), (520, 4096, 300, 4, "f16")])
 def test_two_phase_path_ragged_tiles_and_bands(N, K, M, bits, dtype):
     # the contraction on CTA pairs (tiles of 256 rows x 256 tokens, reached with many tokens and room for the
     # expanded weights): ragged last tiles in both directions, 11 weight tiles (a full band of 8 and a narrower one),
     # a layer smaller than one tile; K a multiple of 128 (the weights expanded block by block) and not; token tiles of
-    # 128 (the small layers) and of 256 (9472 rows x 512 tokens: one tile per pair of SMs); every output
+    # 128 (the small layers) and of 256 (9472 rows x 512 tokens: one tile per pair of SMs); left-over tiles cut into
+    # K-slices whose partial sums a second kernel adds (the last three: 18, 30 and 6 tiles on 74 pairs); every output
     W, G = synth.make_weight_and_grad(N, K, 27)
     L = orc.quantize_layer(W, G, 0.01, bits, 64)
     P = quantize_on_gpu(W, G, 0.01, bits, 64)
