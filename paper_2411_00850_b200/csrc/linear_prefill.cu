@@ -576,7 +576,9 @@ struct PairArgs {
 // tmx: x16 [M][K] with boxes of 64 columns x 128 rows; tmw: expanded weights [N][K], same boxes.
 // tmy: y [M][N] with boxes of 128 output features x 32 tokens.
 // ntn: tiles of 256 weight rows; ntiles: all tiles (order: pair_tile); pairs: clusters of the launch.
-template <int TOK>
+// SLICED: the left-over tiles of the last round are cut into `split` K-slices (a build of its own, so that the
+// common case carries none of it).
+template <int TOK, bool SLICED>
 __global__ void __launch_bounds__(kPairThreads, 1)
 pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUtensorMap tmw,
             const __grid_constant__ CUtensorMap tmy, const __grid_constant__ CUtensorMap tmp, const PairArgs p, const int ntn,
@@ -610,10 +612,9 @@ pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUt
   // the last round are at most half as many as the pairs (split > 1), one K-slice of a left-over tile (its partial sums
   // go to the workspace as FP32 and a second kernel adds the slices), else that tile whole.
   const int full_rounds = ntiles / pairs, rem = ntiles - full_rounds * pairs;
-  const bool sliced = split > 1 && pair < rem * split;
-  const int my_items = full_rounds + ((split > 1 ? sliced : pair < rem) ? 1 : 0);
+  const int my_items = full_rounds + ((SLICED ? pair < rem * split : pair < rem) ? 1 : 0);
   auto item = [&](int w, int& tile, int& kb0, int& kb1) {   // returns true for a K-slice
-    if (w < full_rounds || split <= 1) {
+    if (!SLICED || w < full_rounds) {
       tile = pair + w * pairs; kb0 = 0; kb1 = nkb;
       return false;
     }
@@ -707,7 +708,7 @@ pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUt
     int chunk = 0;                             // chunks handed to the TMA store so far
     for (int w = 0; w < my_items && ok; ++w) {
       int tile, kb0, kb1, tn, tm;
-      const bool slice = item(w, tile, kb0, kb1);
+      const bool slice = item(w, tile, kb0, kb1) && SLICED;
       pair_tile(tile, ntn, ntm, tn, tm);
       const int row = tn * (2 * kTileN) + (int)rank * kTileN + r, m0 = tm * kPairTok;
       const bool live = row < p.N;
@@ -940,7 +941,9 @@ gwq_status launch_pairs_tok(const gwq_packed* P, const void* x, const float* tok
       return GWQ_ERR_CUDA;
   }
   const size_t smem = (size_t)PairCfg<TOK>::kStages * PairCfg<TOK>::kStageBytes + 2 * kOutStageBytes + 1024;
-  if (cudaFuncSetAttribute(pair_kernel<TOK>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return GWQ_ERR_CUDA;
+  if (cudaFuncSetAttribute(pair_kernel<TOK, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
+      cudaFuncSetAttribute(pair_kernel<TOK, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+    return GWQ_ERR_CUDA;
   PairArgs a;
   a.y = y; a.yd = yd; a.status = pv->dev_status; a.tok_scale = tok_scale; a.N = P->N; a.K = P->K; a.M = M;
   a.tma_store = tma_store;
@@ -965,7 +968,7 @@ gwq_status launch_pairs_tok(const gwq_packed* P, const void* x, const float* tok
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) dev = 63;
   int resident = resident_on[dev].load(std::memory_order_relaxed);
   if (resident == 0) {
-    if (cudaOccupancyMaxActiveClusters(&resident, pair_kernel<TOK>, &cfg) != cudaSuccess || resident < 1) {
+    if (cudaOccupancyMaxActiveClusters(&resident, pair_kernel<TOK, false>, &cfg) != cudaSuccess || resident < 1) {
       (void)cudaGetLastError();
       resident = -1;
     }
@@ -976,7 +979,9 @@ gwq_status launch_pairs_tok(const gwq_packed* P, const void* x, const float* tok
   const int split = partial ? pair_split(ntiles, pairs, P->K / kBlockK) : 1;   // fewer tiles than pairs: all of them left over
   if (split == 1 && pairs > ntiles) pairs = ntiles;
   cfg.gridDim = dim3(2u * (unsigned)pairs);
-  if (cudaLaunchKernelEx(&cfg, pair_kernel<TOK>, tmx, tmw, tmy, tmp, a, ntn, ntiles, pairs, split) != cudaSuccess) {
+  const cudaError_t le = split > 1 ? cudaLaunchKernelEx(&cfg, pair_kernel<TOK, true>, tmx, tmw, tmy, tmp, a, ntn, ntiles, pairs, split)
+                                   : cudaLaunchKernelEx(&cfg, pair_kernel<TOK, false>, tmx, tmw, tmy, tmp, a, ntn, ntiles, pairs, split);
+  if (le != cudaSuccess) {
     (void)cudaGetLastError();
     return GWQ_ERR_CUDA;
   }
