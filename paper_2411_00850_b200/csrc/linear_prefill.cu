@@ -30,6 +30,26 @@
 namespace {
 using namespace gwq_tc;
 
+// The kernels of the two-phase path are launched with programmatic stream serialization: each lets its successor
+// start at once (griddepcontrol.launch_dependents) and waits for its predecessor to complete (griddepcontrol.wait)
+// before it touches anything a kernel before it writes or still reads; what depends on the weights alone comes first.
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;"); }
+__device__ __forceinline__ void pdl_sync() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+template <class... KArgs, class... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args... args) {
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 constexpr int kTileN = 128;      // weight rows per CTA (UMMA M)
 constexpr int kBlockK = 64;      // k-block: 128 bytes of 16-bit operands
 constexpr int kDequantWarps = 4;   // warps of one dequantisation group (one thread per tile row)
@@ -58,6 +78,8 @@ struct PrefillArgs {
 __global__ void __launch_bounds__(256) bf16_rows_to_scaled_f16(const uint16_t* __restrict__ x, uint16_t* __restrict__ x16,
                                                                float* __restrict__ tok_scale, int K) {
   __shared__ float red[8];
+  pdl_trigger();
+  pdl_sync();   // x may still be being written
   const uint16_t* row = x + (size_t)blockIdx.x * K;
   uint16_t* out = x16 + (size_t)blockIdx.x * K;
   unsigned amax = 0;   // largest |x| as a bf16 bit pattern (monotone in magnitude)
@@ -648,6 +670,8 @@ pair_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUt
   cluster_sync_all();   // both CTAs' barriers exist before either signals the other
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const unsigned tmem_acc = tmem_base_s;
+  pdl_trigger();
+  pdl_sync();   // the operands are written, and y may still be read, by the kernels before
   bool ok = *reinterpret_cast<volatile int32_t*>(p.status) == 0;   // an earlier CTA gave up: do no work
   int issued = 0;   // k-block copies started (producer thread only), counted over all tiles
 
@@ -872,6 +896,8 @@ template <int TOK>
 __global__ void __launch_bounds__(1024) pair_fixup_kernel(const float* __restrict__ partial, void* y, gwq_dtype yd,
                                                           const float* __restrict__ tok_scale, int N, int M, int ntn, int ntm,
                                                           int first_tile, int split) {
+  pdl_trigger();
+  pdl_sync();
   int tn, tm;
   pair_tile(first_tile + blockIdx.x, ntn, ntm, tn, tm);
   const int n = tn * 256 + threadIdx.x, ml = blockIdx.y * 4 + threadIdx.y, m = tm * TOK + ml;
@@ -949,17 +975,19 @@ gwq_status launch_pairs_tok(const gwq_packed* P, const void* x, const float* tok
   a.tma_store = tma_store;
   a.wait_cycles = pv->wait_cycles;
   const int ntn = (P->N + 2 * kTileN - 1) / (2 * kTileN), ntiles = ntn * ((M + TOK - 1) / TOK);
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 2;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cudaLaunchConfig_t cfg = {};
   cfg.blockDim = dim3(kPairThreads);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = stream;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = 2;
   // persistent: as many pairs as the device holds at once (pairs sit inside one GPC, so this may be fewer than SMs / 2)
   cfg.gridDim = dim3(2u * (unsigned)(pv->sm_count / 2));
   // (asked once per device and token-tile size: the answer depends on nothing else)
@@ -987,9 +1015,11 @@ gwq_status launch_pairs_tok(const gwq_packed* P, const void* x, const float* tok
   }
   if (split > 1) {
     const int rem = ntiles % pairs;
-    pair_fixup_kernel<TOK><<<dim3((unsigned)rem, TOK / 4), dim3(256, 4), 0, stream>>>(partial, y, yd, tok_scale, P->N, M, ntn, ntiles / ntn,
-                                                                          ntiles - rem, split);
-    if (cudaGetLastError() != cudaSuccess) return GWQ_ERR_CUDA;
+    if (launch_pdl(pair_fixup_kernel<TOK>, dim3((unsigned)rem, TOK / 4), dim3(256, 4), 0, stream, (const float*)partial, y, yd, tok_scale,
+                   P->N, M, ntn, ntiles / ntn, ntiles - rem, split) != cudaSuccess) {
+      (void)cudaGetLastError();
+      return GWQ_ERR_CUDA;
+    }
   }
   return GWQ_OK;
 }
@@ -1074,6 +1104,7 @@ __global__ void __launch_bounds__(256) expand_block_kernel(const uint32_t* __res
                                                            uint16_t* __restrict__ w16, int N, int K, int group) {
   constexpr int kPitch = 128 + 8;                  // halves per row of the tile: 16 bytes of padding
   __shared__ __align__(16) uint16_t tile[128 * kPitch];
+  pdl_trigger();
   const int G = K >> 7;
   const int blk = blockIdx.x, row0 = (blk / G) * 128, g = blk % G;
   const int e0 = __ldg(ob_ptr + blk), e1 = __ldg(ob_ptr + blk + 1);
@@ -1125,6 +1156,7 @@ __global__ void __launch_bounds__(256) expand_block_kernel(const uint32_t* __res
     tile[((v >> 23) & 127u) * kPitch + ((v >> 16) & 127u)] = (uint16_t)v;
   }
   __syncthreads();
+  pdl_sync();   // the workspace may still be read by the kernel before (everything above depends on the weights alone)
 #pragma unroll
   for (int u = 0; u < 8; ++u) {
     const int id = threadIdx.x + 256 * u, r = id >> 4, pc = id & 15;   // 16-byte piece pc of row r
@@ -1161,9 +1193,11 @@ gwq_status launch_expanded(const gwq_packed* P, const void* x, const float* tok_
   if (pv->ob && pv->ob_ptr && P->K % 128 == 0) {
     const unsigned blocks = (unsigned)((P->N + 127) / 128) * (unsigned)(P->K / 128);
     if (P->bits == 4)
-      expand_block_kernel<4><<<blocks, 256, 0, stream>>>(P->codes, pv->sz_t, pv->ob, pv->ob_ptr, w16, P->N, P->K, P->group);
+      (void)launch_pdl(expand_block_kernel<4>, dim3(blocks), dim3(256), 0, stream, (const uint32_t*)P->codes, (const uint32_t*)pv->sz_t,
+                       (const uint32_t*)pv->ob, (const int32_t*)pv->ob_ptr, w16, P->N, P->K, P->group);
     else
-      expand_block_kernel<3><<<blocks, 256, 0, stream>>>(P->codes, pv->sz_t, pv->ob, pv->ob_ptr, w16, P->N, P->K, P->group);
+      (void)launch_pdl(expand_block_kernel<3>, dim3(blocks), dim3(256), 0, stream, (const uint32_t*)P->codes, (const uint32_t*)pv->sz_t,
+                       (const uint32_t*)pv->ob, (const int32_t*)pv->ob_ptr, w16, P->N, P->K, P->group);
   } else {
     const long long runs = (long long)P->N * (P->K / 32);
     if (P->bits == 4)
@@ -1205,8 +1239,11 @@ gwq_status gwq_launch_prefill(const gwq_packed* P, const void* x, gwq_dtype xd, 
   if (xd == GWQ_BF16) {
     uint16_t* x16 = static_cast<uint16_t*>(ws);
     float* ts = reinterpret_cast<float*>(static_cast<char*>(ws) + (((size_t)M * P->K * 2 + 255) & ~(size_t)255));
-    bf16_rows_to_scaled_f16<<<M, 256, 0, stream>>>(static_cast<const uint16_t*>(x), x16, ts, P->K);
-    if (cudaGetLastError() != cudaSuccess) return GWQ_ERR_CUDA;
+    if (launch_pdl(bf16_rows_to_scaled_f16, dim3((unsigned)M), dim3(256), 0, stream, static_cast<const uint16_t*>(x), x16, ts, P->K) !=
+        cudaSuccess) {
+      (void)cudaGetLastError();
+      return GWQ_ERR_CUDA;
+    }
     x = x16;
     tok_scale = ts;
   }
