@@ -514,19 +514,35 @@ decode_kernel(const MultiArgs ma) {
   constexpr int kBufs = NBUF == 0 ? 1 : NBUF;
   const int tile_pieces = M * kTilePitch;
   uint4* wtile = sm_x + warp * kBufs * tile_pieces;
-  // lane L copies piece L & 15 of the token rows (L >> 4), (L >> 4) + 2, ...: constant strides, three
-  // instructions per 16-byte piece
+  // lane L copies piece L & 15 of the token rows (L >> 4), (L >> 4) + 2, ...  The place of a piece inside its row
+  // (tile_piece) takes two values only, 64 bytes apart, for the rows m and m + 2 (they differ in (m & 3) << 1), and the
+  // rows are a fixed number of bytes apart: the copies of a step cost an address each.  (Unrolled this way for 4 and 16
+  // tokens; with 8 tokens, and with 3-bit codes at 16, the plain loop measured faster: registers.)
+  constexpr bool kUnrolledCopies = TP == 4 || (TP == 16 && BITS == 4);
   const int st_m0 = lane >> 4, st_pc = lane & 15;
   const unsigned st_dst0 = (unsigned)__cvta_generic_to_shared(wtile);
+  const unsigned st_place = (unsigned)(tile_piece(st_pc, st_m0) - st_m0 * kTilePitch) * 16u;
   const uint16_t* st_src0 = ma.x + (size_t)st_m0 * K + (size_t)warp * 128 + st_pc * 8;
   auto stage_tile = [&](int c) {
     if (c < nsteps) {
       const uint16_t* src = st_src0 + (size_t)c * (kWarps * 128);
-      const unsigned dst = st_dst0 + (unsigned)((c % kBufs) * tile_pieces) * 16u;
-      for (int m = st_m0; m < M; m += 2) {
-        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + (unsigned)tile_piece(st_pc, m) * 16u),
-                     "l"(src));
-        src += 2 * (size_t)K;
+      if constexpr (kUnrolledCopies) {
+        const unsigned dst = st_dst0 + (unsigned)((c % kBufs) * tile_pieces + st_m0 * kTilePitch) * 16u;
+        const unsigned d0 = dst + st_place, d1 = dst + (st_place ^ 64u);
+#pragma unroll
+        for (int j = 0; j < (TP + 1) / 2; ++j) {   // row st_m0 + 2 j
+          if (st_m0 + 2 * j < M)
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(((j & 1) ? d1 : d0) + (unsigned)(2 * j * kTilePitch * 16)),
+                         "l"(src));
+          src += 2 * (size_t)K;
+        }
+      } else {
+        const unsigned dst = st_dst0 + (unsigned)((c % kBufs) * tile_pieces) * 16u;
+        for (int m = st_m0; m < M; m += 2) {
+          asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + (unsigned)tile_piece(st_pc, m) * 16u),
+                       "l"(src));
+          src += 2 * (size_t)K;
+        }
       }
     }
   };
