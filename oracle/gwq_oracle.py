@@ -208,8 +208,13 @@ def _bit_positions(bits: int):
             else:
                 e = i - 30               # columns 30 / 31: bit b lives in word b, bit 15 / 31
                 pos.append([(b, 16 * e + 15, b) for b in range(3)])
+        elif bits in (2, 8):
+            per = 32 // bits             # columns per word
+            t, r = divmod(i, per)        # word t holds columns per*t .. per*t + per - 1
+            j, e = divmod(r, 2)          # column per*t + 2j + e
+            pos.append([(t, 16 * e + bits * j + b, b) for b in range(bits)])
         else:
-            raise ValueError("bits must be 3 or 4")
+            raise ValueError("bits must be 2, 3, 4 or 8")
     return pos
 
 
@@ -221,6 +226,8 @@ def pack_codes(codes: np.ndarray, bits: int) -> np.ndarray:
     yields a (column 2j, column 2j+1) pair in the two halves of a register.
       4 bits: word t of a row holds columns 8t..8t+7; column 8t + 2j + e
               (j = 0..3, e = 0,1) sits in bits [16e + 4j, 16e + 4j + 4).
+      2 and 8 bits, likewise: word t holds columns ct..ct+c-1 with c = 32/bits;
+              column ct + 2j + e sits in bits [16e + bits j, 16e + bits j + bits).
       3 bits: word w (0..2) of run r holds columns 32r + 10w + 2p + e
               (p = 0..4, e = 0,1) in bits [16e + 3p, 16e + 3p + 3); bit b of the
               codes of columns 32r+30 and 32r+31 sits in bit 15 and bit 31 of

@@ -66,7 +66,8 @@ def test_degenerate_groups():
 
 # ---------------------------------------------------------------- properties
 @pytest.mark.parametrize("bits,group,frac,seed", [(4, 128, 0.01, 0), (3, 64, 0.02, 1), (4, 64, 0.0, 2),
-                                                   (3, 128, 0.3, 3), (4, 16, 0.01, 4), (3, 32, 0.02, 5)])
+                                                   (3, 128, 0.3, 3), (4, 16, 0.01, 4), (3, 32, 0.02, 5),
+                                                   (8, 128, 0.01, 6), (2, 64, 0.01, 7), (8, 16, 0.0, 8)])
 def test_scale_covers_range_and_is_minimal(bits, group, frac, seed):
     N, K = 64, 512
     W, G = synth.make_weight_and_grad(N, K, seed)
@@ -91,7 +92,8 @@ def test_scale_covers_range_and_is_minimal(bits, group, frac, seed):
 
 
 @pytest.mark.parametrize("bits,group,frac", [(4, 128, 0.01), (3, 128, 0.01), (4, 64, 0.005), (3, 64, 0.02),
-                                             (4, 16, 0.01), (3, 16, 0.01), (4, 32, 0.02)])
+                                             (4, 16, 0.01), (3, 16, 0.01), (4, 32, 0.02), (8, 128, 0.01),
+                                             (2, 128, 0.01), (2, 32, 0.02), (8, 64, 0.005)])
 def test_error_bound_and_outlier_codes(bits, group, frac):
     N, K = 128, 1024
     W, G = synth.make_weight_and_grad(N, K, seed=4)
@@ -108,7 +110,13 @@ def test_error_bound_and_outlier_codes(bits, group, frac):
 
 def test_codes_are_nearest_level_brute_force():
     # given (s, z), the stored code must minimise |w - s (q - z)| over all levels
-    N, K, bits, group = 8, 256, 4, 64
+    _codes_are_nearest_levels(4, 64)
+    _codes_are_nearest_levels(8, 128)
+    _codes_are_nearest_levels(2, 32)
+
+
+def _codes_are_nearest_levels(bits, group):
+    N, K = 8, 256
     W, G = synth.make_weight_and_grad(N, K, seed=6)
     L = _quant(W, G, 0.02, bits, group)
     s = np.repeat(L["scales"].astype(np.float64), group, axis=1)
@@ -184,6 +192,10 @@ def _pack_run_scalar(codes32, bits):
         if bits == 4:
             t, j, e = i // 8, (i % 8) // 2, i % 2
             words[t] |= c << (16 * e + 4 * j)
+        elif bits in (2, 8):
+            per = 32 // bits
+            t, j, e = i // per, (i % per) // 2, i % 2
+            words[t] |= c << (16 * e + bits * j)
         else:
             if i < 30:
                 w, p_, e = i // 10, (i % 10) // 2, i % 2
@@ -194,7 +206,7 @@ def _pack_run_scalar(codes32, bits):
     return words
 
 
-@pytest.mark.parametrize("bits", [3, 4])
+@pytest.mark.parametrize("bits", [2, 3, 4, 8])
 def test_pack_matches_scalar_definition_and_roundtrips(bits):
     rng = np.random.default_rng(bits)
     codes = rng.integers(0, 2 ** bits, size=(5, 160), dtype=np.uint8)
@@ -209,4 +221,4 @@ def test_pack_matches_scalar_definition_and_roundtrips(bits):
     full = orc.pack_codes(np.full((1, 32), 2 ** bits - 1, dtype=np.uint8), bits)
     assert [int(w) for w in full[0]] == [0xFFFFFFFF] * bits
     with pytest.raises(ValueError):
-        orc.pack_codes(np.full((1, 32), 2 ** bits, dtype=np.uint8), bits)
+        orc.pack_codes(np.full((1, 32), 2 ** bits, dtype=np.uint16), bits)
