@@ -36,7 +36,7 @@ extern "C" {
 typedef enum {
   GWQ_OK = 0,
   GWQ_ERR_INVALID_ARG = 1, /* null or misaligned pointer, non-positive size, frac outside [0,1] */
-  GWQ_ERR_UNSUPPORTED = 2, /* bits not in {3,4}, group not in {16,32,64,128}, K % group != 0 */
+  GWQ_ERR_UNSUPPORTED = 2, /* bits not in {2,3,4,8}, group not in {16,32,64,128}, K % group != 0 */
   GWQ_ERR_ALLOC = 3,       /* device or host allocation failed                                  */
   GWQ_ERR_NONFINITE = 4,   /* W holds an inf or NaN                                             */
   GWQ_ERR_TIMEOUT = 5,     /* a bounded device-side wait ran out (kernel returned early)        */
@@ -63,6 +63,8 @@ typedef struct gwq_outliers {
  *   the odd columns that follow them.
  *     4 bits: word t of a row holds columns 8t..8t+7; column 8t + 2j + e (j = 0..3,
  *             e = 0,1) is in bits [16e + 4j, 16e + 4j + 4).
+ *     2 and 8 bits, likewise: word t holds the c = 32 / bits columns ct..ct+c-1; column ct + 2j + e is in
+ *             bits [16e + bits j, 16e + bits j + bits).
  *     3 bits: word w (0..2) of run r holds columns 32r + 10w + 2p + e (p = 0..4, e = 0,1)
  *             in bits [16e + 3p, 16e + 3p + 3); bit b of the codes of columns 32r+30 and
  *             32r+31 is in bit 15 and bit 31 of word b.
@@ -129,8 +131,8 @@ gwq_status gwq_outliers_rows(const gwq_outliers* S, int32_t row0, int32_t row1, 
  * rounded up to fp16 (the paper's printed denominator 2^{b-1} is read as 2^b - 1);
  * z = clip(rint(-lo / s), 0, 2^bits - 1); q = clip(rint(w / s) + z, 0, 2^bits - 1),
  * round-half-to-even; outliers get q = z.  A group with hi == lo gets s = 1, z = 0.
- *   bits: 3 or 4.  group: 16 (the value Section 3.2 names), 32, 64 or 128; K a multiple of 32 and of
- *      group.  Which kernel of gwq_linear serves a layer depends on its shape: with K a multiple of 128 (up to
+ *   bits: 3 or 4 (the widths of the paper's experiments), or 2 or 8 (Eqs. "s", "z", "q" hold for any b).
+ *   group: 16 (the value Section 3.2 names), 32, 64 or 128; K a multiple of 32 and of group.  Which kernel of gwq_linear serves a layer depends on its shape: with K a multiple of 128 (up to
  *      65536) the streaming kernels take groups of 128 up to 32 tokens, of 64 up to 16, of 32 up to 4 and of 16
  *      for one token; with K a multiple of 64 the tensor-core kernel takes every group size and token count;
  *      anything else is served by a general (slow) kernel.

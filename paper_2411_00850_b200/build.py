@@ -15,7 +15,8 @@ OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libgwq.so")
 AID_SRC = os.path.join(HERE, "bench_aid", "read_probe.cu")    # the benchmark's read-only launch, a library of its own
 AID_LIB = os.path.join(HERE, "bench_aid", "libbench_read_probe.so")
-SOURCES = ("decode_w4_f16.cu", "decode_w4_bf16.cu", "decode_w3_f16.cu", "decode_w3_bf16.cu", "select.cu",
+SOURCES = ("decode_w4_f16.cu", "decode_w4_bf16.cu", "decode_w3_f16.cu", "decode_w3_bf16.cu", "decode_w8_f16.cu",
+           "decode_w8_bf16.cu", "decode_w2_f16.cu", "decode_w2_bf16.cu", "select.cu",
            "select_static.cu", "pack.cu", "linear_simt.cu", "linear_decode.cu", "linear_skinny.cu", "linear_prefill.cu",
            "quality.cu", "gradmean.cu", "api.cu")
 NVCC_FLAGS = (

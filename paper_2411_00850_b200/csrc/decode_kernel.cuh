@@ -71,6 +71,10 @@ cudaError_t launch_w4_f16(const Variant& v, const MultiArgs& a, cudaStream_t str
 cudaError_t launch_w4_bf16(const Variant& v, const MultiArgs& a, cudaStream_t stream);
 cudaError_t launch_w3_f16(const Variant& v, const MultiArgs& a, cudaStream_t stream);
 cudaError_t launch_w3_bf16(const Variant& v, const MultiArgs& a, cudaStream_t stream);
+cudaError_t launch_w8_f16(const Variant& v, const MultiArgs& a, cudaStream_t stream);
+cudaError_t launch_w8_bf16(const Variant& v, const MultiArgs& a, cudaStream_t stream);
+cudaError_t launch_w2_f16(const Variant& v, const MultiArgs& a, cudaStream_t stream);
+cudaError_t launch_w2_bf16(const Variant& v, const MultiArgs& a, cudaStream_t stream);
 
 constexpr int kChunkGroups = kWarps;                 // groups per chunk
 constexpr int kChunkPieces = kChunkGroups * 16;      // 16-byte pieces per token row per chunk
@@ -201,6 +205,60 @@ __device__ __forceinline__ void step_raw3(const unsigned (&qa)[3], const unsigne
   }
 }
 
+// 8-bit codes: pair 2i is the low byte of both halves of word i, pair 2i+1 the high byte (one shift, two masks per
+// word); codes up to 255 are still fp16 subnormals q 2^-24.  One position, one accumulator.
+template <int NB>
+struct AccRaw8 {
+  float c0[NB][4];
+};
+template <int NB>
+__device__ __forceinline__ void step_raw8(const unsigned (&qa)[8], const unsigned (&qb)[8],
+                                          const unsigned (&xr)[NB][16], AccRaw8<NB>& acc) {
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const unsigned a0 = qa[i] & 0x00FF00FFu, b0 = qb[i] & 0x00FF00FFu;
+    const unsigned a1 = (qa[i] >> 8) & 0x00FF00FFu, b1 = (qb[i] >> 8) & 0x00FF00FFu;
+#pragma unroll
+    for (int nb = 0; nb < NB; ++nb) {
+      if (i == 0) mma16816<false, true>(acc.c0[nb], a0, b0, a1, b1, xr[nb][2 * i], xr[nb][2 * i + 1]);
+      else mma16816<false, false>(acc.c0[nb], a0, b0, a1, b1, xr[nb][2 * i], xr[nb][2 * i + 1]);
+    }
+  }
+}
+
+// 2-bit codes: word i holds pairs 8i .. 8i+7, pair 8i+p at bits 2p of both halves.  Three shifts (by 4, 8, 12) leave
+// the even pairs at position 0 and the odd ones at position 2: two accumulators, merged with 1/4 in the epilogue.
+template <int NB>
+struct AccRaw2 {
+  float c0[NB][4], c2[NB][4];
+};
+template <int NB>
+__device__ __forceinline__ void step_raw2(const unsigned (&qa)[2], const unsigned (&qb)[2],
+                                          const unsigned (&xr)[NB][16], AccRaw2<NB>& acc) {
+#pragma unroll
+  for (int i = 0; i < 2; ++i) {
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {   // pairs 8i + 4u .. 8i + 4u + 3
+      const unsigned ta = qa[i] >> (8 * u), tb = qb[i] >> (8 * u), ua = ta >> 4, ub = tb >> 4;
+      const unsigned a0 = ta & 0x00030003u, b0 = tb & 0x00030003u;   // pair 8i+4u   (position 0)
+      const unsigned a1 = ta & 0x000C000Cu, b1 = tb & 0x000C000Cu;   // pair 8i+4u+1 (position 2)
+      const unsigned a2 = ua & 0x00030003u, b2 = ub & 0x00030003u;   // pair 8i+4u+2 (position 0)
+      const unsigned a3 = ua & 0x000C000Cu, b3 = ub & 0x000C000Cu;   // pair 8i+4u+3 (position 2)
+      const int h = 8 * i + 4 * u;
+#pragma unroll
+      for (int nb = 0; nb < NB; ++nb) {
+        if (i == 0 && u == 0) {
+          mma16816<false, true>(acc.c0[nb], a0, b0, a2, b2, xr[nb][h], xr[nb][h + 2]);
+          mma16816<false, true>(acc.c2[nb], a1, b1, a3, b3, xr[nb][h + 1], xr[nb][h + 3]);
+        } else {
+          mma16816<false, false>(acc.c0[nb], a0, b0, a2, b2, xr[nb][h], xr[nb][h + 2]);
+          mma16816<false, false>(acc.c2[nb], a1, b1, a3, b3, xr[nb][h + 1], xr[nb][h + 3]);
+        }
+      }
+    }
+  }
+}
+
 // sum_k x_k of the step's columns for every token of the block, through an A operand of all ones
 template <int NB>
 __device__ __forceinline__ void step_ones(const unsigned (&xr)[NB][16], float (&xs)[NB][4]) {
@@ -221,7 +279,28 @@ __device__ __forceinline__ void step_sub(const unsigned (&qa)[BITS], const unsig
                                          const unsigned (&zmb)[2], const unsigned (&xr)[NB][16], AccSub<NB>& acc) {
   constexpr unsigned MAGIC = 0x43004300u;  // bf16 128.0: ulp = 1
   unsigned a[16], b[16];
-  if (BITS == 4) {
+  if (BITS == 8) {
+    // codes up to 255 do not fit under the bf16 magic number: q - z is taken in fp16 (magic 1024, exact) and
+    // converted, exactly, to bf16 (|q - z| <= 255 has 8 significant bits).  zma / zmb hold the fp16 magic | z here.
+#pragma unroll
+    for (int h = 0; h < 16; ++h) {
+      const unsigned va = ((qa[(h >> 1) % BITS] >> (8 * (h & 1))) & 0x00FF00FFu) | 0x64006400u;
+      const unsigned vb = ((qb[(h >> 1) % BITS] >> (8 * (h & 1))) & 0x00FF00FFu) | 0x64006400u;
+      const float2 fa = __half22float2(__hsub2(*reinterpret_cast<const __half2*>(&va),
+                                               *reinterpret_cast<const __half2*>(&zma[h >> 3])));
+      const float2 fb = __half22float2(__hsub2(*reinterpret_cast<const __half2*>(&vb),
+                                               *reinterpret_cast<const __half2*>(&zmb[h >> 3])));
+      const __nv_bfloat162 ca = __floats2bfloat162_rn(fa.x, fa.y), cb = __floats2bfloat162_rn(fb.x, fb.y);
+      a[h] = *reinterpret_cast<const unsigned*>(&ca);
+      b[h] = *reinterpret_cast<const unsigned*>(&cb);
+    }
+  } else if (BITS == 2) {
+#pragma unroll
+    for (int h = 0; h < 16; ++h) {
+      a[h] = sub_zero_bf16(((qa[(h >> 3) % BITS] >> (2 * (h & 7))) & 0x00030003u) | MAGIC, zma[h >> 3]);
+      b[h] = sub_zero_bf16(((qb[(h >> 3) % BITS] >> (2 * (h & 7))) & 0x00030003u) | MAGIC, zmb[h >> 3]);
+    }
+  } else if (BITS == 4) {
 #pragma unroll
     for (int i = 0; i < 4; ++i)
 #pragma unroll
@@ -234,12 +313,12 @@ __device__ __forceinline__ void step_sub(const unsigned (&qa)[BITS], const unsig
     for (int i = 0; i < 3; ++i)
 #pragma unroll
       for (int p = 0; p < 5; ++p) {
-        a[5 * i + p] = sub_zero_bf16(((qa[i] >> (3 * p)) & 0x00070007u) | MAGIC, zma[(5 * i + p) >> 3]);
-        b[5 * i + p] = sub_zero_bf16(((qb[i] >> (3 * p)) & 0x00070007u) | MAGIC, zmb[(5 * i + p) >> 3]);
+        a[5 * i + p] = sub_zero_bf16(((qa[i % BITS] >> (3 * p)) & 0x00070007u) | MAGIC, zma[(5 * i + p) >> 3]);
+        b[5 * i + p] = sub_zero_bf16(((qb[i % BITS] >> (3 * p)) & 0x00070007u) | MAGIC, zmb[(5 * i + p) >> 3]);
       }
-    const unsigned la = ((qa[0] >> 15) & 0x00010001u) | ((qa[1] >> 14) & 0x00020002u) |
+    const unsigned la = ((qa[0] >> 15) & 0x00010001u) | ((qa[1 % BITS] >> 14) & 0x00020002u) |
                         ((qa[BITS - 1] >> 13) & 0x00040004u);
-    const unsigned lb = ((qb[0] >> 15) & 0x00010001u) | ((qb[1] >> 14) & 0x00020002u) |
+    const unsigned lb = ((qb[0] >> 15) & 0x00010001u) | ((qb[1 % BITS] >> 14) & 0x00020002u) |
                         ((qb[BITS - 1] >> 13) & 0x00040004u);
     a[15] = sub_zero_bf16(la | MAGIC, zma[1]);
     b[15] = sub_zero_bf16(lb | MAGIC, zmb[1]);
@@ -259,7 +338,14 @@ __device__ __forceinline__ void load_run(const uint32_t* __restrict__ base, unsi
   const uint32_t* p = base + off;
   if (BITS == 4) {
     const uint4 v = __ldcs(reinterpret_cast<const uint4*>(p));  // streamed once: evict first
-    w[0] = v.x; w[1] = v.y; w[2] = v.z; w[BITS - 1] = v.w;
+    w[0] = v.x; w[1 % BITS] = v.y; w[2 % BITS] = v.z; w[BITS - 1] = v.w;
+  } else if (BITS == 8) {
+    const uint4 v = __ldcs(reinterpret_cast<const uint4*>(p)), u = __ldcs(reinterpret_cast<const uint4*>(p) + 1);
+    w[0] = v.x; w[1 % BITS] = v.y; w[2 % BITS] = v.z; w[3 % BITS] = v.w;
+    w[4 % BITS] = u.x; w[5 % BITS] = u.y; w[6 % BITS] = u.z; w[7 % BITS] = u.w;
+  } else if (BITS == 2) {
+    const uint2 v = __ldcs(reinterpret_cast<const uint2*>(p));
+    w[0] = v.x; w[BITS - 1] = v.y;
   } else {
 #pragma unroll
     for (int i = 0; i < BITS; ++i) w[i] = __ldcs(p + i);
@@ -271,16 +357,28 @@ template <int BITS>
 __device__ __forceinline__ void load_run_if(const uint32_t* __restrict__ base, unsigned off, unsigned (&w)[BITS],
                                             bool pred) {
   const uint32_t* p = base + off;
-  if (BITS == 4) {
+  if constexpr (BITS == 4) {
     asm volatile(
         "{\n .reg .pred q;\n setp.ne.b32 q, %5, 0;\n @q ld.global.cs.v4.u32 {%0,%1,%2,%3}, [%4];\n}\n"
-        : "+r"(w[0]), "+r"(w[1]), "+r"(w[2]), "+r"(w[BITS - 1])
+        : "+r"(w[0]), "+r"(w[1 % BITS]), "+r"(w[2 % BITS]), "+r"(w[BITS - 1])
+        : "l"(p), "r"((int)pred));
+  } else if constexpr (BITS == 8) {
+    asm volatile(
+        "{\n .reg .pred q;\n setp.ne.b32 q, %9, 0;\n @q ld.global.cs.v4.u32 {%0,%1,%2,%3}, [%8];\n"
+        " @q ld.global.cs.v4.u32 {%4,%5,%6,%7}, [%8+16];\n}\n"
+        : "+r"(w[0]), "+r"(w[1 % BITS]), "+r"(w[2 % BITS]), "+r"(w[3 % BITS]), "+r"(w[4 % BITS]), "+r"(w[5 % BITS]),
+          "+r"(w[6 % BITS]), "+r"(w[7 % BITS])
+        : "l"(p), "r"((int)pred));
+  } else if constexpr (BITS == 2) {
+    asm volatile(
+        "{\n .reg .pred q;\n setp.ne.b32 q, %3, 0;\n @q ld.global.cs.v2.u32 {%0,%1}, [%2];\n}\n"
+        : "+r"(w[0]), "+r"(w[BITS - 1])
         : "l"(p), "r"((int)pred));
   } else {
     asm volatile(
         "{\n .reg .pred q;\n setp.ne.b32 q, %4, 0;\n @q ld.global.cs.u32 %0, [%3];\n @q ld.global.cs.u32 %1, [%3+4];\n"
         " @q ld.global.cs.u32 %2, [%3+8];\n}\n"
-        : "+r"(w[0]), "+r"(w[1]), "+r"(w[2])
+        : "+r"(w[0]), "+r"(w[1 % BITS]), "+r"(w[2 % BITS])
         : "l"(p), "r"((int)pred));
   }
 }
@@ -340,6 +438,8 @@ template <int BITS, int NB, bool BF16>
 struct StepAcc;
 template <int NB> struct StepAcc<4, NB, false> { using type = AccRaw4<NB>; };
 template <int NB> struct StepAcc<3, NB, false> { using type = AccRaw3<NB>; };
+template <int NB> struct StepAcc<8, NB, false> { using type = AccRaw8<NB>; };
+template <int NB> struct StepAcc<2, NB, false> { using type = AccRaw2<NB>; };
 template <int BITS, int NB> struct StepAcc<BITS, NB, true> { using type = AccSub<NB>; };
 
 // resident CTAs the register budget is cut for
@@ -376,7 +476,8 @@ template <int BITS, int TP, bool BF16, int NBUF, int GS, int RT, bool DEEP>
 __global__ void __launch_bounds__(kThreads, min_blocks(token_blocks(TP, GS), RT, DEEP))
 decode_kernel(const MultiArgs ma) {
   constexpr int R = 16 * RT;                       // rows of the CTA
-  constexpr int D = DEEP ? 8 : (RT == 1 ? 4 : 2);  // groups of codes in flight per warp and tile
+  // groups of codes in flight per warp and tile (about the same bytes whatever the code width)
+  constexpr int D = (DEEP ? 8 : (RT == 1 ? 4 : 2)) * (BITS == 2 ? 2 : 1) / (BITS == 8 ? 2 : 1);
   constexpr bool G64 = GS == 2;
   constexpr int TB = 8 / GS;                       // tokens of a block
   constexpr int NB = token_blocks(TP, GS);         // token blocks of the MMA
@@ -715,8 +816,9 @@ decode_kernel(const MultiArgs ma) {
         const float sb = __half2float(__ushort_as_half((unsigned short)szb));
         const unsigned za = sza >> 16, zb = szb >> 16;
         if (BF16) {
-          ta[e] = make_float2(sa, __uint_as_float(0x43004300u | (za * 0x00010001u)));
-          tb[e] = make_float2(sb, __uint_as_float(0x43004300u | (zb * 0x00010001u)));
+          constexpr unsigned kZeroMagic = BITS == 8 ? 0x64006400u : 0x43004300u;   // see step_sub
+          ta[e] = make_float2(sa, __uint_as_float(kZeroMagic | (za * 0x00010001u)));
+          tb[e] = make_float2(sb, __uint_as_float(kZeroMagic | (zb * 0x00010001u)));
         } else {
           ta[e] = make_float2(sa * 16777216.f, sa * (float)za);
           tb[e] = make_float2(sb * 16777216.f, sb * (float)zb);
@@ -730,6 +832,10 @@ decode_kernel(const MultiArgs ma) {
         step_sub<BITS, NB>(wa[rt][d], wb[rt][d], zma, zmb, xr, acc);
       } else if constexpr (BITS == 4) {
         step_raw4<NB>(wa[rt][d], wb[rt][d], xr, acc);
+      } else if constexpr (BITS == 8) {
+        step_raw8<NB>(wa[rt][d], wb[rt][d], xr, acc);
+      } else if constexpr (BITS == 2) {
+        step_raw2<NB>(wa[rt][d], wb[rt][d], xr, acc);
       } else {
         step_raw3<NB>(wa[rt][d], wb[rt][d], xr, acc);
       }
@@ -748,6 +854,11 @@ decode_kernel(const MultiArgs ma) {
             yacc[rt][nb][i] = fmaf(tt.x, acc.c[nb][i], yacc[rt][nb][i]);
           } else if constexpr (BITS == 4) {
             const float code_sum = fmaf(acc.c4[nb][i], 0.0625f, acc.c0[nb][i]);  // units of 2^-24
+            yacc[rt][nb][i] = fmaf(tt.x, code_sum, fmaf(-tt.y, xs[nb][i & 1], yacc[rt][nb][i]));
+          } else if constexpr (BITS == 8) {
+            yacc[rt][nb][i] = fmaf(tt.x, acc.c0[nb][i], fmaf(-tt.y, xs[nb][i & 1], yacc[rt][nb][i]));
+          } else if constexpr (BITS == 2) {
+            const float code_sum = fmaf(acc.c2[nb][i], 0.25f, acc.c0[nb][i]);
             yacc[rt][nb][i] = fmaf(tt.x, code_sum, fmaf(-tt.y, xs[nb][i & 1], yacc[rt][nb][i]));
           } else {
             const float code_sum = fmaf(acc.c6[nb][i], 0.015625f, fmaf(acc.c3[nb][i], 0.125f, acc.c0[nb][i]));
@@ -855,24 +966,26 @@ cudaError_t launch_tp(const Variant& v, const MultiArgs& a, cudaStream_t stream)
   } else {
     if (v.nbuf == 0) {
       if constexpr (TP <= 8) {
+        constexpr bool kWide = BITS == 3 || BITS == 4;   // two tiles per CTA and the deep variant: these widths only
         if (v.rt == 2) {
-          if constexpr (GS == 1) return launch<BITS, TP, BF16, 0, GS, 2>(v, a, stream);
+          if constexpr (GS == 1 && kWide) return launch<BITS, TP, BF16, 0, GS, 2>(v, a, stream);
           return cudaErrorInvalidValue;
         }
-        if constexpr (GS == 1) {
+        if constexpr (GS == 1 && kWide) {
           if (v.deep) return launch<BITS, TP, BF16, 0, GS, 1, true>(v, a, stream);
         }
         return launch<BITS, TP, BF16, 0, GS, 1>(v, a, stream);
       }
       return cudaErrorInvalidValue;
     }
+    constexpr bool kWide = BITS == 3 || BITS == 4;
     if (v.rt == 2) {
-      if constexpr (GS == 1 && TP <= 8) {
+      if constexpr (GS == 1 && TP <= 8 && kWide) {
         if (v.nbuf == 2) return launch<BITS, TP, BF16, 2, GS, 2>(v, a, stream);
       }
       return cudaErrorInvalidValue;
     }
-    if constexpr (GS == 1 && TP <= 8) {
+    if constexpr (GS == 1 && TP <= 8 && kWide) {
       if (v.deep && v.nbuf == 2) return launch<BITS, TP, BF16, 2, GS, 1, true>(v, a, stream);
     }
     if (v.nbuf == 2) return launch<BITS, TP, BF16, 2, GS, 1>(v, a, stream);

@@ -113,15 +113,16 @@ bool plan(const gwq_packed* const* P, int count, int M, Variant* v, int* cvcap) 
     blocks1 += (P[i]->N + 15) / 16;
     blocks2 += (P[i]->N + 31) / 32;
   }
-  v->rt = (gs == 1 && v->tp <= 8 && blocks1 > 3LL * sms && blocks2 <= 2LL * sms) ? 2 : 1;
-  if (GWQ_TUNE_RT == 1 || (GWQ_TUNE_RT == 2 && gs == 1 && v->tp <= 8)) v->rt = GWQ_TUNE_RT;
+  const bool wide = P[0]->bits == 3 || P[0]->bits == 4;   // two tiles per CTA and the deep variant exist for these widths
+  v->rt = (wide && gs == 1 && v->tp <= 8 && blocks1 > 3LL * sms && blocks2 <= 2LL * sms) ? 2 : 1;
+  if (GWQ_TUNE_RT == 1 || (GWQ_TUNE_RT == 2 && wide && gs == 1 && v->tp <= 8)) v->rt = GWQ_TUNE_RT;
   long long blocks = 0;
   for (int i = 0; i < count; ++i) blocks += (P[i]->N + 16 * v->rt - 1) / (16 * v->rt);
   // a grid that leaves an SM two CTAs at most anyway: twice the codes in flight per warp (more registers, which then
   // cost no occupancy)
-  v->deep = (v->rt == 1 && gs == 1 && v->tp <= 8 && blocks <= 2LL * sms) ? 1 : 0;
+  v->deep = (wide && v->rt == 1 && gs == 1 && v->tp <= 8 && blocks <= 2LL * sms) ? 1 : 0;
 #ifdef GWQ_TUNE_DEEP
-  v->deep = (v->rt == 1 && gs == 1 && v->tp <= 8) ? GWQ_TUNE_DEEP : 0;
+  v->deep = (wide && v->rt == 1 && gs == 1 && v->tp <= 8) ? GWQ_TUNE_DEEP : 0;
 #endif
   const int nchunks = (K / 128 + kChunkGroups - 1) / kChunkGroups;
   const size_t lim = v->rt == 2 ? kStageAllLimitTwoTiles : (blocks <= 2LL * sms ? kStageAllLimitSmallGrid : kStageAllLimit);
@@ -211,8 +212,14 @@ gwq_status gwq_launch_decode_multi(const gwq_packed* const* P, int count, const 
     a.xg = xg;
   }
   cudaError_t e;
-  if (P[0]->bits == 4) e = (xd == GWQ_BF16) ? launch_w4_bf16(v, a, stream) : launch_w4_f16(v, a, stream);
-  else e = (xd == GWQ_BF16) ? launch_w3_bf16(v, a, stream) : launch_w3_f16(v, a, stream);
+  const bool bf = xd == GWQ_BF16;
+  switch (P[0]->bits) {
+    case 4: e = bf ? launch_w4_bf16(v, a, stream) : launch_w4_f16(v, a, stream); break;
+    case 3: e = bf ? launch_w3_bf16(v, a, stream) : launch_w3_f16(v, a, stream); break;
+    case 8: e = bf ? launch_w8_bf16(v, a, stream) : launch_w8_f16(v, a, stream); break;
+    case 2: e = bf ? launch_w2_bf16(v, a, stream) : launch_w2_f16(v, a, stream); break;
+    default: return GWQ_ERR_UNSUPPORTED;
+  }
   if (e != cudaSuccess) {
     (void)cudaGetLastError();
     return GWQ_ERR_CUDA;

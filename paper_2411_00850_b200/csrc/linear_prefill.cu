@@ -117,7 +117,7 @@ __global__ void __launch_bounds__(256) bf16_rows_to_scaled_f16(const uint16_t* _
 }
 
 
-// Packed words of one row for one k-block (8 words for 4 bits, 6 for 3 bits) with the widest loads
+// Packed words of one row for one k-block (8 words for 4 bits, 6 for 3, 4 for 2, 16 for 8) with the widest loads
 // the alignment allows: a thread reads its own row, so every load instruction of a warp touches 32
 // different lines, and the number of load instructions is what the load pipe pays for.
 template <int WPB>
@@ -125,10 +125,16 @@ __device__ __forceinline__ void load_words(const uint32_t* __restrict__ p, unsig
   if (WPB == 8) {
     const uint4 a = __ldg(reinterpret_cast<const uint4*>(p)), b = __ldg(reinterpret_cast<const uint4*>(p) + 1);
     w[0] = a.x; w[1] = a.y; w[2] = a.z; w[3] = a.w; w[4 % WPB] = b.x; w[5 % WPB] = b.y; w[6 % WPB] = b.z; w[7 % WPB] = b.w;
+  } else if (WPB == 16 || WPB == 4) {   // 8 bits: 64 bytes; 2 bits: 16 bytes
+#pragma unroll
+    for (int i = 0; i < WPB / 4; ++i) {
+      const uint4 a = __ldg(reinterpret_cast<const uint4*>(p) + i);
+      w[(4 * i) % WPB] = a.x; w[(4 * i + 1) % WPB] = a.y; w[(4 * i + 2) % WPB] = a.z; w[(4 * i + 3) % WPB] = a.w;
+    }
   } else {   // 24 bytes, 8-byte aligned
     const uint2 a = __ldg(reinterpret_cast<const uint2*>(p)), b = __ldg(reinterpret_cast<const uint2*>(p) + 1),
                 c = __ldg(reinterpret_cast<const uint2*>(p) + 2);
-    w[0] = a.x; w[1] = a.y; w[2] = b.x; w[3] = b.y; w[4] = c.x; w[5] = c.y;
+    w[0] = a.x; w[1] = a.y; w[2 % WPB] = b.x; w[3 % WPB] = b.y; w[4 % WPB] = c.x; w[5 % WPB] = c.y;
   }
 }
 
@@ -327,6 +333,14 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmx, const PrefillArgs p,
               out[4 * i + q4] = mul_scale<BF16>(
                   sub_magic<BF16>(((cur[i % WPB] >> (4 * q4)) & 0x000F000Fu) | MAGIC, zm[(4 * i + q4) * GPK / 32]),
                   s_hi2[(4 * i + q4) * GPK / 32], s_lo2[(4 * i + q4) * GPK / 32]);
+        } else if (BITS == 2 || BITS == 8) {   // pair h: word h / (16 / BITS), BITS (h % (16 / BITS)) bits up
+          constexpr int PPW = 16 / BITS;
+          constexpr unsigned CMASK = ((1u << BITS) - 1u) * 0x00010001u;
+#pragma unroll
+          for (int h = 0; h < 32; ++h)
+            out[h] = mul_scale<BF16>(
+                sub_magic<BF16>(((cur[(h / PPW) % WPB] >> (BITS * (h % PPW))) & CMASK) | MAGIC, zm[h * GPK / 32]),
+                s_hi2[h * GPK / 32], s_lo2[h * GPK / 32]);
         } else {
 #pragma unroll
           for (int run = 0; run < 2; ++run) {
@@ -459,7 +473,7 @@ __global__ void __launch_bounds__(256) expand_kernel(const uint32_t* __restrict_
   unsigned w[BITS];
   if (BITS == 4) {
     const uint4 v = __ldg(reinterpret_cast<const uint4*>(src));
-    w[0] = v.x; w[1] = v.y; w[2] = v.z; w[BITS - 1] = v.w;
+    w[0] = v.x; w[1 % BITS] = v.y; w[2 % BITS] = v.z; w[3 % BITS] = v.w;
   } else {
 #pragma unroll
     for (int k = 0; k < BITS; ++k) w[k] = __ldg(src + k);
@@ -480,14 +494,21 @@ __global__ void __launch_bounds__(256) expand_kernel(const uint32_t* __restrict_
       for (int j = 0; j < 4; ++j)
         out[4 * t + j] = mul_scale<false>(sub_magic<false>(((w[t % BITS] >> (4 * j)) & 0x000F000Fu) | 0x64006400u, zm[t / 2]),
                                           s2[t / 2], 0);
+  } else if (BITS == 2 || BITS == 8) {
+    constexpr int PPW = 16 / BITS;
+    constexpr unsigned CMASK = ((1u << BITS) - 1u) * 0x00010001u;
+#pragma unroll
+    for (int h = 0; h < 16; ++h)
+      out[h] = mul_scale<false>(sub_magic<false>(((w[(h / PPW) % BITS] >> (BITS * (h % PPW))) & CMASK) | 0x64006400u, zm[h / 8]),
+                                s2[h / 8], 0);
   } else {
 #pragma unroll
     for (int k = 0; k < 3; ++k)
 #pragma unroll
       for (int pp = 0; pp < 5; ++pp)
-        out[5 * k + pp] = mul_scale<false>(sub_magic<false>(((w[k] >> (3 * pp)) & 0x00070007u) | 0x64006400u, zm[(5 * k + pp) / 8]),
+        out[5 * k + pp] = mul_scale<false>(sub_magic<false>(((w[k % BITS] >> (3 * pp)) & 0x00070007u) | 0x64006400u, zm[(5 * k + pp) / 8]),
                                            s2[(5 * k + pp) / 8], 0);
-    const unsigned last = ((w[0] >> 15) & 0x00010001u) | ((w[1] >> 14) & 0x00020002u) | ((w[BITS - 1] >> 13) & 0x00040004u);
+    const unsigned last = ((w[0] >> 15) & 0x00010001u) | ((w[1 % BITS] >> 14) & 0x00020002u) | ((w[BITS - 1] >> 13) & 0x00040004u);
     out[15] = mul_scale<false>(sub_magic<false>(last | 0x64006400u, zm[1]), s2[1], 0);
   }
   uint4* dst = reinterpret_cast<uint4*>(w16 + (size_t)row * K + run * 32);
@@ -1116,7 +1137,7 @@ __global__ void __launch_bounds__(256) expand_block_kernel(const uint32_t* __res
     unsigned w[BITS];
     if (BITS == 4) {
       const uint4 v = __ldg(reinterpret_cast<const uint4*>(src));
-      w[0] = v.x; w[1] = v.y; w[2] = v.z; w[BITS - 1] = v.w;
+      w[0] = v.x; w[1 % BITS] = v.y; w[2 % BITS] = v.z; w[3 % BITS] = v.w;
     } else {
 #pragma unroll
       for (int k = 0; k < BITS; ++k) w[k] = __ldg(src + k);
@@ -1136,14 +1157,21 @@ __global__ void __launch_bounds__(256) expand_block_kernel(const uint32_t* __res
         for (int j = 0; j < 4; ++j)
           out[4 * t + j] = mul_scale<false>(sub_magic<false>(((w[t % BITS] >> (4 * j)) & 0x000F000Fu) | 0x64006400u, zm[t / 2]),
                                             s2[t / 2], 0);
+    } else if (BITS == 2 || BITS == 8) {
+      constexpr int PPW = 16 / BITS;
+      constexpr unsigned CMASK = ((1u << BITS) - 1u) * 0x00010001u;
+#pragma unroll
+      for (int h = 0; h < 16; ++h)
+        out[h] = mul_scale<false>(sub_magic<false>(((w[(h / PPW) % BITS] >> (BITS * (h % PPW))) & CMASK) | 0x64006400u, zm[h / 8]),
+                                  s2[h / 8], 0);
     } else {
 #pragma unroll
       for (int k = 0; k < 3; ++k)
 #pragma unroll
         for (int pp = 0; pp < 5; ++pp)
-          out[5 * k + pp] = mul_scale<false>(sub_magic<false>(((w[k] >> (3 * pp)) & 0x00070007u) | 0x64006400u, zm[(5 * k + pp) / 8]),
+          out[5 * k + pp] = mul_scale<false>(sub_magic<false>(((w[k % BITS] >> (3 * pp)) & 0x00070007u) | 0x64006400u, zm[(5 * k + pp) / 8]),
                                              s2[(5 * k + pp) / 8], 0);
-      const unsigned last = ((w[0] >> 15) & 0x00010001u) | ((w[1] >> 14) & 0x00020002u) | ((w[BITS - 1] >> 13) & 0x00040004u);
+      const unsigned last = ((w[0] >> 15) & 0x00010001u) | ((w[1 % BITS] >> 14) & 0x00020002u) | ((w[BITS - 1] >> 13) & 0x00040004u);
       out[15] = mul_scale<false>(sub_magic<false>(last | 0x64006400u, zm[1]), s2[1], 0);
     }
     uint4* dst = reinterpret_cast<uint4*>(tile + r * kPitch + q * 32);
@@ -1192,18 +1220,25 @@ gwq_status launch_expanded(const gwq_packed* P, const void* x, const float* tok_
   const gwq_priv* pv = static_cast<const gwq_priv*>(P->priv);
   if (pv->ob && pv->ob_ptr && P->K % 128 == 0) {
     const unsigned blocks = (unsigned)((P->N + 127) / 128) * (unsigned)(P->K / 128);
-    if (P->bits == 4)
-      (void)launch_pdl(expand_block_kernel<4>, dim3(blocks), dim3(256), 0, stream, (const uint32_t*)P->codes, (const uint32_t*)pv->sz_t,
-                       (const uint32_t*)pv->ob, (const int32_t*)pv->ob_ptr, w16, P->N, P->K, P->group);
-    else
-      (void)launch_pdl(expand_block_kernel<3>, dim3(blocks), dim3(256), 0, stream, (const uint32_t*)P->codes, (const uint32_t*)pv->sz_t,
-                       (const uint32_t*)pv->ob, (const int32_t*)pv->ob_ptr, w16, P->N, P->K, P->group);
+#define GWQ_EXPAND_BLOCK(B)                                                                                                  \
+  (void)launch_pdl(expand_block_kernel<B>, dim3(blocks), dim3(256), 0, stream, (const uint32_t*)P->codes, (const uint32_t*)pv->sz_t, \
+                   (const uint32_t*)pv->ob, (const int32_t*)pv->ob_ptr, w16, P->N, P->K, P->group)
+    switch (P->bits) {
+      case 4: GWQ_EXPAND_BLOCK(4); break;
+      case 3: GWQ_EXPAND_BLOCK(3); break;
+      case 8: GWQ_EXPAND_BLOCK(8); break;
+      default: GWQ_EXPAND_BLOCK(2); break;
+    }
+#undef GWQ_EXPAND_BLOCK
   } else {
     const long long runs = (long long)P->N * (P->K / 32);
-    if (P->bits == 4)
-      expand_kernel<4><<<(unsigned)((runs + 255) / 256), 256, 0, stream>>>(P->codes, pv->sz_t, w16, P->N, P->K, P->group);
-    else
-      expand_kernel<3><<<(unsigned)((runs + 255) / 256), 256, 0, stream>>>(P->codes, pv->sz_t, w16, P->N, P->K, P->group);
+    const unsigned grid = (unsigned)((runs + 255) / 256);
+    switch (P->bits) {
+      case 4: expand_kernel<4><<<grid, 256, 0, stream>>>(P->codes, pv->sz_t, w16, P->N, P->K, P->group); break;
+      case 3: expand_kernel<3><<<grid, 256, 0, stream>>>(P->codes, pv->sz_t, w16, P->N, P->K, P->group); break;
+      case 8: expand_kernel<8><<<grid, 256, 0, stream>>>(P->codes, pv->sz_t, w16, P->N, P->K, P->group); break;
+      default: expand_kernel<2><<<grid, 256, 0, stream>>>(P->codes, pv->sz_t, w16, P->N, P->K, P->group); break;
+    }
     expand_outliers_kernel<<<(P->N + 7) / 8, 256, 0, stream>>>(P->S->row_ptr, pv->cv, w16, P->N, P->K);
   }
   if (cudaGetLastError() != cudaSuccess) return GWQ_ERR_CUDA;
@@ -1254,6 +1289,11 @@ gwq_status gwq_launch_prefill(const gwq_packed* P, const void* x, gwq_dtype xd, 
     const gwq_status st = launch_expanded(P, x, tok_scale, reinterpret_cast<uint16_t*>(w16), partial, M, y, yd, stream);
     if (st != GWQ_ERR_UNSUPPORTED) return st;   // a device that holds no cluster of two such CTAs: the fused kernel
   }
-  if (P->bits == 4) return launch_tok<4>(P, x, tok_scale, M, y, yd, stream);
-  return launch_tok<3>(P, x, tok_scale, M, y, yd, stream);
+  switch (P->bits) {
+    case 4: return launch_tok<4>(P, x, tok_scale, M, y, yd, stream);
+    case 3: return launch_tok<3>(P, x, tok_scale, M, y, yd, stream);
+    case 8: return launch_tok<8>(P, x, tok_scale, M, y, yd, stream);
+    case 2: return launch_tok<2>(P, x, tok_scale, M, y, yd, stream);
+  }
+  return GWQ_ERR_UNSUPPORTED;
 }

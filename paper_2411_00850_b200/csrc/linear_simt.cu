@@ -50,7 +50,7 @@ linear_simt_kernel(const uint32_t* __restrict__ codes, const uint16_t* __restric
       for (int t = 0; t < MT; ++t) acc[t] = 0.f;
       const int gsz = group < 32 ? group : 32;   // columns of a run that share one scale and zero-point
       for (int r = lane; r < nruns; r += 32) {
-        unsigned int w[4] = {0, 0, 0, 0};
+        unsigned int w[8] = {0, 0, 0, 0, 0, 0, 0, 0};
         for (int j = 0; j < bits; ++j) w[j] = __ldg(crow + r * bits + j);
         for (int seg = 0; seg < 32; seg += gsz) {
           const int g = (r * 32 + seg) / group;
@@ -65,6 +65,9 @@ linear_simt_kernel(const uint32_t* __restrict__ codes, const uint16_t* __restric
             const int e = i & 1;
             if (bits == 4) {
               code = (w[i >> 3] >> (16 * e + 4 * ((i & 7) >> 1))) & 15u;
+            } else if (bits != 3) {   // 2 and 8 bits: 32 / bits columns per word
+              const int per = 32 / bits;
+              code = (w[i / per] >> (16 * e + bits * ((i % per) >> 1))) & ((1u << bits) - 1u);
             } else if (i < 30) {
               const int wi = i / 10, r10 = i - 10 * wi;
               code = (w[wi] >> (16 * e + 3 * (r10 >> 1))) & 7u;

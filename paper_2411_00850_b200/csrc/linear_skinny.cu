@@ -644,7 +644,7 @@ gwq_status launch(const gwq_packed* P, const void* x, int M, void* y, gwq_dtype 
 // The skinny kernel takes fp16 activations, up to 32 tokens, groups of 64 or 128, K a multiple of 128 up to 65536.
 bool gwq_skinny_takes(const gwq_packed* P, gwq_dtype xd, int M) {
   const gwq_priv* pv = static_cast<const gwq_priv*>(P->priv);
-  return xd == GWQ_F16 && M >= 1 && M <= 32 && (P->group == 64 || P->group == 128) && P->K % 128 == 0 && P->K <= 65536 &&
+  return xd == GWQ_F16 && (P->bits == 3 || P->bits == 4) && M >= 1 && M <= 32 && (P->group == 64 || P->group == 128) && P->K % 128 == 0 && P->K <= 65536 &&
          pv->ob && pv->ob_ptr && pv->sz_t;
 }
 

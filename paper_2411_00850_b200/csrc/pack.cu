@@ -136,6 +136,7 @@ pack_row_kernel(const uint16_t* __restrict__ W, const int32_t* __restrict__ row_
 
   // pack (pair-interleaved order: even columns in the low half-word, odd in the high):
   //  4 bits: word j of a run holds its columns 8j..8j+7, column 8j+2p+e in bits [16e+4p, +4)
+  //          (2 and 8 bits likewise: 16 / 4 columns per word, column 16j+2p+e / 4j+2p+e in bits [16e+bits p, +bits))
   //  3 bits: word j holds columns 10j..10j+9, column 10j+2p+e in bits [16e+3p, +3); bit j of the
   //          codes of columns 30 / 31 goes to bit 15 / 31 of word j
   const int nwords = K / 32 * bits;
@@ -149,6 +150,11 @@ pack_row_kernel(const uint16_t* __restrict__ W, const int32_t* __restrict__ row_
 #pragma unroll
       for (int p = 0; p < 4; ++p)
         word |= ((unsigned int)c[2 * p] << (4 * p)) | ((unsigned int)c[2 * p + 1] << (16 + 4 * p));
+    } else if (bits != 3) {   // 2 and 8 bits: the 4-bit rule with 32 / bits columns per word
+      const int per = 32 / bits;
+      const unsigned char* c = r + per * j;
+      for (int p = 0; p < per / 2; ++p)
+        word |= ((unsigned int)c[2 * p] << (bits * p)) | ((unsigned int)c[2 * p + 1] << (16 + bits * p));
     } else {
       const unsigned char* c = r + 10 * j;
 #pragma unroll
@@ -235,7 +241,7 @@ extern "C" gwq_status gwq_pack(const uint16_t* W, gwq_outliers* S, int32_t N, in
   if (!W || !S || !out || N <= 0 || K <= 0) return GWQ_ERR_INVALID_ARG;
   if (S->tag != GWQ_TAG_OUTLIERS || S->N != N || S->K != K) return GWQ_ERR_INVALID_ARG;
   if (!gwq_aligned16(W)) return GWQ_ERR_INVALID_ARG;
-  if (bits != 3 && bits != 4) return GWQ_ERR_UNSUPPORTED;
+  if (bits != 2 && bits != 3 && bits != 4 && bits != 8) return GWQ_ERR_UNSUPPORTED;
   if (group != 16 && group != 32 && group != 64 && group != 128) return GWQ_ERR_UNSUPPORTED;
   if (K % group != 0 || K > 131072) return GWQ_ERR_UNSUPPORTED;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);

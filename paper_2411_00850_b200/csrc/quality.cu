@@ -37,7 +37,7 @@ quality_row_kernel(const uint16_t* __restrict__ W, const float* __restrict__ G, 
   }
   __syncthreads();
   for (int r = tid; r < nruns; r += kThreads) {
-    unsigned w[4] = {0, 0, 0, 0};
+    unsigned w[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     for (int j = 0; j < bits; ++j) w[j] = __ldg(crow + r * bits + j);
     const unsigned m = mask[r];
     for (int i = 0; i < 32; ++i) {
@@ -47,6 +47,9 @@ quality_row_kernel(const uint16_t* __restrict__ W, const float* __restrict__ G, 
       const int e = i & 1;
       if (bits == 4) {
         code = (w[i >> 3] >> (16 * e + 4 * ((i & 7) >> 1))) & 15u;
+      } else if (bits != 3) {   // 2 and 8 bits: 32 / bits columns per word
+        const int per = 32 / bits;
+        code = (w[i / per] >> (16 * e + bits * ((i % per) >> 1))) & ((1u << bits) - 1u);
       } else if (i < 30) {
         const int wi = i / 10, r10 = i - 10 * wi;
         code = (w[wi] >> (16 * e + 3 * (r10 >> 1))) & 7u;
