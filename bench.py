@@ -404,6 +404,7 @@ def run_cuda_arm(args):
         out["config0_single_layer"] = bench_config0(torch, gwq, dev, detail_iters, hbm_peak)
         if not args.skip_70b:
             out["llama70b_cases"] = bench_config4(torch, gwq, dev, 3, hbm_peak, tf_burst, args.prefill_iters)
+        out["other_widths"] = bench_other_widths(args)
         out["prefill"] = bench_prefill(torch, gwq, dev, args, tf_burst, tf_sust)
         best = max(out["prefill"], key=lambda r: r["tflops"])
         out["prefill_roofline"] = {"bound": "tensor", "kernel": "gwq prefill linear (tcgen05)",
@@ -421,6 +422,9 @@ def run_cuda_arm(args):
         for r in out.get("llama70b_cases", []):
             cases.append([r["N"], r["K"], r["bits"], r["group"], round(100 * r["frac"], 1), r["M"], r["us"],
                           r.get("frac_measured_peak", r.get("frac_measured_burst"))])
+        for r in out["other_widths"]:
+            cases.append([r["N"], r["K"], r["bits"], r["group"], 1.0, r["M"], r["us"],
+                          r["frac_measured_peak"] if r["M"] <= 32 else round(r["tflops"] / tf_burst, 4)])
         for r in out["prefill"]:
             cases.append([r["N"], r["K"], 4, GROUP, 1.0, r["M"], r["us"], r["frac_measured_burst"]])
         out["roofline"]["cases"] = cases
@@ -737,7 +741,20 @@ def bench_prefill(torch, gwq, dev, args, tf_burst, tf_sust):
 
 
 # ----------------------------------------------------------------------------- single cases (profiling, sweeps)
-def run_cases(args):
+def bench_other_widths(args):
+    """2- and 8-bit codes (the widths beside the paper's 3 and 4) on two layer shapes: one and sixteen tokens on the
+    streaming kernel, 2048 tokens on the tensor-core path; the same protocol as --case (CUDA graph, cold L2).  The
+    streaming kernel executes the same instructions per weight whatever the width, so these rows show how its time
+    follows the instruction count rather than the bytes."""
+    specs = []
+    for bits in (8, 2):
+        specs += [f"28672,8192,{bits},128,1,f16", f"11008,4096,{bits},128,1,f16", f"11008,4096,{bits},128,16,f16",
+                  f"11008,4096,{bits},128,2048,bf16"]
+    sub = argparse.Namespace(case=specs, case_copies=0, case_iters=max(3, args.prefill_iters // 4), case_stream=False)
+    return run_cases(sub, quiet=True)["cases"]
+
+
+def run_cases(args, quiet: bool = False):
     """--case N,K,bits,group,M,dtype[,frac] (repeatable): one synthetic layer per case, `copies` packed copies
     cycled through so that a launch does not find its weights in L2 (at least 256 MB between reuses unless
     --case-copies says otherwise).  Per case: microseconds per gwq_linear call, cold L2, replayed from a CUDA
@@ -798,7 +815,8 @@ def run_cases(args):
                      "copies": len(packed), "us": round(us_min, 3), "us_median": round(us_med, 3), "bytes": b,
                      "gbs": round(b / us_min / 1e3, 1), "frac_measured_peak": round(b / us_min / 1e3 / hbm_peak, 4),
                      "tflops": round(fl / us_min / 1e6, 2), "status": gwq.gwq_device_status(packed[0])})
-        print(json.dumps(rows[-1]), file=sys.stderr, flush=True)
+        if not quiet:
+            print(json.dumps(rows[-1]), file=sys.stderr, flush=True)
     return {"mode": "cases", "order": "stream" if args.case_stream else "cuda graph, cold L2", "peak_source": peak_src,
             "hbm_peak_gbs": hbm_peak, "cases": rows}
 
