@@ -18,8 +18,10 @@ pytestmark = pytest.mark.gpu
 FRAC, GROUP = 0.01, 128
 
 
-@pytest.mark.parametrize("N,K,bits,layer_index", [(11008, 4096, 4, 4), (4096, 11008, 3, 6)])
-def test_full_size_layer(N, K, bits, layer_index):
+@pytest.mark.parametrize("N,K,bits,layer_index,whole", [(11008, 4096, 4, 4, True), (4096, 11008, 3, 6, True),
+                                                         (11008, 4096, 8, 4, False), (4096, 11008, 2, 6, False)])
+def test_full_size_layer(N, K, bits, layer_index, whole):
+    # whole = False (the widths beside the paper's): the encoding, M = 1, 4, 16 and 2048 only
     W, G = synth.make_weight_and_grad(N, K, synth.layer_seed(1, layer_index))
     row_ptr, col_idx, val = orc.select_outliers(W, G, FRAC)
     Wd, Gd = to_dev(W), to_dev(G)
@@ -60,12 +62,15 @@ def test_full_size_layer(N, K, bits, layer_index):
         assert gwq.gwq_device_status(P) == 0
 
     # tensor-core path: bf16 activations with 8 heavy channels, as in the prefill cases; every output
-    for M in (512, 2048):
+    for M in ((512, 2048) if whole else (2048,)):
         bits16, xv = synth.make_activations(M, K, seed=900 + M, dtype="bf16", heavy_channels=8)
         y = gwq.gwq_linear(P, x_tensor(bits16, "bf16"), out_dtype=torch.float32)
         y_ref, bound = orc.linear(xv, w_hat)
         assert_linear_close(y, y_ref, bound)
         del y, y_ref, bound
+    if not whole:
+        assert gwq.gwq_device_status(P) == 0
+        return
     # M = 8192: all token rows on 256 distinct output rows, and 64 seeded token rows on every output row
     M = 8192
     bits16, xv = synth.make_activations(M, K, seed=900 + M, dtype="bf16", heavy_channels=8)
