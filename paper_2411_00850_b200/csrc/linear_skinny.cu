@@ -128,6 +128,11 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmc, const __grid_constant__ C
   const long long it0 = range_begin(p.total, gridDim.x, blockIdx.x), it1 = range_begin(p.total, gridDim.x, blockIdx.x + 1);
   const int nsteps = (int)(it1 - it0);
   const int G = p.G;
+  // tile and group of step j of this CTA with 32-bit arithmetic: a 64-bit division per step and role costs several
+  // hundred cycles of a single warp, which is what the step has
+  const unsigned tile0 = (unsigned)(it0 / G), grp0 = (unsigned)(it0 % G);
+  auto tile_of = [&](int j) { return (int)(tile0 + (grp0 + (unsigned)j) / (unsigned)G); };
+  auto grp_of = [&](int j) { return (int)((grp0 + (unsigned)j) % (unsigned)G); };
 
   if (tid == 0) {
     abort_s = 0;
@@ -180,16 +185,14 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmc, const __grid_constant__ C
       // the codes of the first stages do not depend on the previous kernel: they are requested before the wait
       const int pre = nsteps < kStages ? nsteps : kStages;
       for (int j = 0; j < pre && ok; ++j) {
-        const long long it = it0 + j;
-        const int tile = (int)(it / G), grp = (int)(it % G);
+        const int tile = tile_of(j), grp = grp_of(j);
         mbar_expect_tx(full(j), kCodeBytes + kXBytes);
         tma_load_2d(smem_u32(code_tile(j)), &tmc, grp * 4 * BITS, tile * kRows, full(j));
         issued = j + 1;
       }
       asm volatile("griddepcontrol.wait;" ::: "memory");
       for (int j = 0; j < nsteps && ok; ++j) {
-        const long long it = it0 + j;
-        const int tile = (int)(it / G), grp = (int)(it % G);
+        const int tile = tile_of(j), grp = grp_of(j);
         const int s = j % kStages;
         if (j >= kStages) {
           ok = mbar_wait(empty(s), ((j / kStages) - 1) & 1, abort_flag, lim);
@@ -209,7 +212,7 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmc, const __grid_constant__ C
       const unsigned idesc = (1u << 4) | ((unsigned)(TOK >> 3) << 17) | ((unsigned)(kRows >> 4) << 24);
       int piece = 0;
       for (int j = 0; j < nsteps && ok; ++j) {
-        const int grp = (int)((it0 + j) % G);
+        const int grp = grp_of(j);
         const int s = j % kStages, b = j % kSets;
         const bool first = j == 0 || grp == 0, last = j == nsteps - 1 || grp == G - 1;
         const int o = piece & 1;
@@ -323,8 +326,7 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmc, const __grid_constant__ C
     unsigned sz_ring[kAhead][AS];
     auto load_sz = [&](int j, unsigned (&dst)[AS]) {
       if (j < nsteps) {
-        const long long itn = it0 + j;
-        const int rown = (int)(itn / G) * kRows + r, grpn = (int)(itn % G);
+        const int rown = tile_of(j) * kRows + r, grpn = grp_of(j);
 #pragma unroll
         for (int h = 0; h < AS; ++h) dst[h] = __ldg(p.szt + (size_t)(grpn * AS + h) * p.N + (rown < p.N ? rown : p.N - 1));
       }
@@ -333,8 +335,7 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmc, const __grid_constant__ C
     for (int a = 0; a < kAhead; ++a) load_sz(a, sz_ring[a]);
     asm volatile("griddepcontrol.wait;" ::: "memory");   // y and the workspace may still be in use by the previous kernel
     for (int j = 0; j < nsteps && ok; ++j) {
-      const long long it = it0 + j;
-      const int tile = (int)(it / G), grp = (int)(it % G);
+      const int tile = tile_of(j), grp = grp_of(j);
       const int row = tile * kRows + r;
       const bool last = j == nsteps - 1 || grp == G - 1;
       const int xq = j % kXs;
@@ -390,7 +391,7 @@ skinny_kernel(const __grid_constant__ CUtensorMap tmc, const __grid_constant__ C
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         __syncwarp();
         if (lane == 0) mbar_arrive(o_empty(o));
-        const bool whole = grp == G - 1 && (head ? (it0 % G) == 0 : true) && (j + 1 >= G);   // the piece is the whole tile
+        const bool whole = grp == G - 1 && (head ? grp0 == 0u : true) && (j + 1 >= G);   // the piece is the whole tile
         if (whole) {
           if (row < p.N) {
 #pragma unroll
