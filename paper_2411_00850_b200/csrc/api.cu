@@ -23,7 +23,7 @@ static bool prefers_tensor_core(const gwq_packed* P, int M) {
 #ifndef GWQ_TUNE_SKINNY_MIN_M
 // fewest tokens that go to the tcgen05 streaming kernel when a workspace is given: its cost per step hardly depends on
 // the token count, the mma.sync kernel's grows with it; measured cross-over between 16 and 17 tokens (4 bit, 16 tokens:
-// 40 against 35 us on 8192 x 8192, 31 against 27 us on 11008 x 4096; 32 tokens: 52 against 70 us, 39 against 44 us)
+// 37 against 35 us on 8192 x 8192, 31 against 25 us on 11008 x 4096; 32 tokens: 37 against 70 us, 31 against 44 us)
 #define GWQ_TUNE_SKINNY_MIN_M 17
 #endif
 
