@@ -57,6 +57,12 @@ constexpr int kDequantGroups = 3;  // groups; group g takes the k-blocks g, g + 
 constexpr int kEpilogueWarps = 4;  // one thread per tile row
 constexpr int kCtaThreads = 32 * (2 + kDequantWarps * kDequantGroups + kEpilogueWarps);
 constexpr int kMaxStages = 8;   // of the fused kernel
+// stages of the fused kernel's ring for a token tile: what 219 KB hold, at most kMaxStages (a compile-time constant in
+// the kernel: the stage of a k-block is a remainder that every role takes per k-block)
+__host__ __device__ constexpr int fused_stages(int tok) {
+  return (220 * 1024 - 1024) / (128 * 64 * 2 + tok * 64 * 2) > kMaxStages ? kMaxStages
+                                                                           : (220 * 1024 - 1024) / (128 * 64 * 2 + tok * 64 * 2);
+}
 
 struct PrefillArgs {
   const uint32_t* codes;
@@ -167,7 +173,8 @@ __device__ __forceinline__ unsigned sub_magic(unsigned qm, unsigned zm) {
 template <int BITS, int TOK, bool BF16, int GPK>
 __global__ void __launch_bounds__(kCtaThreads, 1)
 prefill_kernel(const __grid_constant__ CUtensorMap tmx, const PrefillArgs p,
-               const int stages, const int ntn, const int ntiles) {
+               const int ntn, const int ntiles) {
+  constexpr int stages = fused_stages(TOK);
   constexpr int kABytes = kTileN * kBlockK * 2;   // 16 KB
   constexpr int kBBytes = TOK * kBlockK * 2;
   constexpr int kAccCols = TOK < 32 ? 32 : TOK;   // tensor-memory columns of one accumulator
@@ -1082,8 +1089,8 @@ gwq_status launch(const gwq_packed* P, const void* x, const float* tok_scale, in
       return GWQ_ERR_CUDA;
   }
   const int stage_bytes = kTileN * kBlockK * 2 + TOK * kBlockK * 2;
-  int stages = (220 * 1024 - 1024) / stage_bytes;
-  if (stages > kMaxStages) stages = kMaxStages;
+  static_assert(kTileN == 128 && kBlockK == 64, "fused_stages() is written for these tile sizes");
+  constexpr int stages = fused_stages(TOK);
   const size_t smem = (size_t)stages * stage_bytes + 1024;
   if (cudaFuncSetAttribute(prefill_kernel<BITS, TOK, BF16, GPK>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            (int)smem) != cudaSuccess)
@@ -1094,7 +1101,7 @@ gwq_status launch(const gwq_packed* P, const void* x, const float* tok_scale, in
   a.wait_cycles = pv->wait_cycles;
   const int ntn = (P->N + kTileN - 1) / kTileN, ntiles = ntn * ((M + TOK - 1) / TOK);
   const int grid = ntiles < pv->sm_count ? ntiles : pv->sm_count;   // persistent: at most one CTA per SM
-  prefill_kernel<BITS, TOK, BF16, GPK><<<grid, kCtaThreads, smem, stream>>>(tmx, a, stages, ntn, ntiles);
+  prefill_kernel<BITS, TOK, BF16, GPK><<<grid, kCtaThreads, smem, stream>>>(tmx, a, ntn, ntiles);
   return cudaGetLastError() == cudaSuccess ? GWQ_OK : GWQ_ERR_CUDA;
 }
 
