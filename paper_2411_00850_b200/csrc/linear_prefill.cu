@@ -279,6 +279,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmx, const PrefillArgs p,
     constexpr int WPB = kBlockK * BITS / 32;   // packed words per row per k-block (8 or 6)
     constexpr unsigned MAGIC = BF16 ? 0x43004300u : 0x64006400u;   // 128.0 / 1024.0: ulp = 1
     constexpr int kOutWin = 8;                 // outliers of the row kept this many entries ahead
+    const int gshift = __ffs(p.group) - 1;     // the group size is a power of two: no division per k-block
     for (int ti = 0; ti < my_tiles && ok; ++ti) {
       const int tile = blockIdx.x + ti * gridDim.x;
       const int row = (tile % ntn) * kTileN + r;
@@ -303,7 +304,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmx, const PrefillArgs p,
       if (kb < nkb) {
         load_words<WPB>(crow + (size_t)kb * WPB, wq);
 #pragma unroll
-        for (int g = 0; g < GPK; ++g) sz_nx[g] = __ldg(szcol + (size_t)((kb * kBlockK) / p.group + g) * p.N);
+        for (int g = 0; g < GPK; ++g) sz_nx[g] = __ldg(szcol + (size_t)(((kb * kBlockK) >> gshift) + g) * p.N);
       }
       for (; kb < nkb && ok; kb += G) {
         const int it = ti * nkb + kb, s = it % stages, round = it / stages;
@@ -328,7 +329,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmx, const PrefillArgs p,
         if (kb + G < nkb) {   // codes, scale and zero-point of this group's next k-block
           load_words<WPB>(crow + (size_t)(kb + G) * WPB, wq);
 #pragma unroll
-          for (int g = 0; g < GPK; ++g) sz_nx[g] = __ldg(szcol + (size_t)(((kb + G) * kBlockK) / p.group + g) * p.N);
+          for (int g = 0; g < GPK; ++g) sz_nx[g] = __ldg(szcol + (size_t)((((kb + G) * kBlockK) >> gshift) + g) * p.N);
         }
         // 64 codes -> 32 pairs (columns 2h, 2h+1) -> 8 chunks of 16 bytes
         unsigned out[32];
